@@ -1,0 +1,184 @@
+/*
+ * fastsgd.h -- C ABI of the B200 (sm_100a) FastSGD gradient codec.
+ *
+ * The calls follow the paper's statement of the problem (arxiv 2112.04291):
+ * a worker's gradient, read as key-value pairs (Sec. 2.2), goes through the
+ * gradient value encoder (Sec. 3.2, Eq. 2-3, Algorithm 1: reciprocal mapper,
+ * logarithm quantisation, threshold filter) and the gradient key encoder
+ * (Sec. 3.3, Eq. 4, Algorithm 2: delta keys, length flags, bit-level binary
+ * encoding); the decoder (Sec. 3.1, decoder phases 1-4) inverts both and the
+ * decoded gradients of the W workers are aggregated (Sec. 2.1).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses on the current
+ *     device, "host" pointers are ordinary process memory.
+ *   - The caller owns every buffer.  The library allocates nothing; its scratch
+ *     memory is the workspace the caller registers with fastsgd_set_workspace.
+ *   - fastsgd_compress and fastsgd_decompress_accumulate only enqueue kernels
+ *     on `stream` (a cudaStream_t passed as void*) and return at once.  All
+ *     calls that share a workspace must be issued on one stream (or otherwise
+ *     serialised): they share the workspace.
+ *   - Return value: 0 or a negative FASTSGD_E_* for what the host can see.
+ *     What only the device can see is reported in a status word: the stream
+ *     header's for compress (fastsgd_stream_info), the workspace's for
+ *     decompress (fastsgd_decode_status).
+ *   - There is no CPU fallback.
+ *
+ * Stream layout (little-endian; the paper fixes only that the codes travel
+ * with `sum` and the keys as the binary sequence BK):
+ *   header, 64 bytes: u32 magic "FSG1", u32 version, u32 status, u32 tau,
+ *     u64 n, u64 d, u64 total_bytes, f64 sum, f64 b, u8 l, u8 group_log2,
+ *     u16 0, u32 G
+ *   directory, G = ceil(n / 2^group_log2) entries: u32 count | M << 24,
+ *     u32 offset of the group's blob in 4-byte words from the stream start
+ *   blobs, in group order: count code bytes (bit 7 sign, bits 0-6 L-1), count
+ *     length flags of l bits, the deltas in the widths the flags select,
+ *     zero bits up to a multiple of 32; all fields most significant bit first.
+ *   Each group is one instance of Algorithm 2 over the kept keys that fall
+ *   in [g*T, (g+1)*T), T = 2^group_log2, with preKey starting at g*T.
+ *   When status != 0 only the header is defined (d = 0, total_bytes = 64).
+ */
+#ifndef FASTSGD_H
+#define FASTSGD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Hyper-parameters (Sec. 4.2 recommends b ~ 1.1, tau = 128, l = 2). */
+typedef struct fastsgd_params {
+    double   base;        /* b > 1, with b^tau finite (Eq. 3)                        */
+    uint32_t tau;         /* threshold, 1..128: kept codes L satisfy 1 <= L <= tau    */
+    uint32_t flag_bits;   /* l, 1..5: size of the length flag (Sec. 3.3, Phase 5)     */
+    uint32_t group_log2;  /* log2 of the group size T; this build supports 14        */
+    uint32_t reserved;    /* must be 0                                               */
+} fastsgd_params;
+
+/* host-visible errors (return values) */
+#define FASTSGD_OK                 0
+#define FASTSGD_E_NULL            (-1)
+#define FASTSGD_E_ALIGN           (-2)   /* grad / out / stream_in not 16-byte aligned, dense_out not 4-byte */
+#define FASTSGD_E_BAD_PARAM       (-3)
+#define FASTSGD_E_BAD_N           (-4)   /* n = 0 or n >= 2^31                                                */
+#define FASTSGD_E_CAPACITY        (-5)   /* out_bytes smaller than header + directory                        */
+#define FASTSGD_E_NO_WORKSPACE    (-6)   /* no workspace registered, or too small for this n                 */
+#define FASTSGD_E_NOT_IMPLEMENTED (-7)   /* valid parameters this build has no kernel for                    */
+#define FASTSGD_E_CUDA            (-8)   /* a CUDA runtime call failed                                       */
+#define FASTSGD_E_TRUNCATED       (-9)   /* decompress: fewer than 64 bytes given                            */
+
+/* device-visible status words */
+#define FASTSGD_ST_OK              0
+#define FASTSGD_ST_NONFINITE       1     /* compress: sum of |v| is Inf or NaN                               */
+#define FASTSGD_ST_CAPACITY        2     /* compress: stream does not fit in out_bytes                       */
+#define FASTSGD_ST_TIMEOUT         3     /* compress: a bounded wait between thread blocks ran out           */
+#define FASTSGD_ST_BAD_MAGIC      16
+#define FASTSGD_ST_BAD_VERSION    17
+#define FASTSGD_ST_BAD_STATUS     18     /* decompress: the stream's own status is not OK                    */
+#define FASTSGD_ST_N_MISMATCH     19
+#define FASTSGD_ST_PARAM_MISMATCH 20
+#define FASTSGD_ST_TRUNCATED      21
+#define FASTSGD_ST_BAD_DIRECTORY  22
+#define FASTSGD_ST_BAD_KEY        23     /* a decoded key leaves its group or repeats                        */
+#define FASTSGD_ST_BAD_CODE       24     /* a code byte with L > tau                                         */
+
+/*
+ * Encoder (Sec. 3.2 Algorithm 1 followed by Sec. 3.3 Algorithm 2).
+ *   grad       device, n floats, 16-byte aligned; read twice, never written
+ *   n          number of gradient entries D_m, 1 <= n < 2^31
+ *   params     host
+ *   out        device, 16-byte aligned, receives the stream
+ *   out_bytes  capacity of `out` in bytes (by value); at least
+ *              64 + 8*G; fastsgd_compress_bound(n, params) always suffices.
+ *              The produced length is header.total_bytes (device memory;
+ *              fastsgd_stream_info reads it back).
+ *   stream     cudaStream_t
+ * Computes sum = sum|v_i| on a fixed fp64 pairwise tree, the boundaries
+ * B_k = sum / b^k, keeps entry i iff |v_i| >= B_tau (the early-stop threshold
+ * tau_e), gives it the code L = min{k : |v_i| >= B_k} = ceil(log_b(sum/|v_i|))
+ * (raised to 1 if 0) with the sign of v_i, and writes the stream.
+ * If the stream does not fit, or the sum is not finite, only a 64-byte header
+ * carrying the status is written.  Nothing outside out[0, out_bytes) is
+ * written.
+ */
+int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
+                     void* out, uint64_t out_bytes, void* stream);
+
+/*
+ * Decoder and aggregation (Sec. 3.1 decoder phases 1-4; Sec. 2.1 aggregation).
+ *   stream_in  device, 16-byte aligned, a stream made by fastsgd_compress
+ *   bytes      number of valid bytes at stream_in (>= header.total_bytes)
+ *   n, params  must equal the header's, else FASTSGD_ST_N_MISMATCH /
+ *              FASTSGD_ST_PARAM_MISMATCH
+ *   dense_out  device, n floats: dense_out[k] += sign * (float)(sum / b^L) for
+ *              every kept (k, L); never cleared, so that the streams of several
+ *              workers add up in call order
+ * A damaged stream never causes an access outside stream_in[0, bytes) or
+ * dense_out[0, n); its status is recorded (fastsgd_decode_status) and the
+ * contents of dense_out are then unspecified.  Header-level damage leaves
+ * dense_out untouched.
+ */
+int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
+                                  const fastsgd_params* params, float* dense_out, void* stream);
+
+/* ---- helpers, not on the timed path (no counterpart in the paper) ---------- */
+
+/* worst-case stream size in bytes (every entry kept, every delta at the widest
+ * level); 0 for invalid arguments */
+uint64_t fastsgd_compress_bound(uint64_t n, const fastsgd_params* params);
+
+/* bytes of device scratch the two calls need for gradients of up to n entries */
+uint64_t fastsgd_workspace_bytes(uint64_t n, const fastsgd_params* params);
+
+/* Registers caller-owned device memory (256-byte aligned) as the library's
+ * scratch and initialises it on `stream`.  The memory must stay valid until
+ * another workspace is registered. */
+int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream);
+
+/* Synchronises `stream`, then copies total_bytes, d and status out of a
+ * stream's header (any pointer may be NULL). */
+int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_bytes,
+                        uint64_t* d, int* status);
+
+/* Synchronises `stream`, returns in *status the status of the decompress calls
+ * since the last query (FASTSGD_ST_OK if none failed; else that of the lowest
+ * damaged group seen), and clears it. */
+int fastsgd_decode_status(void* stream, int* status);
+
+/* Step 1 of Algorithm 1 alone: *sum_out (device, one double) = sum|v_i| on the
+ * same fp64 pairwise tree fastsgd_compress uses.  Uses the workspace. */
+int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream);
+
+/*
+ * Host-buffer forms of the two calls, for callers whose gradients live in host
+ * memory: copy in, run the device path, copy the result out, all on `stream`,
+ * then synchronise.  `dev_scratch` is caller-owned device memory of at least
+ * fastsgd_host_scratch_bytes(n, params) bytes (16-byte aligned).
+ *   fastsgd_compress_host: grad_host (n floats) -> out_host (capacity
+ *     out_bytes); *produced = bytes written to out_host; *status = header status.
+ *   fastsgd_decompress_accumulate_host: decodes `num_streams` streams (host
+ *     pointers streams_host[i] of bytes[i] bytes each, in that order) into one
+ *     dense vector and copies it to dense_host (n floats).  accumulate = 0
+ *     starts from zero, accumulate = 1 from dense_host's contents.
+ *     *status = decoder status.
+ */
+uint64_t fastsgd_host_scratch_bytes(uint64_t n, const fastsgd_params* params);
+int fastsgd_compress_host(const float* grad_host, uint64_t n, const fastsgd_params* params,
+                          void* out_host, uint64_t out_bytes, uint64_t* produced, int* status,
+                          void* dev_scratch, uint64_t dev_scratch_bytes, void* stream);
+int fastsgd_decompress_accumulate_host(const void* const* streams_host, const uint64_t* bytes,
+                                       uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                       float* dense_host, int accumulate, int* status,
+                                       void* dev_scratch, uint64_t dev_scratch_bytes, void* stream);
+
+/* number of kernels the library has launched since it was loaded */
+uint64_t fastsgd_launch_count(void);
+
+const char* fastsgd_strerror(int code);
+int fastsgd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTSGD_H */

@@ -1,0 +1,201 @@
+"""Thin ctypes binding of ``libfastsgd_b200.so`` (same names as ``include/fastsgd.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch supplies device memory and streams.  Loading fails loudly if the library has not
+been built; there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libfastsgd_b200.so")
+
+OK = 0
+E_NULL, E_ALIGN, E_BAD_PARAM, E_BAD_N, E_CAPACITY, E_NO_WORKSPACE, E_NOT_IMPLEMENTED, E_CUDA, E_TRUNCATED = range(-1, -10, -1)
+ST_OK, ST_NONFINITE, ST_CAPACITY, ST_TIMEOUT = 0, 1, 2, 3
+ST_BAD_MAGIC, ST_BAD_VERSION, ST_BAD_STATUS, ST_N_MISMATCH, ST_PARAM_MISMATCH = 16, 17, 18, 19, 20
+ST_TRUNCATED, ST_BAD_DIRECTORY, ST_BAD_KEY, ST_BAD_CODE = 21, 22, 23, 24
+
+EXPORTS = [
+    "fastsgd_compress", "fastsgd_decompress_accumulate", "fastsgd_compress_bound",
+    "fastsgd_workspace_bytes", "fastsgd_set_workspace", "fastsgd_stream_info",
+    "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
+    "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
+    "fastsgd_strerror", "fastsgd_version",
+]
+
+
+class Params(C.Structure):
+    _fields_ = [("base", C.c_double), ("tau", C.c_uint32), ("flag_bits", C.c_uint32),
+                ("group_log2", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+def params(base: float, tau: int = 128, flag_bits: int = 2, group_log2: int = 14) -> Params:
+    return Params(float(base), int(tau), int(flag_bits), int(group_log2), 0)
+
+
+class FastSGDError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it was not built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2112_04291_b200.build` "
+                "(needs nvcc; there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, u64, PP = C.c_void_p, C.c_uint64, C.POINTER(Params)
+        u64p, intp = C.POINTER(C.c_uint64), C.POINTER(C.c_int)
+        L.fastsgd_compress.restype = C.c_int
+        L.fastsgd_compress.argtypes = [vp, u64, PP, vp, u64, vp]
+        L.fastsgd_decompress_accumulate.restype = C.c_int
+        L.fastsgd_decompress_accumulate.argtypes = [vp, u64, u64, PP, vp, vp]
+        L.fastsgd_compress_bound.restype = u64
+        L.fastsgd_compress_bound.argtypes = [u64, PP]
+        L.fastsgd_workspace_bytes.restype = u64
+        L.fastsgd_workspace_bytes.argtypes = [u64, PP]
+        L.fastsgd_set_workspace.restype = C.c_int
+        L.fastsgd_set_workspace.argtypes = [vp, u64, vp]
+        L.fastsgd_stream_info.restype = C.c_int
+        L.fastsgd_stream_info.argtypes = [vp, vp, u64p, u64p, intp]
+        L.fastsgd_decode_status.restype = C.c_int
+        L.fastsgd_decode_status.argtypes = [vp, intp]
+        L.fastsgd_abs_sum.restype = C.c_int
+        L.fastsgd_abs_sum.argtypes = [vp, u64, vp, vp]
+        L.fastsgd_host_scratch_bytes.restype = u64
+        L.fastsgd_host_scratch_bytes.argtypes = [u64, PP]
+        L.fastsgd_compress_host.restype = C.c_int
+        L.fastsgd_compress_host.argtypes = [vp, u64, PP, vp, u64, u64p, intp, vp, u64, vp]
+        L.fastsgd_decompress_accumulate_host.restype = C.c_int
+        L.fastsgd_decompress_accumulate_host.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, C.c_int, intp, vp, u64, vp]
+        L.fastsgd_launch_count.restype = u64
+        L.fastsgd_launch_count.argtypes = []
+        L.fastsgd_strerror.restype = C.c_char_p
+        L.fastsgd_strerror.argtypes = [C.c_int]
+        L.fastsgd_version.restype = C.c_int
+        L.fastsgd_version.argtypes = []
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().fastsgd_strerror(int(code)).decode()
+
+
+def _stream_handle(stream=None) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise FastSGDError(rc, where)
+
+
+def compress_bound(n: int, p: Params) -> int:
+    return int(lib().fastsgd_compress_bound(n, C.byref(p)))
+
+
+def workspace_bytes(n: int, p: Params) -> int:
+    return int(lib().fastsgd_workspace_bytes(n, C.byref(p)))
+
+
+_workspace_keepalive = None
+
+
+def set_workspace(ws: torch.Tensor, stream=None) -> None:
+    """Registers a uint8 CUDA tensor as the library's scratch (kept alive here)."""
+    global _workspace_keepalive
+    assert ws.is_cuda and ws.dtype == torch.uint8 and ws.is_contiguous()
+    _check(lib().fastsgd_set_workspace(ws.data_ptr(), ws.numel(), _stream_handle(stream)), "fastsgd_set_workspace")
+    _workspace_keepalive = ws
+
+
+def ensure_workspace(n: int, p: Params, device="cuda") -> torch.Tensor:
+    """Allocates (torch) and registers a workspace large enough for n entries, if needed."""
+    need = workspace_bytes(n, p)
+    ws = _workspace_keepalive
+    if ws is None or ws.numel() < need or ws.device != torch.device(device, torch.cuda.current_device()):
+        ws = torch.empty(max(need, 4096), dtype=torch.uint8, device=device)
+        set_workspace(ws)
+    return ws
+
+
+def compress(grad: torch.Tensor, p: Params, out: torch.Tensor, stream=None) -> int:
+    """fastsgd_compress: enqueues the encoder; returns the host-visible return code."""
+    assert grad.is_cuda and grad.dtype == torch.float32 and grad.is_contiguous()
+    assert out.is_cuda and out.dtype == torch.uint8 and out.is_contiguous()
+    return lib().fastsgd_compress(grad.data_ptr(), grad.numel(), C.byref(p), out.data_ptr(), out.numel(),
+                                  _stream_handle(stream))
+
+
+def decompress_accumulate(stream_in: torch.Tensor, nbytes: int, n: int, p: Params, dense: torch.Tensor,
+                          stream=None) -> int:
+    assert stream_in.is_cuda and stream_in.dtype == torch.uint8
+    assert dense.is_cuda and dense.dtype == torch.float32 and dense.is_contiguous() and dense.numel() == n
+    return lib().fastsgd_decompress_accumulate(stream_in.data_ptr(), int(nbytes), int(n), C.byref(p),
+                                               dense.data_ptr(), _stream_handle(stream))
+
+
+def stream_info(stream_in: torch.Tensor, stream=None):
+    """(total_bytes, d, status) of a stream's header; synchronises."""
+    tb, d, st = C.c_uint64(0), C.c_uint64(0), C.c_int(0)
+    _check(lib().fastsgd_stream_info(stream_in.data_ptr(), _stream_handle(stream), C.byref(tb), C.byref(d),
+                                     C.byref(st)), "fastsgd_stream_info")
+    return tb.value, d.value, st.value
+
+
+def decode_status(stream=None) -> int:
+    st = C.c_int(0)
+    _check(lib().fastsgd_decode_status(_stream_handle(stream), C.byref(st)), "fastsgd_decode_status")
+    return st.value
+
+
+def abs_sum(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int:
+    assert grad.is_cuda and grad.dtype == torch.float32 and out.is_cuda and out.dtype == torch.float64
+    return lib().fastsgd_abs_sum(grad.data_ptr(), grad.numel(), out.data_ptr(), _stream_handle(stream))
+
+
+def host_scratch_bytes(n: int, p: Params) -> int:
+    return int(lib().fastsgd_host_scratch_bytes(n, C.byref(p)))
+
+
+def compress_host(grad_host: torch.Tensor, p: Params, out_host: torch.Tensor, scratch: torch.Tensor, stream=None):
+    """Host-buffer encoder -> (return code, produced bytes, header status)."""
+    assert not grad_host.is_cuda and grad_host.dtype == torch.float32 and grad_host.is_contiguous()
+    assert not out_host.is_cuda and out_host.dtype == torch.uint8 and scratch.is_cuda
+    produced, st = C.c_uint64(0), C.c_int(0)
+    rc = lib().fastsgd_compress_host(grad_host.data_ptr(), grad_host.numel(), C.byref(p), out_host.data_ptr(),
+                                     out_host.numel(), C.byref(produced), C.byref(st), scratch.data_ptr(),
+                                     scratch.numel(), _stream_handle(stream))
+    return rc, produced.value, st.value
+
+
+def decompress_accumulate_host(streams_host, nbytes, n: int, p: Params, dense_host: torch.Tensor,
+                               scratch: torch.Tensor, accumulate: bool = False, stream=None):
+    """Host-buffer decoder + aggregation of several streams -> (return code, decoder status)."""
+    assert not dense_host.is_cuda and dense_host.dtype == torch.float32 and dense_host.numel() == n
+    k = len(streams_host)
+    ptrs = (C.c_void_p * k)(*[int(s.data_ptr()) for s in streams_host])
+    sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
+    st = C.c_int(0)
+    rc = lib().fastsgd_decompress_accumulate_host(ptrs, sizes, k, int(n), C.byref(p), dense_host.data_ptr(),
+                                                  int(bool(accumulate)), C.byref(st), scratch.data_ptr(),
+                                                  scratch.numel(), _stream_handle(stream))
+    return rc, st.value
+
+
+def launch_count() -> int:
+    return int(lib().fastsgd_launch_count())

@@ -1,0 +1,348 @@
+// C-ABI shim: argument checks, workspace bookkeeping and kernel launches on the caller's
+// stream.  No computation of the path happens here except the parameter-only table b^k.
+#include "../../include/fastsgd.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "sum.cuh"
+#include "encode.cuh"
+#include "decode.cuh"
+
+namespace {
+
+using namespace fsg;
+
+struct State {
+    std::mutex mu;
+    void*      ws = nullptr;
+    uint64_t   ws_bytes = 0;
+    int        device = -1;
+    int        sm_count = 0;
+    int        sum_blocks_per_sm = 0;
+    int        dec_blocks_per_sm = 0;
+    bool       attrs_set = false;
+};
+State g_state;
+std::atomic<uint64_t> g_launches{0};
+
+int check_params(const fastsgd_params* p, PowTable* pw) {
+    if (!p) return FASTSGD_E_NULL;
+    if (!(p->base > 1.0) || !std::isfinite(p->base)) return FASTSGD_E_BAD_PARAM;
+    if (p->tau < 1 || p->tau > (uint32_t)kMaxTau) return FASTSGD_E_BAD_PARAM;
+    if (p->flag_bits < 1 || p->flag_bits > 5) return FASTSGD_E_BAD_PARAM;
+    if (p->group_log2 < 1 || p->group_log2 > 20) return FASTSGD_E_BAD_PARAM;
+    if (p->reserved != 0) return FASTSGD_E_BAD_PARAM;
+    PowTable local;
+    PowTable& t = pw ? *pw : local;
+    volatile double acc = 1.0;            // one rounded fp64 product per step
+    t.P[0] = 1.0;
+    for (uint32_t k = 1; k <= (uint32_t)kMaxTau; ++k) {
+        if (k <= p->tau) { acc = acc * p->base; t.P[k] = acc; }
+        else t.P[k] = t.P[p->tau];
+    }
+    if (!std::isfinite(t.P[p->tau])) return FASTSGD_E_BAD_PARAM;
+    if (p->group_log2 != (uint32_t)kGroupLog2) return FASTSGD_E_NOT_IMPLEMENTED;
+    return FASTSGD_OK;
+}
+
+int check_n(uint64_t n) { return (n == 0 || n >= (1ull << 31)) ? FASTSGD_E_BAD_N : FASTSGD_OK; }
+
+uint64_t groups_of(uint64_t n, uint32_t group_log2) { return (n + (1ull << group_log2) - 1) >> group_log2; }
+uint64_t chunks_of(uint64_t n) { return (n + kChunk - 1) >> kChunkLog2; }
+
+uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
+    const uint64_t T = 1ull << p->group_log2, G = groups_of(n, p->group_log2);
+    const uint64_t per_group_words = (T * (8ull + p->flag_bits + p->group_log2) + 31ull) / 32ull;
+    return kHeaderBytes + 8ull * G + 4ull * G * per_group_words;
+}
+
+uint64_t ws_bytes_for(uint64_t n, uint32_t group_log2) {
+    const uint64_t b = kPartialsOffset + 8ull * chunks_of(n) + 8ull * groups_of(n, group_log2);
+    return (b + 255ull) & ~255ull;
+}
+
+WorkspaceView view(void* ws, uint64_t n) {
+    WorkspaceView v;
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    v.ctl = reinterpret_cast<Control*>(base);
+    v.thr = reinterpret_cast<float*>(base + kThrOffset);
+    v.partials = reinterpret_cast<double*>(base + kPartialsOffset);
+    v.desc = reinterpret_cast<unsigned long long*>(base + kPartialsOffset + 8ull * chunks_of(n));
+    return v;
+}
+
+int ensure_device_setup() {
+    // caller holds g_state.mu
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (g_state.attrs_set && g_state.device == dev) return FASTSGD_OK;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EncSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    int b1 = 0, b2 = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, k_decode_accumulate, kDecThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
+    g_state.device = dev;
+    g_state.sm_count = sms;
+    g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
+    g_state.dec_blocks_per_sm = b2 > 0 ? b2 : 1;
+    g_state.attrs_set = true;
+    return FASTSGD_OK;
+}
+
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int launch_sum(const float* grad, uint64_t n, uint32_t groups, uint32_t tau, const PowTable& pw,
+               const WorkspaceView& w, double* sum_out, cudaStream_t st) {
+    SumArgs sa;
+    sa.grad = grad; sa.n = n; sa.chunks = (uint32_t)chunks_of(n); sa.groups = groups; sa.tau = tau;
+    sa.ctl = w.ctl; sa.thr = w.thr; sa.partials = w.partials; sa.desc = w.desc; sa.sum_out = sum_out;
+    uint64_t grid = (uint64_t)g_state.sm_count * g_state.sum_blocks_per_sm;
+    if (grid > sa.chunks) grid = sa.chunks;
+    k_abs_sum<<<(unsigned)grid, kSumThreads, 0, st>>>(sa, pw);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fastsgd_version(void) { return 1; }
+
+uint64_t fastsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* fastsgd_strerror(int code) {
+    switch (code) {
+        case FASTSGD_OK: return "ok";
+        case FASTSGD_E_NULL: return "null pointer argument";
+        case FASTSGD_E_ALIGN: return "pointer not aligned as required";
+        case FASTSGD_E_BAD_PARAM: return "invalid parameters";
+        case FASTSGD_E_BAD_N: return "n must satisfy 1 <= n < 2^31";
+        case FASTSGD_E_CAPACITY: return "output capacity smaller than header + directory";
+        case FASTSGD_E_NO_WORKSPACE: return "no workspace registered or workspace too small";
+        case FASTSGD_E_NOT_IMPLEMENTED: return "parameter combination not implemented in this build";
+        case FASTSGD_E_CUDA: return "CUDA runtime error";
+        case FASTSGD_E_TRUNCATED: return "stream shorter than its header";
+        case FASTSGD_ST_NONFINITE: return "sum of |v| is not finite";
+        case FASTSGD_ST_CAPACITY: return "stream does not fit in the output buffer";
+        case FASTSGD_ST_TIMEOUT: return "bounded wait between thread blocks ran out";
+        case FASTSGD_ST_BAD_MAGIC: return "bad magic";
+        case FASTSGD_ST_BAD_VERSION: return "bad version";
+        case FASTSGD_ST_BAD_STATUS: return "stream carries an error status";
+        case FASTSGD_ST_N_MISMATCH: return "n differs from the header";
+        case FASTSGD_ST_PARAM_MISMATCH: return "parameters differ from the header";
+        case FASTSGD_ST_TRUNCATED: return "stream truncated";
+        case FASTSGD_ST_BAD_DIRECTORY: return "inconsistent directory";
+        case FASTSGD_ST_BAD_KEY: return "decoded key out of range";
+        case FASTSGD_ST_BAD_CODE: return "code byte out of range";
+        default: return "unknown code";
+    }
+}
+
+uint64_t fastsgd_compress_bound(uint64_t n, const fastsgd_params* params) {
+    int rc = check_params(params, nullptr);
+    if ((rc != FASTSGD_OK && rc != FASTSGD_E_NOT_IMPLEMENTED) || n == 0) return 0;
+    return bound_bytes(n, params);
+}
+
+uint64_t fastsgd_workspace_bytes(uint64_t n, const fastsgd_params* params) {
+    int rc = check_params(params, nullptr);
+    if ((rc != FASTSGD_OK && rc != FASTSGD_E_NOT_IMPLEMENTED) || n == 0) return 0;
+    return ws_bytes_for(n, params->group_log2);
+}
+
+int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
+    if (!dev_ptr) return FASTSGD_E_NULL;
+    if (!aligned(dev_ptr, 256)) return FASTSGD_E_ALIGN;
+    if (bytes < kPartialsOffset) return FASTSGD_E_NO_WORKSPACE;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    int rc = ensure_device_setup();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(dev_ptr, 0, kPartialsOffset, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaMemsetAsync(static_cast<unsigned char*>(dev_ptr) + offsetof(Control, decode_status), 0xFF, 8, st) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    g_state.ws = dev_ptr;
+    g_state.ws_bytes = bytes;
+    return FASTSGD_OK;
+}
+
+int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream) {
+    if (!grad || !sum_out) return FASTSGD_E_NULL;
+    if (!aligned(grad, 16) || !aligned(sum_out, 8)) return FASTSGD_E_ALIGN;
+    int rc = check_n(n);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, kGroupLog2)) return FASTSGD_E_NO_WORKSPACE;
+    rc = ensure_device_setup();
+    if (rc) return rc;
+    PowTable pw;
+    for (int k = 0; k <= kMaxTau; ++k) pw.P[k] = 1.0;
+    return launch_sum(grad, n, 0u, 0u, pw, view(g_state.ws, n), sum_out, static_cast<cudaStream_t>(stream));
+}
+
+int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
+                     void* out, uint64_t out_bytes, void* stream) {
+    if (!grad || !out || !params) return FASTSGD_E_NULL;
+    if (!aligned(grad, 16) || !aligned(out, 16)) return FASTSGD_E_ALIGN;
+    PowTable pw;
+    int rc = check_params(params, &pw);
+    if (rc) return rc;
+    rc = check_n(n);
+    if (rc) return rc;
+    const uint64_t G = groups_of(n, params->group_log2);
+    if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
+    if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;   // look-back fields are 31 bits
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
+    rc = ensure_device_setup();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    WorkspaceView w = view(g_state.ws, n);
+
+    rc = launch_sum(grad, n, (uint32_t)G, params->tau, pw, w, nullptr, st);
+    if (rc) return rc;
+
+    EncArgs ea;
+    ea.grad = grad; ea.n = n; ea.out = static_cast<uint8_t*>(out); ea.out_bytes = out_bytes;
+    ea.ctl = w.ctl; ea.thr = w.thr; ea.desc = w.desc; ea.base = params->base;
+    ea.G = (uint32_t)G; ea.tau = params->tau; ea.l = params->flag_bits;
+    k_encode<<<(unsigned)G, kEncThreads, sizeof(EncSmem), st>>>(ea);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+}
+
+int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
+                                  const fastsgd_params* params, float* dense_out, void* stream) {
+    if (!stream_in || !dense_out || !params) return FASTSGD_E_NULL;
+    if (!aligned(stream_in, 16) || !aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
+    PowTable pw;
+    int rc = check_params(params, &pw);
+    if (rc) return rc;
+    rc = check_n(n);
+    if (rc) return rc;
+    if (bytes < kHeaderBytes) return FASTSGD_E_TRUNCATED;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    if (!g_state.ws) return FASTSGD_E_NO_WORKSPACE;
+    rc = ensure_device_setup();
+    if (rc) return rc;
+    const uint64_t G = groups_of(n, params->group_log2);
+    DecArgs da;
+    da.stream = static_cast<const uint8_t*>(stream_in); da.bytes = bytes; da.n = n; da.dense = dense_out;
+    da.status = &view(g_state.ws, n).ctl->decode_status;
+    da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
+    da.group_log2 = params->group_log2;
+    const int warps_per_block = kDecThreads / 32;
+    uint64_t grid = (G + warps_per_block - 1) / warps_per_block;
+    const uint64_t cap = (uint64_t)g_state.sm_count * g_state.dec_blocks_per_sm;
+    if (grid > cap) grid = cap;
+    k_decode_accumulate<<<(unsigned)grid, kDecThreads, 0, static_cast<cudaStream_t>(stream)>>>(da, pw);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+}
+
+int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_bytes, uint64_t* d, int* status) {
+    if (!stream_in) return FASTSGD_E_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char h[kHeaderBytes];
+    if (cudaMemcpyAsync(h, stream_in, kHeaderBytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
+    uint32_t s32; uint64_t v;
+    if (status) { std::memcpy(&s32, h + 8, 4); *status = (int)s32; }
+    if (d) { std::memcpy(&v, h + 24, 8); *d = v; }
+    if (total_bytes) { std::memcpy(&v, h + 32, 8); *total_bytes = v; }
+    return FASTSGD_OK;
+}
+
+int fastsgd_decode_status(void* stream, int* status) {
+    if (!status) return FASTSGD_E_NULL;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    if (!g_state.ws) return FASTSGD_E_NO_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long v = 0;
+    unsigned char* p = static_cast<unsigned char*>(g_state.ws) + offsetof(Control, decode_status);
+    if (cudaMemcpyAsync(&v, p, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
+    *status = (v == ~0ull) ? FASTSGD_ST_OK : (int)(v & 0xFFull);
+    if (v != ~0ull) {
+        if (cudaMemsetAsync(p, 0xFF, 8, st) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
+    }
+    return FASTSGD_OK;
+}
+
+uint64_t fastsgd_host_scratch_bytes(uint64_t n, const fastsgd_params* params) {
+    const uint64_t b = fastsgd_compress_bound(n, params);
+    if (!b) return 0;
+    return ((4ull * n + 255ull) & ~255ull) + ((b + 255ull) & ~255ull);
+}
+
+int fastsgd_compress_host(const float* grad_host, uint64_t n, const fastsgd_params* params,
+                          void* out_host, uint64_t out_bytes, uint64_t* produced, int* status,
+                          void* dev_scratch, uint64_t dev_scratch_bytes, void* stream) {
+    if (!grad_host || !out_host || !dev_scratch || !params) return FASTSGD_E_NULL;
+    if (!aligned(dev_scratch, 16)) return FASTSGD_E_ALIGN;
+    const uint64_t need = fastsgd_host_scratch_bytes(n, params);
+    if (!need) return FASTSGD_E_BAD_PARAM;
+    if (dev_scratch_bytes < need) return FASTSGD_E_NO_WORKSPACE;
+    if (out_bytes < kHeaderBytes) return FASTSGD_E_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* dgrad = static_cast<float*>(dev_scratch);
+    unsigned char* dout = static_cast<unsigned char*>(dev_scratch) + ((4ull * n + 255ull) & ~255ull);
+    const uint64_t bound = fastsgd_compress_bound(n, params);
+    const uint64_t cap = out_bytes < bound ? out_bytes : bound;
+    if (cudaMemcpyAsync(dgrad, grad_host, 4ull * n, cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    int rc = fastsgd_compress(dgrad, n, params, dout, cap, stream);
+    if (rc) return rc;
+    uint64_t total = 0; int hst = 0;
+    rc = fastsgd_stream_info(dout, stream, &total, nullptr, &hst);
+    if (rc) return rc;
+    if (total > cap) return FASTSGD_E_CUDA;
+    if (cudaMemcpyAsync(out_host, dout, total, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (produced) *produced = total;
+    if (status) *status = hst;
+    return FASTSGD_OK;
+}
+
+int fastsgd_decompress_accumulate_host(const void* const* streams_host, const uint64_t* bytes,
+                                       uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                       float* dense_host, int accumulate, int* status,
+                                       void* dev_scratch, uint64_t dev_scratch_bytes, void* stream) {
+    if (!streams_host || !bytes || !dense_host || !dev_scratch || !params) return FASTSGD_E_NULL;
+    if (!aligned(dev_scratch, 16)) return FASTSGD_E_ALIGN;
+    const uint64_t need = fastsgd_host_scratch_bytes(n, params);
+    if (!need) return FASTSGD_E_BAD_PARAM;
+    const uint64_t dense_bytes = (4ull * n + 255ull) & ~255ull;
+    if (dev_scratch_bytes < need) return FASTSGD_E_NO_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* ddense = static_cast<float*>(dev_scratch);
+    unsigned char* dstream = static_cast<unsigned char*>(dev_scratch) + dense_bytes;
+    if (accumulate) {
+        if (cudaMemcpyAsync(ddense, dense_host, 4ull * n, cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    } else {
+        if (cudaMemsetAsync(ddense, 0, 4ull * n, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    }
+    for (uint32_t i = 0; i < num_streams; ++i) {
+        if (!streams_host[i]) return FASTSGD_E_NULL;
+        if (bytes[i] > need - dense_bytes) return FASTSGD_E_NO_WORKSPACE;
+        // the staging area is reused: stream order keeps copy i+1 behind decode i
+        if (cudaMemcpyAsync(dstream, streams_host[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
+        int rc = fastsgd_decompress_accumulate(dstream, bytes[i], n, params, ddense, stream);
+        if (rc) return rc;
+    }
+    if (cudaMemcpyAsync(dense_host, ddense, 4ull * n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    int dst = 0;
+    int rc = fastsgd_decode_status(stream, &dst);
+    if (rc) return rc;
+    if (status) *status = dst;
+    return FASTSGD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,87 @@
+// Shared definitions of the CUDA side: stream constants, the workspace layout and small
+// device helpers.  sm_100a only.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fsg {
+
+constexpr uint32_t kMagic       = 0x31475346u;   // "FSG1"
+constexpr uint32_t kVersion     = 1u;
+constexpr uint32_t kHeaderBytes = 64u;
+constexpr int      kMaxTau      = 128;
+
+// The sum tree is cut into aligned chunks of 2^14 entries: one fp64 partial per chunk.
+constexpr int      kChunkLog2   = 14;
+constexpr uint32_t kChunk       = 1u << kChunkLog2;
+
+constexpr int kStOk = 0, kStNonfinite = 1, kStCapacity = 2, kStTimeout = 3;
+constexpr int kStBadMagic = 16, kStBadVersion = 17, kStBadStatus = 18, kStNMismatch = 19,
+              kStParamMismatch = 20, kStTruncated = 21, kStBadDirectory = 22, kStBadKey = 23,
+              kStBadCode = 24;
+
+// b^k, k = 0..tau, by the recurrence P_k = P_{k-1} * b in fp64 (a function of the
+// parameters alone; passed to the kernels by value).
+struct PowTable {
+    double P[kMaxTau + 1];
+};
+
+// Control block at the start of the workspace.
+struct Control {
+    unsigned int       done;           // blocks of the sum kernel that have finished (self-resetting)
+    unsigned int       ticket;         // next group for the encode kernel
+    unsigned int       error;          // encode: non-zero once a bounded wait ran out
+    unsigned int       skip;           // 0 encode normally, 1 sum == 0, 2 sum not finite
+    unsigned long long decode_status;  // min over failures of (group << 32 | key index << 8 | status)
+    double             sum;            // S
+    unsigned int       pad[56];
+};
+static_assert(sizeof(Control) == 256, "control block is 256 bytes");
+
+constexpr uint64_t kThrOffset      = 256;    // float thr[132]: RU32(B_k)
+constexpr uint64_t kPartialsOffset = 1024;   // double partial[chunks], then u64 desc[G]
+
+struct WorkspaceView {
+    Control*            ctl;
+    float*              thr;
+    double*             partials;
+    unsigned long long* desc;
+};
+
+__host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+
+// ---- look-back descriptors: status(2) | count(31) | words(31) -----------------------------
+constexpr unsigned long long kDescInvalid = 0ull, kDescAggregate = 1ull, kDescPrefix = 2ull, kDescPoison = 3ull;
+constexpr unsigned long long kDescValueMask = (1ull << 62) - 1ull;
+
+__device__ __forceinline__ unsigned long long desc_pack(unsigned long long st, uint32_t count, uint32_t words) {
+    return (st << 62) | ((unsigned long long)count << 31) | (unsigned long long)words;
+}
+__device__ __forceinline__ uint32_t desc_count(unsigned long long v) { return (uint32_t)((v >> 31) & 0x7FFFFFFFull); }
+__device__ __forceinline__ uint32_t desc_words(unsigned long long v) { return (uint32_t)(v & 0x7FFFFFFFull); }
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t bswap32(uint32_t x) { return __byte_perm(x, 0, 0x0123); }
+
+// bits [pos, pos+nb) of a most-significant-bit-first sequence stored as bytes; `words` is the
+// sequence viewed as little-endian 32-bit words, `nwords` its length.  nb <= 32.
+__device__ __forceinline__ uint32_t get_bits_be(const uint32_t* __restrict__ words, uint32_t nwords,
+                                                uint32_t pos, uint32_t nb) {
+    uint32_t wi = pos >> 5, sh = pos & 31u;
+    uint32_t w0 = wi < nwords ? bswap32(__ldg(words + wi)) : 0u;
+    uint32_t w1 = (wi + 1u) < nwords ? bswap32(__ldg(words + wi + 1u)) : 0u;
+    unsigned long long both = ((unsigned long long)w0 << 32) | w1;
+    if (nb == 0) return 0u;
+    return (uint32_t)((both >> (64u - sh - nb)) & ((nb >= 32u) ? 0xFFFFFFFFull : ((1ull << nb) - 1ull)));
+}
+
+}  // namespace fsg

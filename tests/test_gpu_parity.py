@@ -1,0 +1,260 @@
+"""GPU-vs-oracle parity through the C-ABI: sum bit-equal, stream byte-equal, kept keys and
+codes equal, decoded and accumulated values within 1e-6 relative / 1e-12 absolute (they are
+expected to be bit-equal, which is asserted too).  Sizes span several tiles and ragged tails."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2112_04291_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-6, 1e-12
+
+
+def _params(b, tau=128, l=2):
+    return binding.params(b, tau, l, 14), oracle.params(b, tau, l, 14)
+
+
+def _check_roundtrip(v, b, tau=128, l=2, workers_dense0=None):
+    import gpu_util as G
+    v = np.ascontiguousarray(v, np.float32)
+    n = v.size
+    pg, po = _params(b, tau, l)
+    orc, ostream = oracle.compress(v, po)
+    rc, status, gstream, intact = G.gpu_compress(v, pg, fill=0xEE)
+    assert rc == 0 and intact
+    assert status == orc
+    # header (incl. the fp64 sum) and every byte of the stream
+    assert gstream.size == ostream.size, (gstream.size, ostream.size)
+    assert np.array_equal(gstream[:64], ostream[:64]), "header differs"
+    assert np.array_equal(gstream, ostream), "stream differs"
+    if orc != 0:
+        return ostream
+    # kept keys and integer codes
+    rc1, keys, codes, S = oracle.parse(gstream, n, po)
+    rc2, okeys, ocodes, oS = oracle.value_encode(v, b, tau)
+    assert rc1 == 0 and np.array_equal(keys, okeys) and np.array_equal(codes, ocodes) and S == oS
+    assert np.all((np.abs(codes) >= 1) & (np.abs(codes) <= tau))
+    # decode + accumulate
+    dense0 = workers_dense0 if workers_dense0 is not None else np.zeros(n, np.float32)
+    odense = dense0.copy()
+    assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+    rc, st, gdense, intact = G.gpu_decompress(gstream, n, pg, dense0)
+    assert rc == 0 and st == 0 and intact
+    assert np.allclose(gdense, odense, rtol=RTOL, atol=ATOL)
+    assert np.array_equal(gdense, odense)
+    return ostream
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 15, 16, 17, 127, 128, 129, 1023, 1024, 1025, 4097,
+                               16383, 16384, 16385, 32768 + 5, 49152, 100_003, 1_000_000])
+def test_sizes_and_ragged_tails(n):
+    rng = np.random.default_rng(n)
+    v = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    b = workloads.base_for_keep(v, max(1, n // 20))
+    _check_roundtrip(v, b)
+
+
+@pytest.mark.parametrize("l", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("keep", [0.001, 0.05, 0.5])
+def test_flag_sizes_and_keep_ratios(l, keep):
+    n = 70_000
+    rng = np.random.default_rng(l * 100 + int(keep * 1000))
+    v = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    b = workloads.base_for_keep(v, int(keep * n))
+    _check_roundtrip(v, b, l=l)
+
+
+@pytest.mark.parametrize("tau", [1, 7, 64, 100, 128])
+def test_thresholds(tau):
+    n = 40_000
+    rng = np.random.default_rng(tau)
+    v = rng.standard_normal(n).astype(np.float32)
+    b = workloads.base_for_keep(v, n // 50, tau=tau)
+    _check_roundtrip(v, b, tau=tau)
+
+
+def test_all_kept_dense_tiles():
+    # b^tau huge: every nonzero entry survives; blobs reach their widest form
+    n = 3 * 16384 + 77
+    rng = np.random.default_rng(5)
+    v = rng.standard_normal(n).astype(np.float32)
+    _check_roundtrip(v, 2.0, tau=128, l=2)
+    _check_roundtrip(v, 2.0, tau=128, l=5)
+
+
+def test_degenerate_inputs():
+    n = 40_000
+    z = np.zeros(n, np.float32)
+    _check_roundtrip(z, 1.1)                                   # all zero: d = 0
+    one = z.copy(); one[12345] = -3.0
+    _check_roundtrip(one, 1.1)                                 # single nonzero: L = 0 raised to 1
+    ends = z.copy(); ends[0] = 1.0; ends[n - 1] = -1.0
+    _check_roundtrip(ends, 1.1)                                # keys 0 and n-1
+    neg0 = z.copy(); neg0[::7] = -0.0; neg0[5] = 1e-3
+    _check_roundtrip(neg0, 1.1)
+    rng = np.random.default_rng(8)
+    den = (rng.standard_normal(n) * 1e-41).astype(np.float32)  # denormals, no flush to zero
+    assert np.any(den != 0) and np.all(np.abs(den) < 1.2e-38)
+    _check_roundtrip(den, 1.05)
+    mixed = den.copy(); mixed[::3] *= np.float32(1e20)
+    _check_roundtrip(mixed, 1.3)
+    # none kept: tau = 1 and b barely above 1 put the threshold above every entry
+    flat = np.ones(n, np.float32)
+    s = _check_roundtrip(flat, 1.0001, tau=1)
+    assert int(np.frombuffer(s[24:32].tobytes(), np.uint64)[0]) == 0
+    # values exactly on boundaries: powers of two with b = 2
+    pw = (2.0 ** -rng.integers(0, 30, n)).astype(np.float32)
+    _check_roundtrip(pw, 2.0, tau=40)
+
+
+def test_nonfinite_and_capacity():
+    import gpu_util as G
+    n = 50_000
+    rng = np.random.default_rng(9)
+    v = rng.standard_normal(n).astype(np.float32)
+    for bad in (np.inf, -np.inf, np.nan):
+        w = v.copy(); w[31337] = bad
+        s = _check_roundtrip(w, 1.1)
+        assert s.size == 64
+    pg, po = _params(1.2)
+    orc, full = oracle.compress(v, po)
+    assert orc == 0
+    for cap in (full.size - 4, 64 + 8 * 4 + 16, full.size):
+        orc, ostream = oracle.compress(v, po, cap=cap)
+        rc, status, gstream, intact = G.gpu_compress(v, pg, cap=cap, fill=0x11)
+        assert rc == 0 and intact and status == orc
+        assert np.array_equal(gstream, ostream)
+    rc, status, gstream, intact = G.gpu_compress(v, pg, cap=64)
+    assert rc == binding.E_CAPACITY and intact
+
+
+def test_sum_entry_point_bit_equal():
+    import torch
+    import gpu_util as G
+    for n in (1, 5, 1000, 16384, 16385, 123_457, 3_000_001):
+        rng = np.random.default_rng(n)
+        v = (rng.standard_normal(n) * 10.0 ** rng.integers(-6, 3, n)).astype(np.float32)
+        g = G.to_dev(v)
+        binding.ensure_workspace(n, binding.params(1.1))
+        out = torch.zeros(1, dtype=torch.float64, device=g.device)
+        assert binding.abs_sum(g, out) == 0
+        torch.cuda.synchronize()
+        assert out.item() == oracle.abs_sum(v)
+
+
+def test_workers_accumulate_in_call_order():
+    import gpu_util as G
+    n = 200_000
+    W = 4
+    pg = po = None
+    rng = np.random.default_rng(3)
+    dense_o = rng.standard_normal(n).astype(np.float32)
+    dense_g = dense_o.copy()
+    for w in range(W):
+        v = workloads.student_t_layers(n, seed=w, blocks=9)
+        b = workloads.base_for_keep(v, n // 100)
+        pg, po = _params(b)
+        orc, ostream = oracle.compress(v, po)
+        rc, status, gstream, intact = G.gpu_compress(v, pg)
+        assert np.array_equal(gstream, ostream)
+        assert oracle.decompress_accumulate(ostream, n, po, dense_o) == 0
+        rc, st, dense_g, intact = G.gpu_decompress(gstream, n, pg, dense_g)
+        assert rc == 0 and st == 0 and intact
+    assert np.allclose(dense_g, dense_o, rtol=RTOL, atol=ATOL)
+    assert np.array_equal(dense_g, dense_o)
+
+
+def test_repeatable():
+    import gpu_util as G
+    n = 300_000
+    v = workloads.normal_outliers(n, seed=4)
+    pg, po = _params(workloads.base_for_keep(v, n // 10))
+    first = None
+    for _ in range(10):
+        rc, status, s, intact = G.gpu_compress(v, pg)
+        assert rc == 0 and status == 0 and intact
+        first = s if first is None else first
+        assert np.array_equal(s, first)
+
+
+def _damage(stream, pos, value, width=4):
+    s = stream.copy()
+    s[pos:pos + width] = np.frombuffer(int(value).to_bytes(width, "little"), np.uint8)
+    return s
+
+
+def test_damaged_streams_report_the_oracles_status_and_stay_in_bounds():
+    import gpu_util as G
+    n = 5 * 16384 + 100
+    rng = np.random.default_rng(21)
+    v = rng.standard_normal(n).astype(np.float32)
+    b = 1.1            # threshold ~0.4: most entries survive, every group is non-empty
+    pg, po = _params(b)
+    orc, st0 = oracle.compress(v, po)
+    assert orc == 0
+    G_ = (n + 16383) // 16384
+    cases = [
+        _damage(st0, 0, 0x12345678), _damage(st0, 4, 7), _damage(st0, 8, 2), _damage(st0, 16, n + 1, 8),
+        _damage(st0, 12, 127), _damage(st0, 56, 3, 1), _damage(st0, 60, G_ + 1), _damage(st0, 32, st0.size + 4, 8),
+        _damage(st0, 32, 60, 8),
+    ]
+    a0 = int.from_bytes(st0[64:68].tobytes(), "little")
+    cases.append(_damage(st0, 64, (a0 & 0xFF000000) | 16385))            # count > T
+    cases.append(_damage(st0, 64, (a0 & 0xFFFFFF) | (15 << 24)))          # M > group_log2
+    cases.append(_damage(st0, 64, (a0 & 0xFFFFFF)))                       # M = 0
+    off1 = int.from_bytes(st0[76:80].tobytes(), "little")
+    cases.append(_damage(st0, 76, off1 + 1))
+    cases.append(_damage(st0, 76, off1 - 1))
+    cases.append(_damage(st0, 68, 5))                                     # first offset inside the header
+    cases.append(_damage(st0, 64 + 8 * 3, 0))                             # non-empty group marked empty
+    last = G_ - 1
+    offl = int.from_bytes(st0[64 + 8 * last + 4:64 + 8 * last + 8].tobytes(), "little")
+    cnt = int.from_bytes(st0[64 + 8 * last:64 + 8 * last + 4].tobytes(), "little") & 0xFFFFFF
+    s2 = st0.copy(); s2[4 * offl + cnt:] = 0xFF                           # last group: widest flags, max deltas
+    cases.append(s2)
+    s3 = st0.copy(); s3[4 * off1] = 0x7F | 0x80                           # code byte L = 128 is fine for tau = 128
+    cases.append(s3)
+    for i, s in enumerate(cases):
+        expect = oracle.decompress_accumulate(s, n, po, np.zeros(n, np.float32))
+        rc, st, dense, intact = G.gpu_decompress(s, n, pg)
+        assert rc == 0 and intact, i
+        assert st == expect, (i, st, expect)
+    # BAD_CODE needs tau < 128
+    pg2, po2 = _params(1.3, tau=20)
+    orc, st1 = oracle.compress(v, po2)
+    o1 = int.from_bytes(st1[68:72].tobytes(), "little")
+    s4 = st1.copy(); s4[4 * o1 + 2] = 90
+    expect = oracle.decompress_accumulate(s4, n, po2, np.zeros(n, np.float32))
+    rc, st, dense, intact = G.gpu_decompress(s4, n, pg2)
+    assert expect == oracle.DEC_BAD_CODE and st == expect and intact
+    # truncated buffer
+    expect = oracle.decompress_accumulate(st0, n, po, np.zeros(n, np.float32), nbytes=st0.size - 8)
+    rc, st, dense, intact = G.gpu_decompress(st0, n, pg, nbytes=st0.size - 8)
+    assert st == expect == oracle.DEC_TRUNCATED and intact and not dense.any()
+    # and a clean stream still decodes after all that (the status word was cleared)
+    rc, st, dense, intact = G.gpu_decompress(st0, n, pg)
+    assert rc == 0 and st == 0
+
+
+def test_host_buffer_calls():
+    import torch
+    n = 150_000
+    v = workloads.normal(n, seed=2)
+    b = workloads.base_for_keep(v, n // 100)
+    pg, po = _params(b)
+    binding.ensure_workspace(n, pg)
+    scratch = torch.empty(binding.host_scratch_bytes(n, pg), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(binding.compress_bound(n, pg), dtype=torch.uint8).pin_memory()
+    gh = torch.from_numpy(v).pin_memory()
+    rc, produced, status = binding.compress_host(gh, pg, out, scratch)
+    orc, ostream = oracle.compress(v, po)
+    assert rc == 0 and status == 0 and produced == ostream.size
+    assert np.array_equal(out[:produced].numpy(), ostream)
+    dense = torch.zeros(n, dtype=torch.float32).pin_memory()
+    rc, st = binding.decompress_accumulate_host([out, out], [produced, produced], n, pg, dense, scratch)
+    odense = np.zeros(n, np.float32)
+    oracle.decompress_accumulate(ostream, n, po, odense)
+    oracle.decompress_accumulate(ostream, n, po, odense)
+    assert rc == 0 and st == 0 and np.array_equal(dense.numpy(), odense)
