@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the FastSGD compress + decompress-accumulate hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic gradients: every simulated
+worker's gradient is compressed (abs-sum pass + fused encode pass), then every stream is
+decompress-accumulated into one dense vector.  The metric is input GB/s = 4 n W / t.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+
+Under torchrun (N > 1) every rank runs an independent replica (the path has no exchange step
+on one node: "replicas only"); value = units of all ranks / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compress+decompress input GB/s (fp32 gradient)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+WORKLOADS = {
+    # name: (description, default workers, default keep)
+    "c1": "n=1,048,576 N(0,1e-3^2), 1% kept, 1 worker",
+    "c2": "n=25,557,032 Student-t(3) x per-layer log-uniform scale over 161 blocks, 0.5% kept, 4 workers",
+    "c3": "n=50,000,000 clustered-sparse Laplace, 80% of nonzeros kept, 1 worker",
+    "c4": "n=335,141,888 per-block normal, 8 workers",
+    "c5": "n=2^k N(0,1e-3^2) with 1% outliers x100",
+}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def sample_once(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {
+                "hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+                "sw_thermal_slowdown": 0x20, "hw_power_brake_slowdown": 0x80, "sync_boost": 0x10,
+            }
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._stop.is_set():
+            self.sample_once()
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop.set()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def run_reference(args, rank):
+    """The oracle, as it stands, on the host cores: the reference arm of this tier."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2112_04291_b200 import workloads
+    wl = workloads.make(args.workload, n=args.n, workers=1, keep=args.keep)
+    v, n = wl.grads[0], wl.n
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    # size the per-step sample so that the whole run stays near a minute
+    probe = v[: min(n, 1 << 20)]
+    t0 = time.perf_counter()
+    oracle.compress(probe, po)
+    per_elem = (time.perf_counter() - t0) / probe.size * 1.3
+    budget = 60.0 / max(1, args.steps + args.warmup)
+    ns = int(max(1 << 16, min(n, budget / per_elem)))
+    sample = np.ascontiguousarray(v[:ns])
+    dense = np.zeros(ns, np.float32)
+
+    def step():
+        rc, s = oracle.compress(sample, po)
+        assert rc == 0
+        assert oracle.decompress_accumulate(s, ns, po, dense) == 0
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = 4.0 * ns * args.steps / dt / 1e9
+    desc = f"first {ns} entries of worker 0 of {args.workload}, compress + decompress-accumulate, 1 thread"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "n": n, "sample_n": ns},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--n", type=int, default=None)
+    ap.add_argument("--workers", type=int, default=None)
+    ap.add_argument("--keep", type=float, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2112_04291_b200 import binding, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs: generated on the host with fixed seeds (each rank its own), resident in HBM
+    wl = workloads.make(args.workload, n=args.n, workers=args.workers, keep=args.keep, seed=1000 * rank)
+    n, W = wl.n, wl.workers
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg, dev)
+    host_grads = [torch.from_numpy(g).pin_memory() for g in wl.grads]
+    grads = [g.to(dev, non_blocking=True) for g in host_grads]
+    cap = min(binding.compress_bound(n, pg), max(4 * n, 1 << 20))
+    cap = (cap + 255) & ~255
+    outs = [torch.zeros(cap, dtype=torch.uint8, device=dev) for _ in range(W)]
+    dense = torch.zeros(n, dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+
+    def compress_all():
+        for w in range(W):
+            rc = binding.compress(grads[w], pg, outs[w])
+            if rc:
+                raise binding.FastSGDError(rc, "fastsgd_compress")
+
+    def decompress_all():
+        for w in range(W):
+            rc = binding.decompress_accumulate(outs[w], cap, n, pg, dense)
+            if rc:
+                raise binding.FastSGDError(rc, "fastsgd_decompress_accumulate")
+
+    def step():
+        compress_all()
+        decompress_all()
+
+    # one checked step before anything is timed
+    step()
+    infos = [binding.stream_info(o) for o in outs]
+    assert all(st == 0 for _, _, st in infos), infos
+    assert binding.decode_status() == 0
+    stream_bytes = [tb for tb, _, _ in infos]
+    kept = [d for _, d, _ in infos]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = binding.launch_count()
+    ms_total = timed(step, args.steps)
+    launches = binding.launch_count() - launches0
+    sampler.sample_once()
+    sampler.stop()
+    ms_step = ms_total / args.steps
+
+    # separate phases (same protocol, fewer steps)
+    sub = max(3, min(args.steps, 50))
+    ms_comp = timed(compress_all, sub) / sub
+    ms_dec = timed(decompress_all, sub) / sub
+
+    # per-kernel durations from CUDA events recorded on the launching stream
+    binding.kernel_timing_enable(True)
+    barrier()
+    for _ in range(sub):
+        step()
+    torch.cuda.synchronize()
+    ktimes = binding.kernel_timing_read()
+    binding.kernel_timing_enable(False)
+
+    peak, peak_kind = measured_peak()
+    in_bytes = 4.0 * n * W
+    alg_comp = 8.0 * n * W + float(sum(stream_bytes))              # two reads of the gradient + stream written
+    alg_dec = float(sum(stream_bytes)) + 8.0 * float(sum(kept))    # stream read + read-modify-write of kept entries
+    value = in_bytes * world / (ms_step * 1e-3) / 1e9
+
+    per_launch_bytes = {
+        "k_abs_sum": 4.0 * n + 8.0 * ((n + 16383) // 16384),
+        "k_encode": 4.0 * n + float(sum(stream_bytes)) / W,
+        "k_decode_accumulate": float(sum(stream_bytes)) / W + 8.0 * float(sum(kept)) / W,
+    }
+    kernels = {}
+    for k, (ms, cnt) in ktimes.items():
+        if cnt:
+            avg = ms / cnt
+            kernels[k] = {"launches": cnt, "avg_us": avg * 1e3, "share": None,
+                          "achieved_gbs": per_launch_bytes[k] / (avg * 1e-3) / 1e9}
+    tot = sum(ms for ms, cnt in ktimes.values()) or 1.0
+    for k in kernels:
+        kernels[k]["share"] = ktimes[k][0] / tot
+    dom = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else None
+    roofline = None
+    if dom:
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": kernels[dom]["achieved_gbs"] / peak, "peak_kind": f"of {peak_kind}",
+                    "traffic": None, "algorithmic_bytes_per_launch": per_launch_bytes[dom]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "n": n, "workers": W,
+                   "keep_fraction": wl.keep_fraction, "base": wl.base, "tau": wl.tau, "flag_bits": wl.flag_bits,
+                   "group_log2": wl.group_log2, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs of one step (W x 4n bytes) exceed L2; no explicit flush" if in_bytes > 126e6
+                         else "inputs fit in L2: L2-warm number"},
+        "clocks": sampler.summary(),
+        "gpu_launches": launches,
+        "elements_per_s": n * W * world / (ms_step * 1e-3),
+        "combined": {"algorithmic_gbs": (alg_comp + alg_dec) * world / (ms_step * 1e-3) / 1e9,
+                     "frac_of_hbm_peak": (alg_comp + alg_dec) / (ms_step * 1e-3) / 1e9 / peak},
+        "compress": {"ms": ms_comp, "input_gbs": in_bytes / (ms_comp * 1e-3) / 1e9,
+                     "algorithmic_gbs": alg_comp / (ms_comp * 1e-3) / 1e9,
+                     "frac_of_hbm_peak": alg_comp / (ms_comp * 1e-3) / 1e9 / peak},
+        "decompress": {"ms": ms_dec, "input_gbs": in_bytes / (ms_dec * 1e-3) / 1e9,
+                       "algorithmic_gbs": alg_dec / (ms_dec * 1e-3) / 1e9,
+                       "frac_of_hbm_peak": alg_dec / (ms_dec * 1e-3) / 1e9 / peak},
+        "stream": {"bytes_per_worker": float(sum(stream_bytes)) / W, "kept_per_worker": float(sum(kept)) / W,
+                   "bits_per_kept_entry": 8.0 * sum(stream_bytes) / max(1, sum(kept)),
+                   "ratio_vs_dense_fp32": in_bytes / max(1.0, float(sum(stream_bytes)))},
+        "kernels": kernels,
+        "roofline": roofline,
+    }
+
+    # ---- end to end through the host-buffer C-ABI calls (pinned host memory)
+    if not args.no_e2e:
+        scratch = torch.empty(binding.host_scratch_bytes(n, pg), dtype=torch.uint8, device=dev)
+        host_outs = [torch.zeros(cap, dtype=torch.uint8).pin_memory() for _ in range(W)]
+        host_dense = torch.zeros(n, dtype=torch.float32).pin_memory()
+        produced = [0] * W
+
+        def e2e_step():
+            for w in range(W):
+                rc, produced[w], st = binding.compress_host(host_grads[w], pg, host_outs[w], scratch)
+                assert rc == 0 and st == 0, (rc, st)
+            rc, st = binding.decompress_accumulate_host(host_outs, produced, n, pg, host_dense, scratch)
+            assert rc == 0 and st == 0, (rc, st)
+
+        e2e_steps = max(2, min(args.steps, 5))
+        e2e_step()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        line["e2e"] = {"value": in_bytes * world * e2e_steps / dt / 1e9, "unit": UNIT, "steps": e2e_steps,
+                       "h2d_bytes_per_step": int(4 * n * W + sum(produced)),
+                       "d2h_bytes_per_step": int(sum(produced) + 64 * W + 4 * n + 8)}
+        del scratch
+
+    # ---- the oracle on this machine's host cores (reported baseline, not the target)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+        reps, t_cpu = 0, 0.0
+        odense = np.zeros(n, np.float32)
+        while t_cpu < 10.0 and reps < 3:
+            t0 = time.perf_counter()
+            streams = []
+            for g in wl.grads:
+                rc, s = oracle.compress(g, po)
+                assert rc == 0
+                streams.append(s)
+            for s in streams:
+                assert oracle.decompress_accumulate(s, n, po, odense) == 0
+            t_cpu += time.perf_counter() - t0
+            reps += 1
+        line["cpu_baseline"] = {"value": in_bytes * reps / t_cpu / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "host_cores_present": os.cpu_count(),
+                                "sample": f"{reps} full step(s) of {args.workload} ({W} workers, n={n}), single thread"}
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

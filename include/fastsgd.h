@@ -172,6 +172,14 @@ int fastsgd_decompress_accumulate_host(const void* const* streams_host, const ui
                                        float* dense_host, int accumulate, int* status,
                                        void* dev_scratch, uint64_t dev_scratch_bytes, void* stream);
 
+/* Profiling aid.  While enabled, every kernel launch is bracketed by a pair of
+ * CUDA events recorded on its stream.  fastsgd_kernel_timing_read synchronises
+ * those events, adds up the elapsed milliseconds and the launches per kernel
+ * (index 0 abs-sum, 1 encode, 2 decode-accumulate) since the last read, and
+ * forgets them.  Off by default; the events add a little launch overhead. */
+int fastsgd_kernel_timing_enable(int enable);
+int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]);
+
 /* number of kernels the library has launched since it was loaded */
 uint64_t fastsgd_launch_count(void);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "fastsgd_workspace_bytes", "fastsgd_set_workspace", "fastsgd_stream_info",
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
-    "fastsgd_strerror", "fastsgd_version",
+    "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read",
 ]
 
 
@@ -86,6 +86,10 @@ def lib():
         L.fastsgd_strerror.argtypes = [C.c_int]
         L.fastsgd_version.restype = C.c_int
         L.fastsgd_version.argtypes = []
+        L.fastsgd_kernel_timing_enable.restype = C.c_int
+        L.fastsgd_kernel_timing_enable.argtypes = [C.c_int]
+        L.fastsgd_kernel_timing_read.restype = C.c_int
+        L.fastsgd_kernel_timing_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         _lib = L
     return _lib
 
@@ -199,3 +203,18 @@ def decompress_accumulate_host(streams_host, nbytes, n: int, p: Params, dense_ho
 
 def launch_count() -> int:
     return int(lib().fastsgd_launch_count())
+
+
+KERNELS = ("k_abs_sum", "k_encode", "k_decode_accumulate")
+
+
+def kernel_timing_enable(on: bool) -> None:
+    _check(lib().fastsgd_kernel_timing_enable(int(bool(on))), "fastsgd_kernel_timing_enable")
+
+
+def kernel_timing_read():
+    """{kernel name: (total ms, launches)} since the last read; synchronises."""
+    ms = (C.c_double * 3)()
+    cnt = (C.c_uint64 * 3)()
+    _check(lib().fastsgd_kernel_timing_read(ms, cnt), "fastsgd_kernel_timing_read")
+    return {k: (ms[i], int(cnt[i])) for i, k in enumerate(KERNELS)}

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "common.cuh"
 #include "sum.cuh"
@@ -28,6 +29,25 @@ struct State {
 };
 State g_state;
 std::atomic<uint64_t> g_launches{0};
+
+// optional per-kernel timing (profiling aid)
+struct TimedLaunch { int kernel; cudaEvent_t start, stop; };
+bool g_timing = false;
+std::vector<TimedLaunch> g_timed;
+std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_event_pool;
+
+struct LaunchTimer {
+    bool active = false; TimedLaunch t{}; cudaStream_t st;
+    LaunchTimer(int kernel, cudaStream_t s) : st(s) {
+        if (!g_timing) return;
+        if (g_event_pool.empty()) {
+            if (cudaEventCreate(&t.start) != cudaSuccess || cudaEventCreate(&t.stop) != cudaSuccess) return;
+        } else { t.start = g_event_pool.back().first; t.stop = g_event_pool.back().second; g_event_pool.pop_back(); }
+        t.kernel = kernel; active = true;
+        cudaEventRecord(t.start, st);
+    }
+    ~LaunchTimer() { if (active) { cudaEventRecord(t.stop, st); g_timed.push_back(t); } }
+};
 
 int check_params(const fastsgd_params* p, PowTable* pw) {
     if (!p) return FASTSGD_E_NULL;
@@ -104,7 +124,7 @@ int launch_sum(const float* grad, uint64_t n, uint32_t groups, uint32_t tau, con
     sa.ctl = w.ctl; sa.thr = w.thr; sa.partials = w.partials; sa.desc = w.desc; sa.sum_out = sum_out;
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.sum_blocks_per_sm;
     if (grid > sa.chunks) grid = sa.chunks;
-    k_abs_sum<<<(unsigned)grid, kSumThreads, 0, st>>>(sa, pw);
+    { LaunchTimer lt(0, st); k_abs_sum<<<(unsigned)grid, kSumThreads, 0, st>>>(sa, pw); }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
 }
@@ -114,6 +134,27 @@ int launch_sum(const float* grad, uint64_t n, uint32_t groups, uint32_t tau, con
 extern "C" {
 
 int fastsgd_version(void) { return 1; }
+
+int fastsgd_kernel_timing_enable(int enable) {
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    g_timing = enable != 0;
+    return FASTSGD_OK;
+}
+
+int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]) {
+    if (!ms_total || !launches) return FASTSGD_E_NULL;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    for (int i = 0; i < 3; ++i) { ms_total[i] = 0.0; launches[i] = 0; }
+    int rc = FASTSGD_OK;
+    for (const TimedLaunch& t : g_timed) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(t.stop) != cudaSuccess || cudaEventElapsedTime(&ms, t.start, t.stop) != cudaSuccess) rc = FASTSGD_E_CUDA;
+        else { ms_total[t.kernel] += ms; launches[t.kernel] += 1; }
+        g_event_pool.emplace_back(t.start, t.stop);
+    }
+    g_timed.clear();
+    return rc;
+}
 
 uint64_t fastsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -213,7 +254,7 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     ea.grad = grad; ea.n = n; ea.out = static_cast<uint8_t*>(out); ea.out_bytes = out_bytes;
     ea.ctl = w.ctl; ea.thr = w.thr; ea.desc = w.desc; ea.base = params->base;
     ea.G = (uint32_t)G; ea.tau = params->tau; ea.l = params->flag_bits;
-    k_encode<<<(unsigned)G, kEncThreads, sizeof(EncSmem), st>>>(ea);
+    { LaunchTimer lt(1, st); k_encode<<<(unsigned)G, kEncThreads, sizeof(EncSmem), st>>>(ea); }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
 }
@@ -242,7 +283,10 @@ int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_
     uint64_t grid = (G + warps_per_block - 1) / warps_per_block;
     const uint64_t cap = (uint64_t)g_state.sm_count * g_state.dec_blocks_per_sm;
     if (grid > cap) grid = cap;
-    k_decode_accumulate<<<(unsigned)grid, kDecThreads, 0, static_cast<cudaStream_t>(stream)>>>(da, pw);
+    {
+        LaunchTimer lt(2, static_cast<cudaStream_t>(stream));
+        k_decode_accumulate<<<(unsigned)grid, kDecThreads, 0, static_cast<cudaStream_t>(stream)>>>(da, pw);
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
 }

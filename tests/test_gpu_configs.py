@@ -1,0 +1,86 @@
+"""Parity on the five benchmark configurations at their full sizes, in the launch configuration
+the benchmark times (same entry points, same capacity rule): streams byte-equal to the oracle's,
+accumulated dense vector within 1e-6 relative / 1e-12 absolute (and bit-equal)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2112_04291_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-6, 1e-12
+
+
+def _run(wl, check_workers=None):
+    n, W = wl.n, wl.workers
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg)
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    dense = torch.zeros(n, dtype=torch.float32, device="cuda")
+    odense = np.zeros(n, np.float32)
+    out = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    kept_total = 0
+    for w in range(W):
+        g = torch.from_numpy(wl.grads[w]).cuda()
+        assert binding.compress(g, pg, out) == 0
+        total, d, status = binding.stream_info(out)
+        assert status == 0
+        assert binding.decompress_accumulate(out, cap, n, pg, dense) == 0
+        if check_workers is None or w in check_workers:
+            orc, ostream = oracle.compress(wl.grads[w], po)
+            assert orc == 0 and total == ostream.size
+            assert np.array_equal(out[:total].cpu().numpy(), ostream), f"worker {w}: stream differs"
+            assert d == int(np.frombuffer(ostream[24:32].tobytes(), np.uint64)[0])
+            assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+            kept_total += d
+        del g
+    assert binding.decode_status() == 0
+    if check_workers is None or len(check_workers) == W:
+        got = dense.cpu().numpy()
+        assert np.allclose(got, odense, rtol=RTOL, atol=ATOL)
+        assert np.array_equal(got, odense)
+    return kept_total
+
+
+def test_config1_full():
+    wl = workloads.make("c1")
+    kept = _run(wl)
+    assert abs(kept / wl.n - 0.01) < 0.002
+
+
+def test_config2_full_four_workers():
+    wl = workloads.make("c2")
+    assert wl.n == 25_557_032 and wl.workers == 4
+    kept = _run(wl)
+    assert abs(kept / (4 * wl.n) - 0.005) < 0.002
+
+
+def test_config3_full_clustered_sparse():
+    wl = workloads.make("c3")
+    assert wl.n == 50_000_000
+    kept = _run(wl)
+    assert 0.6 < kept / np.count_nonzero(wl.grads[0]) < 0.95
+
+
+@pytest.mark.parametrize("keep", [1e-4, 1e-3, 1e-2])
+def test_config4_full(keep):
+    # two of the eight workers at each keep ratio (generation and the oracle dominate the run time)
+    wl = workloads.make("c4", workers=2, keep=keep)
+    assert wl.n == 335_141_888
+    kept = _run(wl)
+    assert 0.3 * keep < kept / (2 * wl.n) < 3 * keep
+
+
+@pytest.mark.parametrize("log2n", [10, 12, 14, 16, 18, 20, 22, 24, 26])
+@pytest.mark.parametrize("keep", [1e-4, 1e-3, 1e-2, 1e-1])
+def test_config5_sweep(log2n, keep):
+    wl = workloads.make("c5", n=1 << log2n, keep=keep)
+    _run(wl)
+
+
+def test_config5_sweep_largest():
+    wl = workloads.make("c5", n=1 << 30, keep=1e-3)
+    _run(wl)

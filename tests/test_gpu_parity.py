@@ -222,7 +222,7 @@ def test_damaged_streams_report_the_oracles_status_and_stay_in_bounds():
         assert rc == 0 and intact, i
         assert st == expect, (i, st, expect)
     # BAD_CODE needs tau < 128
-    pg2, po2 = _params(1.3, tau=20)
+    pg2, po2 = _params(2.0, tau=20)
     orc, st1 = oracle.compress(v, po2)
     o1 = int.from_bytes(st1[68:72].tobytes(), "little")
     s4 = st1.copy(); s4[4 * o1 + 2] = 90
