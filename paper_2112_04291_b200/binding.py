@@ -205,7 +205,7 @@ def launch_count() -> int:
     return int(lib().fastsgd_launch_count())
 
 
-KERNELS = ("k_abs_sum", "k_encode", "k_decode_accumulate")
+KERNELS = ("k_abs_sum", "k_compress", "k_decode_accumulate")
 
 
 def kernel_timing_enable(on: bool) -> None:
@@ -218,3 +218,26 @@ def kernel_timing_read():
     cnt = (C.c_uint64 * 3)()
     _check(lib().fastsgd_kernel_timing_read(ms, cnt), "fastsgd_kernel_timing_read")
     return {k: (ms[i], int(cnt[i])) for i, k in enumerate(KERNELS)}
+
+
+def debug_trace():
+    """Block 0's %globaltimer stamps (ns) of the last fastsgd_compress call: start, end of the
+    sum pass, grid barrier passed, boundary table ready, end of the encode pass.  Profiling aid
+    read straight from the registered workspace tensor; synchronises."""
+    ws = _workspace_keepalive
+    if ws is None:
+        return None
+    torch.cuda.synchronize()
+    raw = ws[40:40 + 64].cpu().numpy().view("<u8")
+    return [int(x) for x in raw]
+
+
+def debug_trace_blocks(blocks: int = 148):
+    """Per-block stamps of the last fastsgd_compress call, one row per block: start, end of the sum
+    pass, barrier passed, table ready, end of the encode loop, end; then the nanoseconds thread 0
+    spent waiting for tiles and packing in the encode pass.  Profiling aid; synchronises."""
+    ws = _workspace_keepalive
+    if ws is None:
+        return None
+    torch.cuda.synchronize()
+    return ws[1024:1024 + 64 * blocks].cpu().numpy().view("<u8").reshape(blocks, 8).astype("int64")

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "sum.cuh"
 #include "encode.cuh"
+#include "compress.cuh"
 #include "decode.cuh"
 
 namespace {
@@ -25,6 +26,8 @@ struct State {
     int        sm_count = 0;
     int        sum_blocks_per_sm = 0;
     int        dec_blocks_per_sm = 0;
+    int        cmp_blocks_per_sm = 0;
+    unsigned long long barrier_base = 0;   // value of Control::barrier once all enqueued compress calls are done
     bool       attrs_set = false;
 };
 State g_state;
@@ -80,9 +83,13 @@ uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
     return kHeaderBytes + 8ull * G + 4ull * G * per_group_words;
 }
 
-uint64_t ws_bytes_for(uint64_t n, uint32_t group_log2) {
+uint64_t ws_dense_offset(uint64_t n, uint32_t group_log2) {
     const uint64_t b = kPartialsOffset + 8ull * chunks_of(n) + 8ull * groups_of(n, group_log2);
     return (b + 255ull) & ~255ull;
+}
+
+uint64_t ws_bytes_for(uint64_t n, uint32_t group_log2) {
+    return ws_dense_offset(n, group_log2) + (uint64_t)kMaxCtas * kDenseScratchBytes;
 }
 
 WorkspaceView view(void* ws, uint64_t n) {
@@ -104,7 +111,11 @@ int ensure_device_setup() {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EncSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
-    int b1 = 0, b2 = 0;
+    if (cudaFuncSetAttribute(k_compress, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    int b1 = 0, b2 = 0, b3 = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+    g_state.cmp_blocks_per_sm = b3;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, k_decode_accumulate, kDecThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
     g_state.device = dev;
@@ -211,6 +222,7 @@ int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
         return FASTSGD_E_CUDA;
     g_state.ws = dev_ptr;
     g_state.ws_bytes = bytes;
+    g_state.barrier_base = 0;
     return FASTSGD_OK;
 }
 
@@ -247,16 +259,27 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     WorkspaceView w = view(g_state.ws, n);
 
-    rc = launch_sum(grad, n, (uint32_t)G, params->tau, pw, w, nullptr, st);
-    if (rc) return rc;
-
-    EncArgs ea;
-    ea.grad = grad; ea.n = n; ea.out = static_cast<uint8_t*>(out); ea.out_bytes = out_bytes;
-    ea.ctl = w.ctl; ea.thr = w.thr; ea.desc = w.desc; ea.base = params->base;
-    ea.G = (uint32_t)G; ea.tau = params->tau; ea.l = params->flag_bits;
-    { LaunchTimer lt(1, st); k_encode<<<(unsigned)G, kEncThreads, sizeof(EncSmem), st>>>(ea); }
+    if (g_state.cmp_blocks_per_sm < 1) return FASTSGD_E_CUDA;
+    uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
+    if (grid > kMaxCtas) grid = kMaxCtas;
+    if (grid > G) grid = G;
+    CmpArgs ca;
+    ca.grad = grad; ca.n = n; ca.out = static_cast<uint8_t*>(out); ca.out_bytes = out_bytes;
+    ca.ctl = w.ctl; ca.partials = w.partials; ca.desc = w.desc;
+    ca.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
+    ca.base = params->base; ca.barrier_target = g_state.barrier_base + grid;
+    ca.G = (uint32_t)G; ca.tau = params->tau; ca.l = params->flag_bits;
+    void* kargs[] = {&ca, &pw};
+    cudaError_t err;
+    {
+        LaunchTimer lt(1, st);
+        err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)grid), dim3(kCmpThreads), kargs,
+                                          sizeof(CmpSmem), st);
+    }
+    if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
+    g_state.barrier_base += grid;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+    return FASTSGD_OK;
 }
 
 int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
@@ -283,6 +306,8 @@ int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_
     uint64_t grid = (G + warps_per_block - 1) / warps_per_block;
     const uint64_t cap = (uint64_t)g_state.sm_count * g_state.dec_blocks_per_sm;
     if (grid > cap) grid = cap;
+    const uint64_t min_grid = (G + kDecListMax - 1) / kDecListMax;     // a block owns at most kDecListMax groups
+    if (grid < min_grid) grid = min_grid;
     {
         LaunchTimer lt(2, static_cast<cudaStream_t>(stream));
         k_decode_accumulate<<<(unsigned)grid, kDecThreads, 0, static_cast<cudaStream_t>(stream)>>>(da, pw);

@@ -35,12 +35,15 @@ struct Control {
     unsigned int       skip;           // 0 encode normally, 1 sum == 0, 2 sum not finite
     unsigned long long decode_status;  // min over failures of (group << 32 | key index << 8 | status)
     double             sum;            // S
-    unsigned int       pad[56];
+    unsigned long long barrier;        // blocks that have reached the grid barrier, over all calls so far
+    unsigned long long trace[8];       // %globaltimer of block 0 at its phase boundaries (profiling aid)
+    unsigned int       pad[38];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
 constexpr uint64_t kThrOffset      = 256;    // float thr[132]: RU32(B_k)
-constexpr uint64_t kPartialsOffset = 1024;   // double partial[chunks], then u64 desc[G]
+constexpr uint64_t kTraceOffset    = 1024;   // u64 trace[<=496][8]: per-block %globaltimer stamps (profiling aid)
+constexpr uint64_t kPartialsOffset = 32768;  // double partial[chunks], then u64 desc[G]
 
 struct WorkspaceView {
     Control*            ctl;

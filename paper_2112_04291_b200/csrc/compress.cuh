@@ -1,0 +1,649 @@
+// The encoder as ONE persistent kernel (one thread block per SM, cooperative launch).
+//
+// Phase 1 (Algorithm 1, first step): every block streams its tiles of 2^14 entries through a
+// three-stage ring of shared-memory buffers filled by bulk asynchronous copies (TMA, no
+// multicast) and reduces each tile on the fixed fp64 pairwise tree; one partial per tile.
+// Grid barrier (bounded wait).  Every block then reduces all partials in the same tree order,
+// so that each holds sum and the boundary table B_k = sum / b^k without a second hop.
+// Phase 2 (rest of Algorithm 1, Algorithm 2 per group): the block walks its tiles again in the
+// opposite order, so that the last three tiles of phase 1 are still in shared memory and are
+// not read from HBM a second time; the others arrive through the same ring while the block
+// filters, compacts, quantises, delta-encodes and bit-packs the tile at hand.
+//
+// Device-wide offsets.  A packed blob stays in a shared-memory arena and the tile's
+// (count, words) is published as a descriptor; no block waits for another while it packs.
+// When the arena fills up, and at the end, the block drains it: it brings its running
+// exclusive scan of all descriptors up to its pending tiles (block-wide shuffle scans over
+// 512 descriptors at a time, bounded polls for the ones not published yet), copies the blobs
+// to their places in the stream and writes their directory entries.  The block that owns the
+// lowest unpublished tile never waits for anything, so the scheme cannot deadlock provided all
+// blocks are resident (cooperative launch).  Every wait is bounded; when one runs out the block
+// records FASTSGD_ST_TIMEOUT, poisons its descriptors, waits (bounded) for its own copies in
+// flight and returns.
+#pragma once
+
+#include "common.cuh"
+#include "sum.cuh"
+#include "encode.cuh"
+
+namespace fsg {
+
+constexpr int      kCmpThreads   = 512;
+constexpr int      kCmpWarps     = kCmpThreads / 32;
+constexpr int      kStages       = 1;
+constexpr uint32_t kTile         = 1u << kGroupLog2;          // entries per tile = per group
+constexpr uint32_t kSparseCap    = 2048;                      // kept entries a tile may have on the shared-memory path
+constexpr uint32_t kArenaWords   = 4608;                      // packed blobs waiting for their offsets
+constexpr int      kPendMax      = 32;                        // tiles that may wait in the arena
+constexpr uint32_t kMaxCtas      = 320;                       // scratch slots for the dense path
+constexpr uint32_t kWaitLimit    = 1u << 22;                  // polls before a wait gives up
+constexpr uint32_t kDenseMark    = 0xFFFFFFFFu;               // arena offset of a blob that sits in global scratch
+// dense path scratch per block: values / blob u32[T] | keys u16[T] | codes u8[T]
+constexpr uint64_t kDenseScratchBytes = (uint64_t)kTile * 4u + (uint64_t)kTile * 2u + kTile;
+static_assert(kArenaWords >= (kSparseCap * (8u + 5u + 14u) + 31u) / 32u, "arena holds the widest sparse blob");
+
+constexpr unsigned long long kDescValid = 1ull;               // status of a published descriptor (kDescPoison = 3)
+
+struct CmpSmem {
+    float    stage[kStages][kTile];
+    unsigned long long mbar[kStages];
+    double   s_warp[2][kCmpWarps];
+    double   s_tree[kCmpWarps];
+    unsigned long long scan64[kCmpWarps];
+    float    thr[132];
+    uint32_t warp_tot[2][kCmpWarps];         // by tile parity: an empty tile has no barrier after its read
+    uint32_t scan_tot[kCmpWarps];
+    uint32_t pend_g[kPendMax];
+    uint32_t pend_cm[kPendMax];              // count | M << 24
+    uint32_t pend_words[kPendMax];
+    uint32_t pend_off[kPendMax];             // word offset in the arena, or kDenseMark
+    unsigned long long pend_prefix[kPendMax];// exclusive prefix: count << 32 | words
+    uint32_t max_delta;
+    uint32_t abort_flag;
+    uint32_t poison_seen;
+    uint32_t pad;
+    uint32_t arena[kArenaWords];
+    uint32_t vals[kSparseCap];               // kept values (fp32 bits) of the tile at hand
+    uint16_t keys[kSparseCap];
+    uint8_t  codes[kSparseCap];
+};
+static_assert(sizeof(CmpSmem) <= 232448, "shared memory of one block on sm_100");
+
+struct CmpArgs {
+    const float*        grad;
+    uint64_t            n;
+    uint8_t*            out;
+    uint64_t            out_bytes;
+    Control*            ctl;
+    double*             partials;
+    unsigned long long* desc;
+    unsigned char*      dense_scratch;
+    double              base;
+    unsigned long long  barrier_target;
+    uint32_t            G;
+    uint32_t            tau;
+    uint32_t            l;
+};
+
+// ---- mbarrier / bulk-copy primitives (sm_90+ PTX) -------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait: the hardware suspends the thread for up to about the hinted time per try, so a
+// wait costs a handful of instructions; false when every try ran out.
+constexpr uint32_t kTryHintNs = 10000u;
+constexpr uint32_t kTryLimit  = 1u << 18;
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t t = 0; t < kTryLimit; ++t) {
+        uint32_t ok;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(ok) : "r"(addr), "r"(parity), "r"(kTryHintNs) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_global, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(__cvta_generic_to_global(src_global)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+// descriptors carry their whole payload in one word: relaxed accesses are enough
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long read_globaltimer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Starts the copy of tile `tile` into `stage` (thread 0), and, for the one tile that reaches past
+// n, fills the rest of the buffer (all threads).  Called by the whole block.
+__device__ __forceinline__ void issue_tile(CmpSmem& s, const CmpArgs& a, int stage, uint32_t tile, int tid) {
+    const uint64_t e0 = (uint64_t)tile << kGroupLog2;
+    const uint64_t valid = min((uint64_t)kTile, a.n - e0);           // entries of this tile that exist
+    const uint32_t bulk_bytes = (uint32_t)(valid * 4u) & ~15u;
+    if (tid == 0) {
+        if (bulk_bytes) {
+            mbar_expect_tx(&s.mbar[stage], bulk_bytes);
+            bulk_load(&s.stage[stage][0], a.grad + e0, bulk_bytes, &s.mbar[stage]);
+        } else {
+            mbar_arrive(&s.mbar[stage]);
+        }
+    }
+    if (valid < kTile) {                                             // block-uniform
+        for (uint32_t i = (bulk_bytes >> 2) + tid; i < kTile; i += kCmpThreads)
+            s.stage[stage][i] = i < valid ? __ldg(a.grad + e0 + i) : 0.0f;
+        __syncthreads();
+        // these were generic-proxy writes to a buffer that a later bulk copy (async proxy) overwrites
+        if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+}
+
+// Tree reduction of the per-tile partials, by every block for itself: thread t folds an aligned
+// run of partials with a binary counter, then the tree over the 512 threads.
+__device__ __forceinline__ double reduce_partials(const double* partials, uint32_t chunks, double* s_tree,
+                                                  int tid, int lane, int warp) {
+    uint32_t n2 = 1;
+    while (n2 < chunks) n2 <<= 1;
+    const uint32_t run = n2 > (uint32_t)kCmpThreads ? n2 / kCmpThreads : 1u;
+    double acc = 0.0;
+    double level[20];
+    const uint64_t lo = (uint64_t)tid * run;
+    for (uint32_t i0 = 0; i0 < run; i0 += 8) {
+        double leaf[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint64_t idx = lo + i0 + k;
+            leaf[k] = (i0 + k < run && idx < chunks) ? __ldcg(partials + idx) : 0.0;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t i = i0 + k;
+            if (i < run) {
+                double node = leaf[k];
+#pragma unroll
+                for (int b = 0; b < 20; ++b) {
+                    if ((i >> b) & 1u) node = __dadd_rn(level[b], node);
+                    else { level[b] = node; break; }
+                }
+                acc = node;
+            }
+        }
+    }
+    acc = warp_tree(acc);
+    if (lane == 0) s_tree[warp] = acc;
+    __syncthreads();
+    double t = lane < kCmpWarps ? s_tree[lane] : 0.0;
+    t = warp_tree(t, kCmpWarps);                       // lanes 0..15 of every warp hold the root
+    t = __shfl_sync(kFullMask, t, 0);
+    __syncthreads();
+    return t;
+}
+
+// flag of a delta with bit length bl: least f with ceil((f+1) M / 2^l) >= bl, which is
+// floor((bl-1) 2^l / M) for bl >= 1; the division is a multiplication by ceil(2^16 / M)
+__device__ __forceinline__ uint32_t flag_of(uint32_t delta, uint32_t l, uint32_t inv_m) {
+    const uint32_t bl = delta ? 32u - __clz(delta) : 0u;
+    return bl ? ((((bl - 1u) << l) * inv_m) >> 16) : 0u;
+}
+
+// Phase 2 for one non-empty tile: compaction, quantisation, deltas, M, flags, width scan, packing
+// into `blob`.  DENSE selects where the compacted keys / values / codes live: shared memory
+// (count <= kSparseCap, blob in the arena) or the block's slot of global scratch (blob reuses the
+// values' words).  `m` is the kept mask of this thread's 32 entries, `v` their values.
+template <bool DENSE>
+__device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t count, uint32_t aoff,
+                                          uint32_t warp_base, uint32_t m, const float4 (&v)[8],
+                                          uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
+                                          uint32_t* words_out, uint32_t* M_out, int tid, int lane, int warp) {
+    // (the address space of every pointer is known at compile time in either instantiation:
+    //  shared-memory atomics, not generic ones, do the packing on the sparse path)
+    uint16_t* keys; uint8_t* codes; uint32_t* vals; uint32_t* blob;
+    if (DENSE) {
+        unsigned char* slot = a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
+        vals = reinterpret_cast<uint32_t*>(slot);
+        keys = reinterpret_cast<uint16_t*>(slot + (uint64_t)kTile * 4u);
+        codes = reinterpret_cast<uint8_t*>(slot + (uint64_t)kTile * 6u);
+        blob = vals;
+    } else {
+        vals = s.vals; keys = s.keys; codes = s.codes;
+        blob = s.arena + aoff;
+    }
+
+    // ---- stream compaction in index order: (key, value) of the kept entries
+    if (m != 0u) {
+        uint32_t row_base = warp_base;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const uint32_t tot = r < 4 ? (tot0 >> (8 * r)) & 0xFFu : (tot1 >> (8 * (r - 4))) & 0xFFu;
+            const uint32_t ex  = r < 4 ? (ex0 >> (8 * r)) & 0xFFu : (ex1 >> (8 * (r - 4))) & 0xFFu;
+            const uint32_t mr = (m >> (4 * r)) & 0xFu;
+            uint32_t pos = row_base + ex;
+            const uint32_t k0 = warp * 1024 + r * 128 + lane * 4;
+            if (mr) {
+                if (mr & 1u) { keys[pos] = (uint16_t)(k0);     vals[pos] = __float_as_uint(v[r].x); ++pos; }
+                if (mr & 2u) { keys[pos] = (uint16_t)(k0 + 1); vals[pos] = __float_as_uint(v[r].y); ++pos; }
+                if (mr & 4u) { keys[pos] = (uint16_t)(k0 + 2); vals[pos] = __float_as_uint(v[r].z); ++pos; }
+                if (mr & 8u) { keys[pos] = (uint16_t)(k0 + 3); vals[pos] = __float_as_uint(v[r].w); ++pos; }
+            }
+            row_base += tot;
+        }
+    }
+    if (tid == 0) s.max_delta = 0u;
+    __syncthreads();
+
+    // ---- logarithm quantisation of the kept entries (Eq. 2-3 as a table search) and delta keys (Eq. 4)
+    {
+        uint32_t local_max = 0;
+        for (uint32_t j = tid; j < count; j += kCmpThreads) {
+            const uint32_t key = keys[j];
+            const float val = __uint_as_float(vals[j]);
+            const float av = fabsf(val);
+            uint32_t lo = 0, hi = a.tau;                 // L = least k with |v| >= B_k; holds for k = tau
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (av >= s.thr[mid]) hi = mid; else lo = mid + 1;
+            }
+            const uint32_t L = lo < 1u ? 1u : lo;
+            codes[j] = (uint8_t)((val < 0.0f ? 0x80u : 0u) | (L - 1u));
+            const uint32_t delta = key - (j ? (uint32_t)keys[j - 1] : 0u);
+            local_max = max(local_max, delta);
+        }
+        local_max = __reduce_max_sync(kFullMask, local_max);
+        if (lane == 0 && local_max) atomicMax(&s.max_delta, local_max);
+    }
+    __syncthreads();
+
+    // ---- M, flags and widths; exclusive scan of the widths (a thread owns consecutive keys);
+    //      zero the words the blob can reach (in the dense path they held the values, dead now)
+    const uint32_t maxd = s.max_delta;
+    const uint32_t M = maxd ? (32u - __clz(maxd)) : 1u;
+    const uint32_t inv_m = (65536u + M - 1u) / M;
+    const uint32_t round_up = (1u << a.l) - 1u;
+    const uint32_t ipt = (count + kCmpThreads - 1) / kCmpThreads;
+    const uint32_t j_lo = min(count, tid * ipt), j_hi = min(count, j_lo + ipt);
+    uint32_t my_bits = 0;
+    for (uint32_t j = j_lo; j < j_hi; ++j) {
+        const uint32_t delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
+        my_bits += ((flag_of(delta, a.l, inv_m) + 1u) * M + round_up) >> a.l;
+    }
+    const uint32_t incl = warp_incl_scan(my_bits, lane);
+    if (lane == 31) s.scan_tot[warp] = incl;
+    {
+        const uint32_t bound_words = (count * (8u + a.l + M) + 31u) >> 5;
+        for (uint32_t i = tid; i < bound_words; i += kCmpThreads) blob[i] = 0u;
+    }
+    __syncthreads();
+    uint32_t before = 0, payload_bits = 0;
+#pragma unroll
+    for (int w = 0; w < kCmpWarps; ++w) {
+        const uint32_t t = s.scan_tot[w];
+        if (w < warp) before += t;
+        payload_bits += t;
+    }
+    const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a.l * count;
+    {
+        uint32_t dpos = delta_pos0 + before + (incl - my_bits);
+        for (uint32_t j = j_lo; j < j_hi; ++j) {
+            const uint32_t delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
+            const uint32_t f = flag_of(delta, a.l, inv_m);
+            const uint32_t w = ((f + 1u) * M + round_up) >> a.l;
+            put_bits_smem(blob, 8u * j, codes[j], 8u);
+            put_bits_smem(blob, flag_pos0 + a.l * j, f, a.l);
+            put_bits_smem(blob, dpos, delta, w);
+            dpos += w;
+        }
+    }
+    __syncthreads();      // blob complete; keys / codes / values free for the next tile
+    *words_out = (delta_pos0 + payload_bits + 31u) >> 5;
+    *M_out = M;
+}
+
+// Running exclusive scan of the descriptors, kept by every block for itself.
+struct ScanState {
+    uint32_t pos;          // descriptors [0, pos) are included
+    uint32_t count;        // kept entries in groups [0, pos)
+    uint32_t words;        // blob words of groups [0, pos)
+};
+
+// Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
+// group numbers ascend in steps of gridDim.x.  Returns false if a poisoned descriptor or a
+// timeout was met (the caller aborts).
+__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, ScanState& sc,
+                                      double S, uint32_t skip, int tid, int lane, int warp) {
+    if (npend == 0) return true;
+    const uint32_t g_first = s.pend_g[0], g_last = s.pend_g[npend - 1], grid = gridDim.x;
+    if (tid == 0) s.poison_seen = 0u;
+    __syncthreads();
+    // ---- advance the scan over descriptors [sc.pos, g_last], 512 at a time
+    while (sc.pos <= g_last) {
+        const uint32_t idx = sc.pos + tid;
+        unsigned long long d = 0ull;
+        if (idx <= g_last) {
+            uint32_t spin = 0;
+            d = ld_relaxed_u64(a.desc + idx);
+            while ((d >> 62) == kDescInvalid) {             // not published yet: bounded poll
+                if (++spin > kWaitLimit) { s.poison_seen = 2u; d = 0ull; break; }
+                __nanosleep(64);
+                d = ld_relaxed_u64(a.desc + idx);
+            }
+            if ((d >> 62) == kDescPoison) { s.poison_seen = 1u; d = 0ull; }
+        }
+        const unsigned long long own = ((unsigned long long)desc_count(d) << 32) | desc_words(d);
+        unsigned long long incl = own;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(kFullMask, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s.scan64[warp] = incl;
+        __syncthreads();
+        unsigned long long before = ((unsigned long long)sc.count << 32) | sc.words, all = 0ull;
+#pragma unroll
+        for (int w = 0; w < kCmpWarps; ++w) {
+            const unsigned long long t = s.scan64[w];
+            if (w < warp) before += t;
+            all += t;
+        }
+        // the thread that holds one of this block's pending tiles records that tile's exclusive prefix
+        if (idx >= g_first && idx <= g_last && (idx - g_first) % grid == 0u)
+            s.pend_prefix[(idx - g_first) / grid] = before + incl - own;
+        sc.count += (uint32_t)(all >> 32);
+        sc.words += (uint32_t)all;
+        sc.pos += kCmpThreads;
+        const uint32_t poison_now = s.poison_seen;      // read between the barriers: same value in every thread
+        __syncthreads();
+        if (poison_now) return false;
+    }
+    // the scan ran past g_last by whole steps of 512: pull it back to g_last + 1
+    // (descriptors beyond g_last were read as zero, so only the position needs correcting)
+    sc.pos = g_last + 1u;
+
+    // ---- copy-out, directory entries, header
+    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
+    uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
+    for (int p = 0; p < npend; ++p) {
+        const uint32_t g = s.pend_g[p], cm = s.pend_cm[p], words = s.pend_words[p], aoff = s.pend_off[p];
+        const unsigned long long pre = s.pend_prefix[p];
+        const uint32_t off = fixed_words + (uint32_t)pre;
+        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
+        const uint32_t* blob = aoff == kDenseMark
+            ? reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes)
+            : s.arena + aoff;
+        if (end_bytes <= a.out_bytes)
+            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
+        if (tid == 0) {
+            outw[(kHeaderBytes >> 2) + 2 * g]     = cm;
+            outw[(kHeaderBytes >> 2) + 2 * g + 1] = off;
+        }
+        if (g == a.G - 1 && tid == 0) {
+            int status = kStOk;
+            if (skip == 2u) status = kStNonfinite;
+            else if (end_bytes > a.out_bytes) status = kStCapacity;
+            const uint64_t d_total = status == kStOk ? (pre >> 32) + (cm & 0xFFFFFFu) : 0ull;
+            const uint64_t total = status == kStOk ? end_bytes : (uint64_t)kHeaderBytes;
+            const double Sh = status == kStNonfinite ? 0.0 : S;
+            outw[0] = kMagic;
+            outw[1] = kVersion;
+            outw[2] = (uint32_t)status;
+            outw[3] = a.tau;
+            outw[4] = (uint32_t)a.n;            outw[5] = (uint32_t)(a.n >> 32);
+            outw[6] = (uint32_t)d_total;        outw[7] = (uint32_t)(d_total >> 32);
+            outw[8] = (uint32_t)total;          outw[9] = (uint32_t)(total >> 32);
+            const unsigned long long sb = (unsigned long long)__double_as_longlong(Sh);
+            const unsigned long long bb = (unsigned long long)__double_as_longlong(a.base);
+            outw[10] = (uint32_t)sb;            outw[11] = (uint32_t)(sb >> 32);
+            outw[12] = (uint32_t)bb;            outw[13] = (uint32_t)(bb >> 32);
+            outw[14] = a.l | ((uint32_t)kGroupLog2 << 8);
+            outw[15] = a.G;
+        }
+    }
+    __syncthreads();       // the arena and the pending list are free again
+    return true;
+}
+
+__global__ void __launch_bounds__(kCmpThreads, 2)
+k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
+    extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
+    CmpSmem& s = *reinterpret_cast<CmpSmem*>(cmp_smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t c = blockIdx.x, grid = gridDim.x;
+    const uint32_t k = c < a.G ? (a.G - c + grid - 1) / grid : 0u;      // tiles of this block: c + i * grid
+    const bool tracer = (c == 0 && tid == 0);
+    if (tracer) a.ctl->trace[0] = read_globaltimer();
+    unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(a.ctl) + kTraceOffset) + 8u * c;
+    unsigned long long t_wait = 0ull, t_pack = 0ull;
+    if (tid == 0) btrace[0] = read_globaltimer();
+
+    if (tid == 0) {
+        for (int st = 0; st < kStages; ++st) mbar_init(&s.mbar[st], 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s.abort_flag = 0u;
+    }
+    __syncthreads();
+    uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects
+    uint32_t pending = 0;                     // bit st: a copy into stage st has been started and not waited for
+
+    // =============================== phase 1: partial sums ===============================
+    // load sequence q = 0..k-1 visits the tiles from the block's last to its first
+    for (uint32_t q = 0; q < min(k, (uint32_t)kStages); ++q) {
+        issue_tile(s, a, (int)(q % kStages), c + (k - 1 - q) * grid, tid);
+        pending |= 1u << (q % kStages);
+    }
+    for (uint32_t q = 0; q < k; ++q) {
+        const int st = (int)(q % kStages);
+        const uint32_t tile = c + (k - 1 - q) * grid;
+        if (tid == 0) a.desc[tile] = 0ull;    // descriptors of phase 2 (ordered by the grid barrier)
+        if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
+        parity ^= 1u << st;
+        pending &= ~(1u << st);
+        double x[8];
+        const float4* row = reinterpret_cast<const float4*>(&s.stage[st][warp * 1024]) + lane;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
+        const double u = warp_slab_tree(x, lane);
+        if (lane == 0) s.s_warp[q & 1][warp] = u;
+        __syncthreads();
+        if (s.abort_flag) break;
+        if (warp == 0) {
+            double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
+            t = warp_tree(t, kCmpWarps);
+            if (lane == 0) a.partials[tile] = t;
+        }
+        // the last kStages tiles stay in shared memory for phase 2
+        if (q + kStages < k) {
+            issue_tile(s, a, st, c + (k - 1 - (q + kStages)) * grid, tid);
+            pending |= 1u << st;
+        }
+    }
+    if (tracer) a.ctl->trace[1] = read_globaltimer();
+    if (tid == 0) btrace[1] = read_globaltimer();
+
+    // =============================== grid barrier ===============================
+    __threadfence();
+    __syncthreads();
+    if (tid == 0 && !s.abort_flag) {
+        atomicAdd(&a.ctl->barrier, 1ull);
+        uint32_t spin = 0;
+        while (ld_acquire_u64(&a.ctl->barrier) < a.barrier_target) {
+            if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
+            __nanosleep(64);
+        }
+    }
+    __syncthreads();
+    bool aborted = s.abort_flag != 0u;
+
+    if (!aborted) {
+        if (tracer) a.ctl->trace[2] = read_globaltimer();
+        if (tid == 0) btrace[2] = read_globaltimer();
+
+        // =============================== sum, boundary table ===============================
+        const double S = reduce_partials(a.partials, a.G, s.s_tree, tid, lane, warp);
+        const bool finite = isfinite(S);
+        const uint32_t skip = !finite ? 2u : (S == 0.0 ? 1u : 0u);
+        if (tid <= (int)a.tau) {
+            // |v| >= B_k on an fp32 |v| equals |v| >= RU32(B_k); never below the smallest denormal,
+            // because an entry must also be non-zero to be kept
+            const double Bk = __ddiv_rn(S, pw.P[tid]);
+            s.thr[tid] = finite ? fmaxf(__double2float_ru(Bk), __int_as_float(1)) : __int_as_float(0x7f800000);
+        }
+        if (c == 0 && tid == 0) a.ctl->sum = S;
+        __syncthreads();
+        const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
+        if (tracer) a.ctl->trace[3] = read_globaltimer();
+        if (tid == 0) btrace[3] = read_globaltimer();
+
+        // =============================== phase 2: encode ===============================
+        // tile i of this block sits in stage (k-1-(i%3))%3; tiles 0..min(k,3)-1 are already there
+        ScanState sc; sc.pos = 0u; sc.count = 0u; sc.words = 0u;
+        int npend = 0;
+        uint32_t arena_used = 0;
+        for (uint32_t i = 0; i < k && !aborted; ++i) {
+            const uint32_t g = c + i * grid;
+            const int st = (int)((k - 1 - (i % kStages)) % kStages);
+            if (i >= (uint32_t)kStages) {
+                const unsigned long long tw0 = tid == 0 ? read_globaltimer() : 0ull;
+                if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
+                if (tid == 0) t_wait += read_globaltimer() - tw0;
+                parity ^= 1u << st;
+                pending &= ~(1u << st);
+            }
+            // ---- threshold filter: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c
+            float4 v[8];
+            uint32_t m = 0;
+            {
+                const float4* row = reinterpret_cast<const float4*>(&s.stage[st][warp * 1024]) + lane;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) v[r] = row[r * 32];
+                if (!skip) {
+                    // a row (128 consecutive entries, one float4 per lane) is looked at entry by entry
+                    // only if some lane holds an entry that reaches the threshold
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const float mx = fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w)));
+                        const bool has = mx >= thr_e;
+                        if (__any_sync(kFullMask, has)) {
+                            if (has) {
+                                m |= (fabsf(v[r].x) >= thr_e ? 1u : 0u) << (4 * r);
+                                m |= (fabsf(v[r].y) >= thr_e ? 1u : 0u) << (4 * r + 1);
+                                m |= (fabsf(v[r].z) >= thr_e ? 1u : 0u) << (4 * r + 2);
+                                m |= (fabsf(v[r].w) >= thr_e ? 1u : 0u) << (4 * r + 3);
+                            }
+                        }
+                    }
+                }
+            }
+            // per-row counts scanned over the lanes, four rows per word, one byte per row
+            uint32_t ex0 = 0, ex1 = 0, tot0 = 0, tot1 = 0, warp_total = 0;
+            if (__any_sync(kFullMask, m != 0u)) {
+                uint32_t c0 = 0, c1 = 0;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    c0 |= (uint32_t)__popc((m >> (4 * r)) & 0xFu) << (8 * r);
+                    c1 |= (uint32_t)__popc((m >> (4 * (r + 4))) & 0xFu) << (8 * r);
+                }
+                const uint32_t i0 = warp_incl_scan(c0, lane), i1 = warp_incl_scan(c1, lane);
+                ex0 = i0 - c0; ex1 = i1 - c1;
+                tot0 = __shfl_sync(kFullMask, i0, 31); tot1 = __shfl_sync(kFullMask, i1, 31);
+#pragma unroll
+                for (int r = 0; r < 4; ++r) warp_total += ((tot0 >> (8 * r)) & 0xFFu) + ((tot1 >> (8 * r)) & 0xFFu);
+            }
+            if (lane == 0) s.warp_tot[i & 1u][warp] = warp_total;
+            __syncthreads();                       // every thread has read its part of the stage
+            if (s.abort_flag) { aborted = true; break; }
+            if (i + kStages < k) {                 // refill this stage with the tile three steps ahead
+                issue_tile(s, a, st, c + (i + kStages) * grid, tid);
+                pending |= 1u << st;
+            }
+            uint32_t warp_base = 0, count = 0;
+#pragma unroll
+            for (int w = 0; w < kCmpWarps; ++w) {
+                const uint32_t t = s.warp_tot[i & 1u][w];
+                if (w < warp) warp_base += t;
+                count += t;
+            }
+
+            uint32_t words = 0, M = 0, aoff = 0;
+            const unsigned long long tp0 = tid == 0 ? read_globaltimer() : 0ull;
+            if (count == 0u) {
+                if (npend == kPendMax) { if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
+            } else if (count <= kSparseCap) {
+                const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
+                if (npend == kPendMax || arena_used + worst > kArenaWords) {
+                    if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                    npend = 0; arena_used = 0;
+                }
+                aoff = arena_used;
+                pack_tile<false>(s, a, count, aoff, warp_base, m, v, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+                arena_used += words;
+            } else {
+                // dense tile: packed in global scratch and committed at once
+                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                npend = 0; arena_used = 0;
+                aoff = kDenseMark;
+                pack_tile<true>(s, a, count, 0u, warp_base, m, v, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+            }
+            if (tid == 0) {
+                t_pack += read_globaltimer() - tp0;
+                st_relaxed_u64(a.desc + g, desc_pack(kDescValid, count, words));
+                s.pend_g[npend] = g;
+                s.pend_cm[npend] = count ? (count | (M << 24)) : 0u;
+                s.pend_words[npend] = words;
+                s.pend_off[npend] = aoff;
+            }
+            ++npend;
+            if (aoff == kDenseMark) {
+                __syncthreads();
+                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                npend = 0; arena_used = 0;
+            }
+        }
+        if (tid == 0) btrace[4] = read_globaltimer();
+        if (!aborted) {
+            __syncthreads();                       // pending list written by thread 0
+            if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) aborted = true;
+        }
+        if (tracer) a.ctl->trace[4] = read_globaltimer();
+        if (tid == 0) { btrace[5] = read_globaltimer(); btrace[6] = t_wait; btrace[7] = t_pack; }
+    }
+
+    if (aborted) {
+        // give up: record it, unblock the others, drain this block's copies, return.  The header
+        // is written here by the owner of the last group so that the caller sees the status.
+        __syncthreads();
+        if (tid == 0) {
+            atomicExch(&a.ctl->error, (unsigned)kStTimeout);
+            for (uint32_t i = 0; i < k; ++i) st_relaxed_u64(a.desc + c + i * grid, desc_pack(kDescPoison, 0, 0));
+            for (int st = 0; st < kStages; ++st)
+                if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
+            if (k > 0 && c + (k - 1) * grid == a.G - 1) {
+                uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
+                outw[0] = kMagic; outw[1] = kVersion; outw[2] = (uint32_t)kStTimeout; outw[3] = a.tau;
+                outw[4] = (uint32_t)a.n; outw[5] = (uint32_t)(a.n >> 32);
+                outw[6] = 0u; outw[7] = 0u; outw[8] = kHeaderBytes; outw[9] = 0u;
+                outw[10] = 0u; outw[11] = 0u;
+                const unsigned long long bb = (unsigned long long)__double_as_longlong(a.base);
+                outw[12] = (uint32_t)bb; outw[13] = (uint32_t)(bb >> 32);
+                outw[14] = a.l | ((uint32_t)kGroupLog2 << 8);
+                outw[15] = a.G;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace fsg

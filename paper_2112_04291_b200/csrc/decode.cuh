@@ -1,4 +1,4 @@
-// Decoder (decoder phases 1-4) and aggregation, one warp per group.
+// Decoder (decoder phases 1-4) and aggregation.
 //
 // Phase 1: the length flags give every delta's width; an exclusive scan of the widths gives
 // its bit offset.  Phase 2: an inclusive scan of the deltas, started at g*T, gives the keys
@@ -6,6 +6,11 @@
 // aggregation adds the value into dense_out[key].  Keys are unique within a stream and calls
 // are ordered by the CUDA stream, so the read-modify-write needs no atomics and the result
 // does not depend on the launch shape.
+//
+// Work split: a group with few keys is decoded by one warp, a group with many keys by the
+// whole block; either way a thread owns a run of consecutive keys, so that the scans are one
+// shuffle scan (plus one shared-memory step for the block) per group instead of one per 32 keys,
+// and a group is validated in full before any of it is applied.
 #pragma once
 
 #include "common.cuh"
@@ -13,7 +18,10 @@
 
 namespace fsg {
 
-constexpr int kDecThreads = 256;
+constexpr int      kDecThreads   = 256;
+constexpr int      kDecWarps     = kDecThreads / 32;
+constexpr uint32_t kDecWarpMax   = 128;     // groups with more keys go to the whole block
+constexpr int      kDecListMax   = 512;     // groups one block may own
 
 struct DecArgs {
     const uint8_t*      stream;
@@ -50,12 +58,165 @@ __device__ __forceinline__ int check_header(const DecArgs& a, const uint32_t* w,
     return kStOk;
 }
 
+struct DecShared {
+    float              val[132];
+    uint32_t           scan[kDecWarps];
+    uint32_t           big[kDecListMax];
+    unsigned long long first_bad;     // min over threads of (key index << 8 | status), block path
+    uint32_t           big_count;
+    int                status;
+    unsigned long long total;
+    double             sum;
+};
+
+// exclusive scan of one value per thread over the warp (BLOCK = false) or the block; also returns the total
+template <bool BLOCK>
+__device__ __forceinline__ uint32_t excl_scan(uint32_t v, uint32_t* total, DecShared& s, int lane, int warp) {
+    const uint32_t incl = warp_incl_scan(v, lane);
+    if (!BLOCK) {
+        *total = __shfl_sync(kFullMask, incl, 31);
+        return incl - v;
+    }
+    __syncthreads();                       // s.scan may still be read from the previous scan
+    if (lane == 31) s.scan[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+        const uint32_t t = s.scan[w];
+        if (w < warp) before += t;
+        all += t;
+    }
+    *total = all;
+    return before + incl - v;
+}
+
+// One group, decoded by a warp (BLOCK = false, `t` = lane, `nthreads` = 32) or by the block.
+template <bool BLOCK>
+__device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* __restrict__ sw,
+                                             uint32_t g, uint32_t total_words, uint32_t fixed_words,
+                                             int t, int nthreads, int lane, int warp) {
+    const uint32_t* dir = sw + (kHeaderBytes >> 2);
+    const uint32_t e0 = __ldg(dir + 2 * g), off = __ldg(dir + 2 * g + 1);
+    const uint32_t next_off = (g + 1 < a.G) ? __ldg(dir + 2 * g + 3) : total_words;
+    const uint32_t count = e0 & 0xFFFFFFu, M = e0 >> 24;
+    const uint64_t lo64 = (uint64_t)g << a.group_log2;
+    const uint32_t lo = (uint32_t)lo64;
+    const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+    const uint32_t hi = (uint32_t)(hi64 < a.n ? hi64 : a.n);
+    const bool lead = (t == 0);
+    if ((g == 0 && off != fixed_words) || next_off < off || next_off > total_words || off < fixed_words) {
+        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
+        return;
+    }
+    if (count == 0) {
+        if ((e0 != 0u || next_off != off) && lead) dec_fail(a, g, 0u, kStBadDirectory);
+        return;
+    }
+    const uint32_t nwords = next_off - off;
+    const uint64_t avail_bits = 32ull * nwords;
+    const uint32_t flag_pos0 = 8u * count;
+    const uint64_t delta_pos0_64 = (uint64_t)flag_pos0 + (uint64_t)a.l * count;
+    if (count > hi - lo || M < 1u || M > a.group_log2 || delta_pos0_64 > avail_bits) {
+        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
+        return;
+    }
+    const uint32_t delta_pos0 = (uint32_t)delta_pos0_64;
+    const uint32_t* blob = sw + off;
+    const uint32_t levels_m1 = (1u << a.l) - 1u;
+
+    // this thread's run of consecutive keys [jb, je)
+    const uint32_t K = (count + nthreads - 1) / nthreads;
+    const uint32_t jb = min(count, (uint32_t)t * K), je = min(count, jb + K);
+
+    // phase 1: widths from the flags; their sum fixes the blob's length, which must be the directory's
+    uint32_t wsum = 0;
+    for (uint32_t j = jb; j < je; ++j) {
+        const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+        wsum += ((f + 1u) * M + levels_m1) >> a.l;
+    }
+    uint32_t wtotal;
+    const uint32_t pos0 = delta_pos0 + excl_scan<BLOCK>(wsum, &wtotal, s, lane, warp);
+    if ((((uint64_t)delta_pos0 + wtotal + 31ull) >> 5) != nwords) {
+        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
+        return;
+    }
+
+    // phase 2: sum of this thread's deltas, then the key before its first one
+    uint32_t dsum = 0;
+    {
+        uint32_t pos = pos0;
+        for (uint32_t j = jb; j < je; ++j) {
+            const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
+            dsum = min(dsum + get_bits_be(blob, nwords, pos, w), 1u << 21);   // saturates only when already invalid
+            pos += w;
+        }
+    }
+    uint32_t dtotal;
+    const uint32_t key0 = lo + excl_scan<BLOCK>(dsum, &dtotal, s, lane, warp);
+
+    // validation of the whole group before anything is applied: first key index that repeats,
+    // leaves the group, or carries a code beyond tau
+    unsigned long long bad = ~0ull;
+    {
+        uint32_t pos = pos0, key = key0;
+        for (uint32_t j = jb; j < je; ++j) {
+            const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
+            const uint32_t delta = get_bits_be(blob, nwords, pos, w);
+            pos += w;
+            key += delta;
+            const uint32_t code = (__ldg(blob + (j >> 2)) >> (8u * (j & 3u))) & 0xFFu;
+            if ((j > 0 && delta == 0u) || key >= hi) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey; break; }
+            if ((code & 0x7Fu) + 1u > a.tau) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode; break; }
+        }
+    }
+    if (BLOCK) {
+        __syncthreads();
+        if (t == 0) s.first_bad = ~0ull;
+        __syncthreads();
+        if (bad != ~0ull) atomicMin(&s.first_bad, bad);
+        __syncthreads();
+        bad = s.first_bad;
+    } else {
+        const uint32_t blo = __reduce_min_sync(kFullMask, (uint32_t)(bad < 0xFFFFFFFFull ? bad : 0xFFFFFFFFull));
+        bad = blo == 0xFFFFFFFFu ? ~0ull : (unsigned long long)blo;
+    }
+    if (bad != ~0ull) {
+        if (lead) dec_fail(a, g, (uint32_t)(bad >> 8), (int)(bad & 0xFFull));
+        return;
+    }
+
+    // phases 3-4 and the aggregation, four keys at a time (distinct keys: no aliasing)
+    {
+        uint32_t pos = pos0, key = key0;
+        for (uint32_t j = jb; j < je; j += 4) {
+            uint32_t kk[4]; float vv[4], dd[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                kk[i] = 0xFFFFFFFFu; vv[i] = 0.f;
+                if (j + i < je) {
+                    const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * (j + i), a.l);
+                    const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
+                    key += get_bits_be(blob, nwords, pos, w);
+                    pos += w;
+                    const uint32_t code = (__ldg(blob + ((j + i) >> 2)) >> (8u * ((j + i) & 3u))) & 0xFFu;
+                    const float mag = s.val[(code & 0x7Fu) + 1u];
+                    kk[i] = key; vv[i] = (code & 0x80u) ? -mag : mag;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dd[i] = kk[i] != 0xFFFFFFFFu ? a.dense[kk[i]] : 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) if (kk[i] != 0xFFFFFFFFu) a.dense[kk[i]] = __fadd_rn(dd[i], vv[i]);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kDecThreads)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
-    __shared__ float s_val[132];
-    __shared__ int s_status;
-    __shared__ unsigned long long s_total;
-    __shared__ double s_sum;
+    __shared__ DecShared s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t* sw = reinterpret_cast<const uint32_t*>(a.stream);
 
@@ -65,91 +226,33 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         for (int i = 0; i < 16; ++i) h[i] = __ldg(sw + i);
         uint64_t total = 0; double S = 0.0;
         const int st = check_header(a, h, &total, &S);
-        s_status = st; s_total = total; s_sum = S;
+        s.status = st; s.total = total; s.sum = S; s.big_count = 0u;
         if (st != kStOk && blockIdx.x == 0) dec_fail(a, 0u, 0u, st);
     }
     __syncthreads();
-    if (s_status != kStOk) return;
+    if (s.status != kStOk) return;
     // phases 3-4 as a table: value[L] = (float)(sum / b^L)
-    if (tid <= (int)a.tau) s_val[tid] = __double2float_rn(__ddiv_rn(s_sum, pw.P[tid]));
+    if (tid <= (int)a.tau) s.val[tid] = __double2float_rn(__ddiv_rn(s.sum, pw.P[tid]));
     __syncthreads();
 
-    const uint32_t total_words = (uint32_t)(s_total >> 2);
+    const uint32_t total_words = (uint32_t)(s.total >> 2);
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
-    const uint32_t T = 1u << a.group_log2;
-    const uint32_t levels_m1 = (1u << a.l) - 1u;
     const uint32_t* dir = sw + (kHeaderBytes >> 2);
 
-    const uint32_t warps_total = gridDim.x * (kDecThreads / 32);
-    for (uint32_t g = blockIdx.x * (kDecThreads / 32) + warp; g < a.G; g += warps_total) {
-        const uint32_t e0 = __ldg(dir + 2 * g), off = __ldg(dir + 2 * g + 1);
-        const uint32_t next_off = (g + 1 < a.G) ? __ldg(dir + 2 * g + 3) : total_words;
-        const uint32_t count = e0 & 0xFFFFFFu, M = e0 >> 24;
-        const uint64_t lo64 = (uint64_t)g << a.group_log2;
-        const uint32_t lo = (uint32_t)lo64;
-        const uint32_t hi = (uint32_t)min((uint64_t)a.n, lo64 + T);
-        if ((g == 0 && off != fixed_words) || next_off < off || next_off > total_words || off < fixed_words) {
-            if (lane == 0) dec_fail(a, g, 0u, kStBadDirectory);
+    // this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
+    uint32_t i = warp;
+    for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += kDecWarps * gridDim.x, i += kDecWarps) {
+        const uint32_t count = __ldg(dir + 2 * g) & 0xFFFFFFu;
+        if (count > kDecWarpMax) {
+            if (lane == 0) { const uint32_t slot = atomicAdd(&s.big_count, 1u); if (slot < kDecListMax) s.big[slot] = g; }
             continue;
         }
-        if (count == 0) {
-            if ((e0 != 0u || next_off != off) && lane == 0) dec_fail(a, g, 0u, kStBadDirectory);
-            continue;
-        }
-        const uint32_t nwords = next_off - off;
-        const uint64_t avail_bits = 32ull * nwords;
-        const uint32_t flag_pos0 = 8u * count;
-        const uint64_t delta_pos0_64 = (uint64_t)flag_pos0 + (uint64_t)a.l * count;
-        if (count > hi - lo || M < 1u || M > a.group_log2 || delta_pos0_64 > avail_bits) {
-            if (lane == 0) dec_fail(a, g, 0u, kStBadDirectory);
-            continue;
-        }
-        const uint32_t delta_pos0 = (uint32_t)delta_pos0_64;
-        const uint32_t* blob = sw + off;
-
-        // phase 1a: the flags fix the blob's length; it must be the directory's
-        uint32_t wsum = 0;
-        for (uint32_t j = lane; j < count; j += 32) {
-            const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
-            wsum += ((f + 1u) * M + levels_m1) >> a.l;
-        }
-        wsum = __reduce_add_sync(kFullMask, wsum);
-        if ((((uint64_t)delta_pos0 + wsum + 31ull) >> 5) != nwords) {
-            if (lane == 0) dec_fail(a, g, 0u, kStBadDirectory);
-            continue;
-        }
-
-        uint32_t carry_pos = delta_pos0, carry_key = lo;
-        for (uint32_t j0 = 0; j0 < count; j0 += 32) {
-            const uint32_t j = j0 + lane;
-            const bool act = j < count;
-            uint32_t w = 0, code = 0;
-            if (act) {
-                const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
-                w = ((f + 1u) * M + levels_m1) >> a.l;
-                code = (__ldg(blob + (j >> 2)) >> (8u * (j & 3u))) & 0xFFu;
-            }
-            const uint32_t w_incl = warp_incl_scan(w, lane);
-            const uint32_t delta = act ? get_bits_be(blob, nwords, carry_pos + (w_incl - w), w) : 0u;
-            const uint32_t d_incl = warp_incl_scan(delta, lane);
-            const uint32_t key = carry_key + d_incl;
-            const uint32_t L = (code & 0x7Fu) + 1u;
-            const bool bad_key = act && ((j > 0 && delta == 0u) || key >= hi);
-            const bool bad_code = act && L > a.tau;
-            const uint32_t bad = __ballot_sync(kFullMask, bad_key || bad_code);
-            if (bad) {
-                const int first = __ffs(bad) - 1;
-                if (lane == first) dec_fail(a, g, j, bad_key ? kStBadKey : kStBadCode);
-                break;
-            }
-            if (act) {
-                const float vhat = (code & 0x80u) ? -s_val[L] : s_val[L];
-                a.dense[key] = __fadd_rn(a.dense[key], vhat);
-            }
-            carry_pos += __shfl_sync(kFullMask, w_incl, 31);
-            carry_key += __shfl_sync(kFullMask, d_incl, 31);
-        }
+        decode_group<false>(a, s, sw, g, total_words, fixed_words, lane, 32, lane, warp);
     }
+    __syncthreads();
+    const uint32_t nbig = min(s.big_count, (uint32_t)kDecListMax);
+    for (uint32_t b = 0; b < nbig; ++b)
+        decode_group<true>(a, s, sw, s.big[b], total_words, fixed_words, tid, kDecThreads, lane, warp);
 }
 
 }  // namespace fsg

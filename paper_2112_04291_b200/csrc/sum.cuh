@@ -134,16 +134,26 @@ k_abs_sum(const SumArgs a, const __grid_constant__ PowTable pw) {
         // 2^b partials; a new leaf merges upwards while the matching bit of its index is set
         double level[20];
         const uint64_t lo = (uint64_t)tid * run;
-        volatile const double* parts = a.partials;
-        for (uint32_t i = 0; i < run; ++i) {
-            const uint64_t idx = lo + i;
-            double node = idx < a.chunks ? parts[idx] : 0.0;
+        for (uint32_t i0 = 0; i0 < run; i0 += 8) {
+            double leaf[8];          // eight independent L2 loads in flight
 #pragma unroll
-            for (int b = 0; b < 20; ++b) {
-                if ((i >> b) & 1u) node = __dadd_rn(level[b], node);
-                else { level[b] = node; break; }
+            for (int k = 0; k < 8; ++k) {
+                const uint64_t idx = lo + i0 + k;
+                leaf[k] = (i0 + k < run && idx < a.chunks) ? __ldcg(a.partials + idx) : 0.0;
             }
-            acc = node;   // after the last leaf (i = run-1, all low bits set) this is the run's node
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t i = i0 + k;
+                if (i < run) {
+                    double node = leaf[k];
+#pragma unroll
+                    for (int b = 0; b < 20; ++b) {
+                        if ((i >> b) & 1u) node = __dadd_rn(level[b], node);
+                        else { level[b] = node; break; }
+                    }
+                    acc = node;   // after the last leaf (i = run-1, all low bits set) this is the run's node
+                }
+            }
         }
     }
     acc = warp_tree(acc);
