@@ -8,7 +8,8 @@
 // Phase 2 (rest of Algorithm 1, Algorithm 2 per group): the block walks its tiles again in the
 // opposite order, so that the last three tiles of phase 1 are still in shared memory and are
 // not read from HBM a second time; the others arrive through the same ring while the block
-// filters, compacts, quantises, delta-encodes and bit-packs the tile at hand.
+// filters, compacts, quantises, delta-encodes and bit-packs the tile at hand, every warp on its
+// own slab of 1024 entries, with two block barriers per non-empty tile.
 //
 // Device-wide offsets.  A packed blob stays in a shared-memory arena and the tile's
 // (count, words) is published as a descriptor; no block waits for another while it packs.
@@ -32,7 +33,7 @@ constexpr int      kCmpThreads   = 512;
 constexpr int      kCmpWarps     = kCmpThreads / 32;
 constexpr int      kStages       = 1;
 constexpr uint32_t kTile         = 1u << kGroupLog2;          // entries per tile = per group
-constexpr uint32_t kSparseCap    = 2048;                      // kept entries a tile may have on the shared-memory path
+constexpr uint32_t kSlabCap      = 192;                       // kept entries a warp's 1024-entry slab may have on the shared-memory path
 constexpr uint32_t kArenaWords   = 4608;                      // packed blobs waiting for their offsets
 constexpr int      kPendMax      = 32;                        // tiles that may wait in the arena
 constexpr uint32_t kMaxCtas      = 320;                       // scratch slots for the dense path
@@ -40,7 +41,7 @@ constexpr uint32_t kWaitLimit    = 1u << 22;                  // polls before a 
 constexpr uint32_t kDenseMark    = 0xFFFFFFFFu;               // arena offset of a blob that sits in global scratch
 // dense path scratch per block: values / blob u32[T] | keys u16[T] | codes u8[T]
 constexpr uint64_t kDenseScratchBytes = (uint64_t)kTile * 4u + (uint64_t)kTile * 2u + kTile;
-static_assert(kArenaWords >= (kSparseCap * (8u + 5u + 14u) + 31u) / 32u, "arena holds the widest sparse blob");
+static_assert(kArenaWords >= (kCmpWarps * kSlabCap * (8u + 5u + 14u) + 31u) / 32u, "arena holds the widest sparse blob");
 
 constexpr unsigned long long kDescValid = 1ull;               // status of a published descriptor (kDescPoison = 3)
 
@@ -51,7 +52,12 @@ struct CmpSmem {
     double   s_tree[kCmpWarps];
     unsigned long long scan64[kCmpWarps];
     float    thr[132];
-    uint32_t warp_tot[2][kCmpWarps];         // by tile parity: an empty tile has no barrier after its read
+    // per-slab summaries, by tile parity (an empty tile has no second barrier)
+    uint32_t sum_count[2][kCmpWarps];        // kept entries of the slab; bit 31: more than kSlabCap
+    uint32_t sum_first[2][kCmpWarps];        // first and last kept key (tile-local) of the slab
+    uint32_t sum_last[2][kCmpWarps];
+    uint32_t sum_maxd[2][kCmpWarps];         // largest delta between two kept keys of the slab
+    uint32_t sum_bits[2][kCmpWarps];         // payload bits of the slab
     uint32_t scan_tot[kCmpWarps];
     uint32_t pend_g[kPendMax];
     uint32_t pend_cm[kPendMax];              // count | M << 24
@@ -63,9 +69,8 @@ struct CmpSmem {
     uint32_t poison_seen;
     uint32_t pad;
     uint32_t arena[kArenaWords];
-    uint32_t vals[kSparseCap];               // kept values (fp32 bits) of the tile at hand
-    uint16_t keys[kSparseCap];
-    uint8_t  codes[kSparseCap];
+    uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
+    uint16_t wkeys[kCmpWarps][kSlabCap];     // per warp: kept keys (tile-local), in index order
 };
 static_assert(sizeof(CmpSmem) <= 232448, "shared memory of one block on sm_100");
 
@@ -153,45 +158,39 @@ __device__ __forceinline__ void issue_tile(CmpSmem& s, const CmpArgs& a, int sta
     }
 }
 
-// Tree reduction of the per-tile partials, by every block for itself: thread t folds an aligned
-// run of partials with a binary counter, then the tree over the 512 threads.
-__device__ __forceinline__ double reduce_partials(const double* partials, uint32_t chunks, double* s_tree,
-                                                  int tid, int lane, int warp) {
-    uint32_t n2 = 1;
-    while (n2 < chunks) n2 <<= 1;
-    const uint32_t run = n2 > (uint32_t)kCmpThreads ? n2 / kCmpThreads : 1u;
-    double acc = 0.0;
-    double level[20];
-    const uint64_t lo = (uint64_t)tid * run;
-    for (uint32_t i0 = 0; i0 < run; i0 += 8) {
-        double leaf[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint64_t idx = lo + i0 + k;
-            leaf[k] = (i0 + k < run && idx < chunks) ? __ldcg(partials + idx) : 0.0;
-        }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t i = i0 + k;
-            if (i < run) {
-                double node = leaf[k];
-#pragma unroll
-                for (int b = 0; b < 20; ++b) {
-                    if ((i >> b) & 1u) node = __dadd_rn(level[b], node);
-                    else { level[b] = node; break; }
-                }
-                acc = node;
-            }
-        }
-    }
-    acc = warp_tree(acc);
-    if (lane == 0) s_tree[warp] = acc;
+// Tree reduction of the per-tile partials, by every block for itself, in passes of 512
+// consecutive partials: thread t takes partial 512*p + t, the block forms that aligned node by
+// shuffles (positions = lanes, then warps); the nodes of the passes are then reduced the same
+// way.  Everything stays in registers and shared memory.
+__device__ __forceinline__ double block_tree(double x, double* s_tree, int lane, int warp) {
+    x = warp_tree(x);
+    __syncthreads();                                   // s_tree may still be read from the last use
+    if (lane == 0) s_tree[warp] = x;
     __syncthreads();
     double t = lane < kCmpWarps ? s_tree[lane] : 0.0;
     t = warp_tree(t, kCmpWarps);                       // lanes 0..15 of every warp hold the root
-    t = __shfl_sync(kFullMask, t, 0);
+    return __shfl_sync(kFullMask, t, 0);
+}
+
+__device__ __forceinline__ double reduce_partials(const double* partials, uint32_t chunks, double* s_tree,
+                                                  double* s_nodes, int tid, int lane, int warp) {
+    const uint32_t passes = (chunks + kCmpThreads - 1) / kCmpThreads;       // <= 256 for n < 2^31
+    if (passes == 1) {
+        const double x = (uint32_t)tid < chunks ? __ldcg(partials + tid) : 0.0;
+        return block_tree(x, s_tree, lane, warp);
+    }
+    double next = (uint32_t)tid < chunks ? __ldcg(partials + tid) : 0.0;
+    for (uint32_t p = 0; p < passes; ++p) {
+        const double x = next;
+        const uint64_t idx = (uint64_t)(p + 1) * kCmpThreads + tid;
+        next = (p + 1 < passes && idx < chunks) ? __ldcg(partials + idx) : 0.0;    // in flight during this pass
+        const double node = block_tree(x, s_tree, lane, warp);
+        if (tid == 0) s_nodes[p] = node;
+    }
     __syncthreads();
-    return t;
+    // the nodes of the passes, zero-padded to 512 positions, reduced on the same tree
+    const double y = (uint32_t)tid < passes ? s_nodes[tid] : 0.0;
+    return block_tree(y, s_tree, lane, warp);
 }
 
 // flag of a delta with bit length bl: least f with ceil((f+1) M / 2^l) >= bl, which is
@@ -201,28 +200,32 @@ __device__ __forceinline__ uint32_t flag_of(uint32_t delta, uint32_t l, uint32_t
     return bl ? ((((bl - 1u) << l) * inv_m) >> 16) : 0u;
 }
 
-// Phase 2 for one non-empty tile: compaction, quantisation, deltas, M, flags, width scan, packing
-// into `blob`.  DENSE selects where the compacted keys / values / codes live: shared memory
-// (count <= kSparseCap, blob in the arena) or the block's slot of global scratch (blob reuses the
-// values' words).  `m` is the kept mask of this thread's 32 entries, `v` their values.
-template <bool DENSE>
-__device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t count, uint32_t aoff,
-                                          uint32_t warp_base, uint32_t m, const float4 (&v)[8],
-                                          uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
-                                          uint32_t* words_out, uint32_t* M_out, int tid, int lane, int warp) {
-    // (the address space of every pointer is known at compile time in either instantiation:
-    //  shared-memory atomics, not generic ones, do the packing on the sparse path)
-    uint16_t* keys; uint8_t* codes; uint32_t* vals; uint32_t* blob;
-    if (DENSE) {
-        unsigned char* slot = a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
-        vals = reinterpret_cast<uint32_t*>(slot);
-        keys = reinterpret_cast<uint16_t*>(slot + (uint64_t)kTile * 4u);
-        codes = reinterpret_cast<uint8_t*>(slot + (uint64_t)kTile * 6u);
-        blob = vals;
-    } else {
-        vals = s.vals; keys = s.keys; codes = s.codes;
-        blob = s.arena + aoff;
+// L = least k in [0, tau] with |v| >= B_k (Eq. 2-3 as a table search; holds for k = tau), raised
+// to 1, and the sign: the code byte
+__device__ __forceinline__ uint32_t code_byte_of(const float* thr, uint32_t tau, float val) {
+    const float av = fabsf(val);
+    uint32_t lo = 0, hi = tau;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (av >= thr[mid]) hi = mid; else lo = mid + 1;
     }
+    const uint32_t L = lo < 1u ? 1u : lo;
+    return (val < 0.0f ? 0x80u : 0u) | (L - 1u);
+}
+
+// Phase 2 for a tile too dense for the per-warp lists: block-wide compaction, quantisation,
+// deltas, M, flags, width scan and packing in the block's slot of global scratch (the blob reuses
+// the values' words).  `m` is the kept mask of this thread's 32 entries, `tile` the tile's entries
+// (shared memory).
+__device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, uint32_t count,
+                                             uint32_t warp_base, uint32_t m, const float* tile,
+                                             uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
+                                             uint32_t* words_out, uint32_t* M_out, int tid, int lane, int warp) {
+    unsigned char* slot = a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
+    uint32_t* vals = reinterpret_cast<uint32_t*>(slot);
+    uint16_t* keys = reinterpret_cast<uint16_t*>(slot + (uint64_t)kTile * 4u);
+    uint8_t* codes = reinterpret_cast<uint8_t*>(slot + (uint64_t)kTile * 6u);
+    uint32_t* blob = vals;
 
     // ---- stream compaction in index order: (key, value) of the kept entries
     if (m != 0u) {
@@ -235,10 +238,10 @@ __device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t
             uint32_t pos = row_base + ex;
             const uint32_t k0 = warp * 1024 + r * 128 + lane * 4;
             if (mr) {
-                if (mr & 1u) { keys[pos] = (uint16_t)(k0);     vals[pos] = __float_as_uint(v[r].x); ++pos; }
-                if (mr & 2u) { keys[pos] = (uint16_t)(k0 + 1); vals[pos] = __float_as_uint(v[r].y); ++pos; }
-                if (mr & 4u) { keys[pos] = (uint16_t)(k0 + 2); vals[pos] = __float_as_uint(v[r].z); ++pos; }
-                if (mr & 8u) { keys[pos] = (uint16_t)(k0 + 3); vals[pos] = __float_as_uint(v[r].w); ++pos; }
+                if (mr & 1u) { keys[pos] = (uint16_t)(k0);     vals[pos] = __float_as_uint(tile[k0]);     ++pos; }
+                if (mr & 2u) { keys[pos] = (uint16_t)(k0 + 1); vals[pos] = __float_as_uint(tile[k0 + 1]); ++pos; }
+                if (mr & 4u) { keys[pos] = (uint16_t)(k0 + 2); vals[pos] = __float_as_uint(tile[k0 + 2]); ++pos; }
+                if (mr & 8u) { keys[pos] = (uint16_t)(k0 + 3); vals[pos] = __float_as_uint(tile[k0 + 3]); ++pos; }
             }
             row_base += tot;
         }
@@ -246,20 +249,12 @@ __device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t
     if (tid == 0) s.max_delta = 0u;
     __syncthreads();
 
-    // ---- logarithm quantisation of the kept entries (Eq. 2-3 as a table search) and delta keys (Eq. 4)
+    // ---- logarithm quantisation of the kept entries and delta keys (Eq. 4)
     {
         uint32_t local_max = 0;
         for (uint32_t j = tid; j < count; j += kCmpThreads) {
             const uint32_t key = keys[j];
-            const float val = __uint_as_float(vals[j]);
-            const float av = fabsf(val);
-            uint32_t lo = 0, hi = a.tau;                 // L = least k with |v| >= B_k; holds for k = tau
-            while (lo < hi) {
-                const uint32_t mid = (lo + hi) >> 1;
-                if (av >= s.thr[mid]) hi = mid; else lo = mid + 1;
-            }
-            const uint32_t L = lo < 1u ? 1u : lo;
-            codes[j] = (uint8_t)((val < 0.0f ? 0x80u : 0u) | (L - 1u));
+            codes[j] = (uint8_t)code_byte_of(s.thr, a.tau, __uint_as_float(vals[j]));
             const uint32_t delta = key - (j ? (uint32_t)keys[j - 1] : 0u);
             local_max = max(local_max, delta);
         }
@@ -269,7 +264,7 @@ __device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t
     __syncthreads();
 
     // ---- M, flags and widths; exclusive scan of the widths (a thread owns consecutive keys);
-    //      zero the words the blob can reach (in the dense path they held the values, dead now)
+    //      zero the words the blob can reach (they held the values, dead now)
     const uint32_t maxd = s.max_delta;
     const uint32_t M = maxd ? (32u - __clz(maxd)) : 1u;
     const uint32_t inv_m = (65536u + M - 1u) / M;
@@ -308,7 +303,7 @@ __device__ __forceinline__ void pack_tile(CmpSmem& s, const CmpArgs& a, uint32_t
             dpos += w;
         }
     }
-    __syncthreads();      // blob complete; keys / codes / values free for the next tile
+    __syncthreads();      // blob complete
     *words_out = (delta_pos0 + payload_bits + 31u) >> 5;
     *M_out = M;
 }
@@ -492,7 +487,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[2] = read_globaltimer();
 
         // =============================== sum, boundary table ===============================
-        const double S = reduce_partials(a.partials, a.G, s.s_tree, tid, lane, warp);
+        const double S = reduce_partials(a.partials, a.G, s.s_tree, reinterpret_cast<double*>(s.arena), tid, lane, warp);
         const bool finite = isfinite(S);
         const uint32_t skip = !finite ? 2u : (S == 0.0 ? 1u : 0u);
         if (tid <= (int)a.tau) {
@@ -508,13 +503,19 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[3] = read_globaltimer();
 
         // =============================== phase 2: encode ===============================
-        // tile i of this block sits in stage (k-1-(i%3))%3; tiles 0..min(k,3)-1 are already there
+        // Tile i of this block sits in stage (k-1-(i%kStages))%kStages; the last ones of phase 1 are
+        // already there.  Every warp owns one slab of 1024 consecutive entries of the tile: it
+        // filters it, compacts its kept entries into its own list, quantises them and forms their
+        // deltas without talking to the other warps; two block barriers per non-empty tile exchange
+        // the slab summaries (counts, boundary keys, largest delta -> M) and the payload bits.
         ScanState sc; sc.pos = 0u; sc.count = 0u; sc.words = 0u;
         int npend = 0;
         uint32_t arena_used = 0;
+        const uint32_t round_up = (1u << a.l) - 1u;
         for (uint32_t i = 0; i < k && !aborted; ++i) {
             const uint32_t g = c + i * grid;
             const int st = (int)((k - 1 - (i % kStages)) % kStages);
+            const uint32_t par = i & 1u;
             if (i >= (uint32_t)kStages) {
                 const unsigned long long tw0 = tid == 0 ? read_globaltimer() : 0ull;
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
@@ -522,33 +523,41 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
             }
-            // ---- threshold filter: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c
-            float4 v[8];
+            const unsigned long long tp0 = tid == 0 ? read_globaltimer() : 0ull;
+            // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c.
+            // A row (128 consecutive entries, one float4 per lane) is looked at entry by entry only
+            // if some lane holds an entry that reaches the threshold.
+            const float* tile = s.stage[st];
             uint32_t m = 0;
-            {
-                const float4* row = reinterpret_cast<const float4*>(&s.stage[st][warp * 1024]) + lane;
+            if (!skip) {
+                const float4* row = reinterpret_cast<const float4*>(tile + warp * 1024) + lane;
+                float rowmx[8];
 #pragma unroll
-                for (int r = 0; r < 8; ++r) v[r] = row[r * 32];
-                if (!skip) {
-                    // a row (128 consecutive entries, one float4 per lane) is looked at entry by entry
-                    // only if some lane holds an entry that reaches the threshold
+                for (int r = 0; r < 8; ++r) {
+                    const float4 q = row[r * 32];
+                    rowmx[r] = fmaxf(fmaxf(fabsf(q.x), fabsf(q.y)), fmaxf(fabsf(q.z), fabsf(q.w)));
+                }
+                const float mx = fmaxf(fmaxf(fmaxf(rowmx[0], rowmx[1]), fmaxf(rowmx[2], rowmx[3])),
+                                       fmaxf(fmaxf(rowmx[4], rowmx[5]), fmaxf(rowmx[6], rowmx[7])));
+                if (__any_sync(kFullMask, mx >= thr_e)) {
 #pragma unroll
                     for (int r = 0; r < 8; ++r) {
-                        const float mx = fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w)));
-                        const bool has = mx >= thr_e;
+                        const bool has = rowmx[r] >= thr_e;
                         if (__any_sync(kFullMask, has)) {
                             if (has) {
-                                m |= (fabsf(v[r].x) >= thr_e ? 1u : 0u) << (4 * r);
-                                m |= (fabsf(v[r].y) >= thr_e ? 1u : 0u) << (4 * r + 1);
-                                m |= (fabsf(v[r].z) >= thr_e ? 1u : 0u) << (4 * r + 2);
-                                m |= (fabsf(v[r].w) >= thr_e ? 1u : 0u) << (4 * r + 3);
+                                const float4 q = row[r * 32];
+                                m |= (fabsf(q.x) >= thr_e ? 1u : 0u) << (4 * r);
+                                m |= (fabsf(q.y) >= thr_e ? 1u : 0u) << (4 * r + 1);
+                                m |= (fabsf(q.z) >= thr_e ? 1u : 0u) << (4 * r + 2);
+                                m |= (fabsf(q.w) >= thr_e ? 1u : 0u) << (4 * r + 3);
                             }
                         }
                     }
                 }
             }
-            // per-row counts scanned over the lanes, four rows per word, one byte per row
-            uint32_t ex0 = 0, ex1 = 0, tot0 = 0, tot1 = 0, warp_total = 0;
+            // ---- warp-local compaction in index order: per-row counts scanned over the lanes, four
+            // rows per word, one byte per row; then quantisation and deltas on the warp's own list
+            uint32_t ex0 = 0, ex1 = 0, tot0 = 0, tot1 = 0, slab_count = 0, slab_first = 0, slab_last = 0, slab_maxd = 0;
             if (__any_sync(kFullMask, m != 0u)) {
                 uint32_t c0 = 0, c1 = 0;
 #pragma unroll
@@ -560,42 +569,139 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 ex0 = i0 - c0; ex1 = i1 - c1;
                 tot0 = __shfl_sync(kFullMask, i0, 31); tot1 = __shfl_sync(kFullMask, i1, 31);
 #pragma unroll
-                for (int r = 0; r < 4; ++r) warp_total += ((tot0 >> (8 * r)) & 0xFFu) + ((tot1 >> (8 * r)) & 0xFFu);
-            }
-            if (lane == 0) s.warp_tot[i & 1u][warp] = warp_total;
-            __syncthreads();                       // every thread has read its part of the stage
-            if (s.abort_flag) { aborted = true; break; }
-            if (i + kStages < k) {                 // refill this stage with the tile three steps ahead
-                issue_tile(s, a, st, c + (i + kStages) * grid, tid);
-                pending |= 1u << st;
-            }
-            uint32_t warp_base = 0, count = 0;
+                for (int r = 0; r < 4; ++r) slab_count += ((tot0 >> (8 * r)) & 0xFFu) + ((tot1 >> (8 * r)) & 0xFFu);
+                if (slab_count <= kSlabCap) {
+                    uint16_t* wk = s.wkeys[warp];
+                    uint32_t* wv = s.wvals[warp];
+                    if (m != 0u) {
+                        uint32_t row_base = 0;
 #pragma unroll
-            for (int w = 0; w < kCmpWarps; ++w) {
-                const uint32_t t = s.warp_tot[i & 1u][w];
-                if (w < warp) warp_base += t;
-                count += t;
+                        for (int r = 0; r < 8; ++r) {
+                            const uint32_t tot = r < 4 ? (tot0 >> (8 * r)) & 0xFFu : (tot1 >> (8 * (r - 4))) & 0xFFu;
+                            const uint32_t ex  = r < 4 ? (ex0 >> (8 * r)) & 0xFFu : (ex1 >> (8 * (r - 4))) & 0xFFu;
+                            const uint32_t mr = (m >> (4 * r)) & 0xFu;
+                            uint32_t pos = row_base + ex;
+                            const uint32_t k0 = warp * 1024 + r * 128 + lane * 4;
+                            if (mr) {
+                                if (mr & 1u) { wk[pos] = (uint16_t)(k0);     wv[pos] = __float_as_uint(tile[k0]);     ++pos; }
+                                if (mr & 2u) { wk[pos] = (uint16_t)(k0 + 1); wv[pos] = __float_as_uint(tile[k0 + 1]); ++pos; }
+                                if (mr & 4u) { wk[pos] = (uint16_t)(k0 + 2); wv[pos] = __float_as_uint(tile[k0 + 2]); ++pos; }
+                                if (mr & 8u) { wk[pos] = (uint16_t)(k0 + 3); wv[pos] = __float_as_uint(tile[k0 + 3]); ++pos; }
+                            }
+                            row_base += tot;
+                        }
+                    }
+                    __syncwarp();
+                    for (uint32_t j = lane; j < slab_count; j += 32) {
+                        const uint32_t key = wk[j];
+                        wv[j] = code_byte_of(s.thr, a.tau, __uint_as_float(wv[j]));      // value -> code byte, in place
+                        if (j) slab_maxd = max(slab_maxd, key - (uint32_t)wk[j - 1]);
+                    }
+                    slab_maxd = __reduce_max_sync(kFullMask, slab_maxd);
+                    slab_first = wk[0];
+                    slab_last = wk[slab_count - 1];
+                }
+            }
+            if (lane == 0) {
+                s.sum_count[par][warp] = slab_count | (slab_count > kSlabCap ? 0x80000000u : 0u);
+                s.sum_first[par][warp] = slab_first;
+                s.sum_last[par][warp] = slab_last;
+                s.sum_maxd[par][warp] = slab_maxd;
+            }
+            __syncthreads();                       // summaries written; every thread has read its part of the stage
+            if (s.abort_flag) { aborted = true; break; }
+            // ---- every warp combines the 16 summaries (lane w <-> slab w)
+            const uint32_t sc_raw = lane < kCmpWarps ? s.sum_count[par][lane] : 0u;
+            const uint32_t cnt_l = sc_raw & 0x7FFFFFFFu;
+            const uint32_t count = __reduce_add_sync(kFullMask, cnt_l);
+            const bool overflow = __any_sync(kFullMask, (sc_raw >> 31) != 0u);
+            const uint32_t cnt_incl = warp_incl_scan(cnt_l, lane);
+            const uint32_t warp_base = __shfl_sync(kFullMask, cnt_incl - cnt_l, warp);      // kept entries in the slabs before mine
+            const bool refill = i + kStages < k;
+            if (refill && !overflow) {             // every thread has read its part of the stage (a dense tile
+                issue_tile(s, a, st, c + (i + kStages) * grid, tid);      // still needs its values: refilled below)
+                pending |= 1u << st;
             }
 
             uint32_t words = 0, M = 0, aoff = 0;
-            const unsigned long long tp0 = tid == 0 ? read_globaltimer() : 0ull;
             if (count == 0u) {
                 if (npend == kPendMax) { if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
-            } else if (count <= kSparseCap) {
+            } else if (!overflow) {
                 const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
                 if (npend == kPendMax || arena_used + worst > kArenaWords) {
                     if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                     npend = 0; arena_used = 0;
                 }
                 aoff = arena_used;
-                pack_tile<false>(s, a, count, aoff, warp_base, m, v, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+                uint32_t* blob = s.arena + aoff;
+                // boundary deltas: a slab's first key minus the last kept key before it (0 at the tile's start),
+                // found by a running maximum since the keys ascend with the slab number
+                const uint32_t last_l = (lane < kCmpWarps && cnt_l) ? s.sum_last[par][lane] : 0u;
+                uint32_t run = last_l;
+#pragma unroll
+                for (int o = 1; o < kCmpWarps; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(kFullMask, run, o);
+                    if (lane >= o) run = max(run, t);
+                }
+                const uint32_t prev_last = __shfl_up_sync(kFullMask, run, 1);
+                const uint32_t bd_l = (lane < kCmpWarps && cnt_l) ? s.sum_first[par][lane] - (lane ? prev_last : 0u) : 0u;
+                const uint32_t maxd_l = lane < kCmpWarps ? max(s.sum_maxd[par][lane], bd_l) : 0u;
+                const uint32_t maxd = __reduce_max_sync(kFullMask, maxd_l);
+                M = maxd ? (32u - __clz(maxd)) : 1u;
+                const uint32_t inv_m = (65536u + M - 1u) / M;
+                const uint32_t my_bd = __shfl_sync(kFullMask, bd_l, warp);
+                const uint32_t my_cnt = __shfl_sync(kFullMask, cnt_l, warp);
+                const uint16_t* wk = s.wkeys[warp];
+                const uint32_t* wv = s.wvals[warp];
+                // payload bits of my slab
+                uint32_t bits = 0;
+                for (uint32_t j = lane; j < my_cnt; j += 32) {
+                    const uint32_t delta = j ? (uint32_t)wk[j] - (uint32_t)wk[j - 1] : my_bd;
+                    bits += ((flag_of(delta, a.l, inv_m) + 1u) * M + round_up) >> a.l;
+                }
+                bits = __reduce_add_sync(kFullMask, bits);
+                if (lane == 0) s.sum_bits[par][warp] = bits;
+                {
+                    const uint32_t bound_words = (count * (8u + a.l + M) + 31u) >> 5;
+                    for (uint32_t w = tid; w < bound_words; w += kCmpThreads) blob[w] = 0u;
+                }
+                __syncthreads();                   // payload bits of every slab known; blob zeroed
+                const uint32_t bits_l = lane < kCmpWarps ? s.sum_bits[par][lane] : 0u;
+                const uint32_t bits_incl = warp_incl_scan(bits_l, lane);
+                const uint32_t bits_before = __shfl_sync(kFullMask, bits_incl - bits_l, warp);
+                const uint32_t payload_bits = __shfl_sync(kFullMask, bits_incl, 31);
+                const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a.l * count;
+                words = (delta_pos0 + payload_bits + 31u) >> 5;
+                // pack my slab's entries: codes | flags | deltas (most significant bit first)
+                uint32_t dbase = delta_pos0 + bits_before;
+                for (uint32_t j0 = 0; j0 < my_cnt; j0 += 32) {
+                    const uint32_t j = j0 + lane;
+                    uint32_t delta = 0, f = 0, w = 0;
+                    if (j < my_cnt) {
+                        delta = j ? (uint32_t)wk[j] - (uint32_t)wk[j - 1] : my_bd;
+                        f = flag_of(delta, a.l, inv_m);
+                        w = ((f + 1u) * M + round_up) >> a.l;
+                    }
+                    const uint32_t w_incl = warp_incl_scan(w, lane);
+                    if (j < my_cnt) {
+                        const uint32_t q = warp_base + j;                 // rank of the entry in the group
+                        put_bits_smem(blob, 8u * q, wv[j] & 0xFFu, 8u);
+                        put_bits_smem(blob, flag_pos0 + a.l * q, f, a.l);
+                        put_bits_smem(blob, dbase + (w_incl - w), delta, w);
+                    }
+                    dbase += __shfl_sync(kFullMask, w_incl, 31);
+                }
                 arena_used += words;
             } else {
-                // dense tile: packed in global scratch and committed at once
+                // a slab is too dense for its list: block-wide path in global scratch, committed at once
                 if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 aoff = kDenseMark;
-                pack_tile<true>(s, a, count, 0u, warp_base, m, v, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+                pack_tile_dense(s, a, count, warp_base, m, tile, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+                if (refill) {
+                    issue_tile(s, a, st, c + (i + kStages) * grid, tid);
+                    pending |= 1u << st;
+                }
             }
             if (tid == 0) {
                 t_pack += read_globaltimer() - tp0;
