@@ -2,7 +2,7 @@
 """Benchmark of the FastSGD compress + decompress-accumulate hot path on B200.
 
 One step = one pass of the whole path over one batch of synthetic gradients: every simulated
-worker's gradient is compressed (abs-sum pass + fused encode pass), then every stream is
+worker's gradient is compressed (one fused kernel: abs-sum pass, grid barrier, encode pass), then every stream is
 decompress-accumulated into one dense vector.  The metric is input GB/s = 4 n W / t.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
@@ -156,12 +156,12 @@ def main():
     ap.add_argument("--keep", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph of the step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2112_04291_b200 import multirank
+    rank, world, local_rank = multirank.env_rank()
 
     if args.impl == "reference":
         run_reference(args, rank)
@@ -176,11 +176,10 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+        multirank.init("nccl", dev)
 
     # ---- inputs: generated on the host with fixed seeds (each rank its own), resident in HBM
-    wl = workloads.make(args.workload, n=args.n, workers=args.workers, keep=args.keep, seed=1000 * rank)
+    wl = workloads.make(args.workload, n=args.n, workers=args.workers, keep=args.keep, seed=multirank.rank_seed(rank))
     n, W = wl.n, wl.workers
     pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
     binding.ensure_workspace(n, pg, dev)
@@ -199,10 +198,10 @@ def main():
                 raise binding.FastSGDError(rc, "fastsgd_compress")
 
     def decompress_all():
-        for w in range(W):
-            rc = binding.decompress_accumulate(outs[w], cap, n, pg, dense)
-            if rc:
-                raise binding.FastSGDError(rc, "fastsgd_decompress_accumulate")
+        # all workers' streams in one launch (per 8 streams); same result as one call per stream
+        rc = binding.decompress_accumulate_batch(outs, [cap] * W, n, pg, dense)
+        if rc:
+            raise binding.FastSGDError(rc, "fastsgd_decompress_accumulate_batch")
 
     def step():
         compress_all()
@@ -217,9 +216,7 @@ def main():
     kept = [d for _, d, _ in infos]
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        multirank.barrier(world, cuda=True)
 
     def timed(fn, steps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -229,28 +226,53 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return multirank.max_over_ranks(e0.elapsed_time(e1), world, dev)
+
+    l0 = binding.launch_count()
+    step()
+    launches_per_step = binding.launch_count() - l0
+
+    def make_graph(fn):
+        """The same C-ABI calls, captured once into a CUDA graph and replayed (cuts launch gaps)."""
+        if args.no_graph:
+            return None
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            g.replay()
+            torch.cuda.synchronize()
+            return g
+        except Exception as exc:      # capture not possible: stay eager
+            print(f"[bench] CUDA graph capture failed, launching eagerly: {exc}", file=sys.stderr)
+            return None
+
+    g_step, g_comp, g_dec = make_graph(step), make_graph(compress_all), make_graph(decompress_all)
+    run_step = g_step.replay if g_step else step
+    run_comp = g_comp.replay if g_comp else compress_all
+    run_dec = g_dec.replay if g_dec else decompress_all
 
     for _ in range(args.warmup):
-        step()
+        run_step()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = binding.launch_count()
-    ms_total = timed(step, args.steps)
-    launches = binding.launch_count() - launches0
+    ms_total = timed(run_step, args.steps)
+    launches = launches_per_step * args.steps
     sampler.sample_once()
     sampler.stop()
     ms_step = ms_total / args.steps
 
     # separate phases (same protocol, fewer steps)
     sub = max(3, min(args.steps, 50))
-    ms_comp = timed(compress_all, sub) / sub
-    ms_dec = timed(decompress_all, sub) / sub
+    ms_comp = timed(run_comp, sub) / sub
+    ms_dec = timed(run_dec, sub) / sub
+    assert all(binding.stream_info(o)[2] == 0 for o in outs) and binding.decode_status() == 0
 
     # per-kernel durations from CUDA events recorded on the launching stream
     binding.kernel_timing_enable(True)
@@ -278,7 +300,7 @@ def main():
     per_launch_bytes = {
         "k_abs_sum": 4.0 * n + 8.0 * ((n + 16383) // 16384),
         "k_compress": 8.0 * n + float(sum(stream_bytes)) / W,
-        "k_decode_accumulate": float(sum(stream_bytes)) / W + 8.0 * float(sum(kept)) / W,
+        "k_decode_accumulate": (float(sum(stream_bytes)) + 8.0 * float(sum(kept))) / max(1, (W + 7) // 8),
     }
     kernels = {}
     for k, (ms, cnt) in ktimes.items():
@@ -303,6 +325,7 @@ def main():
         "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "n": n, "workers": W,
                    "keep_fraction": wl.keep_fraction, "base": wl.base, "tau": wl.tau, "flag_bits": wl.flag_bits,
                    "group_log2": wl.group_log2, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "launch": "cuda graph replay of the step's C-ABI calls" if g_step else "eager C-ABI calls",
                    "l2": "inputs of one step (W x 4n bytes) exceed L2; no explicit flush" if in_bytes > 126e6
                          else "inputs fit in L2: L2-warm number"},
         "clocks": sampler.summary(),
@@ -340,18 +363,12 @@ def main():
 
         e2e_steps = max(2, min(args.steps, 5))
         e2e_step()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        barrier()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             e2e_step()
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = multirank.max_over_ranks(time.perf_counter() - t0, world, dev)
         line["e2e"] = {"value": in_bytes * world * e2e_steps / dt / 1e9, "unit": UNIT, "steps": e2e_steps,
                        "h2d_bytes_per_step": int(4 * n * W + sum(produced)),
                        "d2h_bytes_per_step": int(sum(produced) + 64 * W + 4 * n + 8)}

@@ -122,6 +122,20 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
 int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
                                   const fastsgd_params* params, float* dense_out, void* stream);
 
+/*
+ * The same decoder and aggregation for the streams of several workers in one
+ * launch (Sec. 2.1: the W workers' decoded gradients are aggregated).
+ *   streams_in   host array of num_streams device pointers (each 16-byte
+ *                aligned), bytes the matching host array of valid byte counts
+ * The result equals that of num_streams calls of
+ * fastsgd_decompress_accumulate in the given order, bit for bit: a group's
+ * streams are applied one after the other.  Up to 8 streams go into one
+ * kernel launch; longer lists take several launches.
+ */
+int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uint64_t* bytes,
+                                        uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                        float* dense_out, void* stream);
+
 /* ---- helpers, not on the timed path (no counterpart in the paper) ---------- */
 
 /* worst-case stream size in bytes (every entry kept, every delta at the widest

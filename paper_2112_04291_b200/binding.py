@@ -21,7 +21,7 @@ ST_BAD_MAGIC, ST_BAD_VERSION, ST_BAD_STATUS, ST_N_MISMATCH, ST_PARAM_MISMATCH = 
 ST_TRUNCATED, ST_BAD_DIRECTORY, ST_BAD_KEY, ST_BAD_CODE = 21, 22, 23, 24
 
 EXPORTS = [
-    "fastsgd_compress", "fastsgd_decompress_accumulate", "fastsgd_compress_bound",
+    "fastsgd_compress", "fastsgd_decompress_accumulate", "fastsgd_decompress_accumulate_batch", "fastsgd_compress_bound",
     "fastsgd_workspace_bytes", "fastsgd_set_workspace", "fastsgd_stream_info",
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
@@ -62,6 +62,8 @@ def lib():
         L.fastsgd_compress.argtypes = [vp, u64, PP, vp, u64, vp]
         L.fastsgd_decompress_accumulate.restype = C.c_int
         L.fastsgd_decompress_accumulate.argtypes = [vp, u64, u64, PP, vp, vp]
+        L.fastsgd_decompress_accumulate_batch.restype = C.c_int
+        L.fastsgd_decompress_accumulate_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, vp]
         L.fastsgd_compress_bound.restype = u64
         L.fastsgd_compress_bound.argtypes = [u64, PP]
         L.fastsgd_workspace_bytes.restype = u64
@@ -151,6 +153,17 @@ def decompress_accumulate(stream_in: torch.Tensor, nbytes: int, n: int, p: Param
     assert dense.is_cuda and dense.dtype == torch.float32 and dense.is_contiguous() and dense.numel() == n
     return lib().fastsgd_decompress_accumulate(stream_in.data_ptr(), int(nbytes), int(n), C.byref(p),
                                                dense.data_ptr(), _stream_handle(stream))
+
+
+def decompress_accumulate_batch(streams_in, nbytes, n: int, p: Params, dense: torch.Tensor, stream=None) -> int:
+    """fastsgd_decompress_accumulate_batch: all workers' streams in one launch (per 8 streams)."""
+    assert dense.is_cuda and dense.dtype == torch.float32 and dense.is_contiguous() and dense.numel() == n
+    k = len(streams_in)
+    assert all(s.is_cuda and s.dtype == torch.uint8 for s in streams_in) and len(nbytes) == k
+    ptrs = (C.c_void_p * k)(*[int(s.data_ptr()) for s in streams_in])
+    sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
+    return lib().fastsgd_decompress_accumulate_batch(ptrs, sizes, k, int(n), C.byref(p), dense.data_ptr(),
+                                                     _stream_handle(stream))
 
 
 def stream_info(stream_in: torch.Tensor, stream=None):

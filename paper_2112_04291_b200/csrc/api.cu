@@ -27,7 +27,6 @@ struct State {
     int        sum_blocks_per_sm = 0;
     int        dec_blocks_per_sm = 0;
     int        cmp_blocks_per_sm = 0;
-    unsigned long long barrier_base = 0;   // value of Control::barrier once all enqueued compress calls are done
     bool       attrs_set = false;
 };
 State g_state;
@@ -117,7 +116,9 @@ int ensure_device_setup() {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
     g_state.cmp_blocks_per_sm = b3;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, k_decode_accumulate, kDecThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, k_decode_accumulate, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
     g_state.device = dev;
     g_state.sm_count = sms;
     g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
@@ -212,7 +213,7 @@ uint64_t fastsgd_workspace_bytes(uint64_t n, const fastsgd_params* params) {
 int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
     if (!dev_ptr) return FASTSGD_E_NULL;
     if (!aligned(dev_ptr, 256)) return FASTSGD_E_ALIGN;
-    if (bytes < kPartialsOffset) return FASTSGD_E_NO_WORKSPACE;
+    if (bytes < kPartialsOffset) return FASTSGD_E_NO_WORKSPACE;   // control block, tables, trace, decoder queue
     std::lock_guard<std::mutex> lock(g_state.mu);
     int rc = ensure_device_setup();
     if (rc) return rc;
@@ -222,7 +223,6 @@ int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
         return FASTSGD_E_CUDA;
     g_state.ws = dev_ptr;
     g_state.ws_bytes = bytes;
-    g_state.barrier_base = 0;
     return FASTSGD_OK;
 }
 
@@ -267,7 +267,7 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     ca.grad = grad; ca.n = n; ca.out = static_cast<uint8_t*>(out); ca.out_bytes = out_bytes;
     ca.ctl = w.ctl; ca.partials = w.partials; ca.desc = w.desc;
     ca.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
-    ca.base = params->base; ca.barrier_target = g_state.barrier_base + grid;
+    ca.base = params->base;
     ca.G = (uint32_t)G; ca.tau = params->tau; ca.l = params->flag_bits;
     void* kargs[] = {&ca, &pw};
     cudaError_t err;
@@ -277,43 +277,67 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
                                           sizeof(CmpSmem), st);
     }
     if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
-    g_state.barrier_base += grid;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return FASTSGD_OK;
 }
 
-int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
-                                  const fastsgd_params* params, float* dense_out, void* stream) {
-    if (!stream_in || !dense_out || !params) return FASTSGD_E_NULL;
-    if (!aligned(stream_in, 16) || !aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
+int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uint64_t* bytes,
+                                        uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                        float* dense_out, void* stream) {
+    if (!streams_in || !bytes || !dense_out || !params) return FASTSGD_E_NULL;
+    if (!aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
     PowTable pw;
     int rc = check_params(params, &pw);
     if (rc) return rc;
     rc = check_n(n);
     if (rc) return rc;
-    if (bytes < kHeaderBytes) return FASTSGD_E_TRUNCATED;
+    for (uint32_t i = 0; i < num_streams; ++i) {
+        if (!streams_in[i]) return FASTSGD_E_NULL;
+        if (!aligned(streams_in[i], 16)) return FASTSGD_E_ALIGN;
+        if (bytes[i] < kHeaderBytes) return FASTSGD_E_TRUNCATED;
+    }
     std::lock_guard<std::mutex> lock(g_state.mu);
-    if (!g_state.ws) return FASTSGD_E_NO_WORKSPACE;
+    if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
     const uint64_t G = groups_of(n, params->group_log2);
-    DecArgs da;
-    da.stream = static_cast<const uint8_t*>(stream_in); da.bytes = bytes; da.n = n; da.dense = dense_out;
-    da.status = &view(g_state.ws, n).ctl->decode_status;
-    da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
-    da.group_log2 = params->group_log2;
     const int warps_per_block = kDecThreads / 32;
     uint64_t grid = (G + warps_per_block - 1) / warps_per_block;
     const uint64_t cap = (uint64_t)g_state.sm_count * g_state.dec_blocks_per_sm;
     if (grid > cap) grid = cap;
     const uint64_t min_grid = (G + kDecListMax - 1) / kDecListMax;     // a block owns at most kDecListMax groups
     if (grid < min_grid) grid = min_grid;
-    {
-        LaunchTimer lt(2, static_cast<cudaStream_t>(stream));
-        k_decode_accumulate<<<(unsigned)grid, kDecThreads, 0, static_cast<cudaStream_t>(stream)>>>(da, pw);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (uint32_t first = 0; first < num_streams; first += kDecMaxStreams) {
+        DecArgs da;
+        std::memset(&da, 0, sizeof(da));
+        da.W = num_streams - first < (uint32_t)kDecMaxStreams ? num_streams - first : (uint32_t)kDecMaxStreams;
+        for (uint32_t i = 0; i < da.W; ++i) {
+            da.stream[i] = static_cast<const uint8_t*>(streams_in[first + i]);
+            da.bytes[i] = bytes[first + i];
+        }
+        da.n = n; da.dense = dense_out;
+        da.status = &view(g_state.ws, n).ctl->decode_status;
+        da.trace = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(g_state.ws) + kTraceOffset);
+        da.q_ctl = view(g_state.ws, n).ctl->dq;
+        da.q_list = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kQueueOffset);
+        da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
+        da.group_log2 = params->group_log2;
+        {
+            LaunchTimer lt(2, st);
+            k_decode_accumulate<<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+        }
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;
     }
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+    return FASTSGD_OK;
+}
+
+int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,
+                                  const fastsgd_params* params, float* dense_out, void* stream) {
+    if (!stream_in) return FASTSGD_E_NULL;
+    const void* one[1] = {stream_in};
+    return fastsgd_decompress_accumulate_batch(one, &bytes, 1u, n, params, dense_out, stream);
 }
 
 int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_bytes, uint64_t* d, int* status) {
@@ -403,8 +427,8 @@ int fastsgd_decompress_accumulate_host(const void* const* streams_host, const ui
         if (bytes[i] > need - dense_bytes) return FASTSGD_E_NO_WORKSPACE;
         // the staging area is reused: stream order keeps copy i+1 behind decode i
         if (cudaMemcpyAsync(dstream, streams_host[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
-        int rc = fastsgd_decompress_accumulate(dstream, bytes[i], n, params, ddense, stream);
-        if (rc) return rc;
+        int rc2 = fastsgd_decompress_accumulate(dstream, bytes[i], n, params, ddense, stream);
+        if (rc2) return rc2;
     }
     if (cudaMemcpyAsync(dense_host, ddense, 4ull * n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
     int dst = 0;

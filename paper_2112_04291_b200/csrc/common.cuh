@@ -35,15 +35,19 @@ struct Control {
     unsigned int       skip;           // 0 encode normally, 1 sum == 0, 2 sum not finite
     unsigned long long decode_status;  // min over failures of (group << 32 | key index << 8 | status)
     double             sum;            // S
-    unsigned long long barrier;        // blocks that have reached the grid barrier, over all calls so far
+    unsigned int       bar_count;      // blocks that have reached the grid barrier of the running call
+    unsigned int       bar_gen;        // bumped by the last block to arrive (sense of the barrier)
     unsigned long long trace[8];       // %globaltimer of block 0 at its phase boundaries (profiling aid)
-    unsigned int       pad[38];
+    unsigned int       dq[6];          // decoder work queue: pushed, taken, done, exited, reserved (zero between launches)
+    unsigned int       pad[32];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
 constexpr uint64_t kThrOffset      = 256;    // float thr[132]: RU32(B_k)
 constexpr uint64_t kTraceOffset    = 1024;   // u64 trace[<=496][8]: per-block %globaltimer stamps (profiling aid)
-constexpr uint64_t kPartialsOffset = 32768;  // double partial[chunks], then u64 desc[G]
+constexpr uint64_t kQueueOffset    = 32768;  // u32 queue[2^17]: decoder's grid-wide queue of groups (zero between launches)
+constexpr uint64_t kQueueBytes     = 4ull << 17;
+constexpr uint64_t kPartialsOffset = kQueueOffset + kQueueBytes;  // double partial[chunks], then u64 desc[G]
 
 struct WorkspaceView {
     Control*            ctl;

@@ -84,7 +84,6 @@ struct CmpArgs {
     unsigned long long* desc;
     unsigned char*      dense_scratch;
     double              base;
-    unsigned long long  barrier_target;
     uint32_t            G;
     uint32_t            tau;
     uint32_t            l;
@@ -128,6 +127,11 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 }
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 __device__ __forceinline__ unsigned long long read_globaltimer() {
     unsigned long long t;
@@ -424,7 +428,9 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
     unsigned long long t_wait = 0ull, t_pack = 0ull;
     if (tid == 0) btrace[0] = read_globaltimer();
 
+    unsigned int my_gen = 0u;
     if (tid == 0) {
+        my_gen = ld_acquire_u32(&a.ctl->bar_gen);      // before this block can arrive at the barrier
         for (int st = 0; st < kStages; ++st) mbar_init(&s.mbar[st], 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s.abort_flag = 0u;
@@ -472,12 +478,21 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
     __threadfence();
     __syncthreads();
     if (tid == 0 && !s.abort_flag) {
-        atomicAdd(&a.ctl->barrier, 1ull);
-        uint32_t spin = 0;
-        while (ld_acquire_u64(&a.ctl->barrier) < a.barrier_target) {
-            if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
-            __nanosleep(64);
+        // sense-reversing barrier: the last block to arrive clears the count and bumps the generation
+        // every block read when it started (no state outside the workspace, so a launch can be replayed)
+        const unsigned int old = atomicAdd(&a.ctl->bar_count, 1u);
+        if (old == grid - 1u) {
+            a.ctl->bar_count = 0u;
+            __threadfence();
+            atomicAdd(&a.ctl->bar_gen, 1u);
+        } else {
+            uint32_t spin = 0;
+            while (ld_acquire_u32(&a.ctl->bar_gen) == my_gen) {
+                if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
+                __nanosleep(64);
+            }
         }
+        __threadfence();
     }
     __syncthreads();
     bool aborted = s.abort_flag != 0u;

@@ -1,46 +1,66 @@
-// Decoder (decoder phases 1-4) and aggregation.
+// Decoder (decoder phases 1-4) and aggregation, for one stream or for several workers' streams
+// of the same gradient in one launch.
 //
 // Phase 1: the length flags give every delta's width; an exclusive scan of the widths gives
 // its bit offset.  Phase 2: an inclusive scan of the deltas, started at g*T, gives the keys
 // back.  Phases 3-4: code L -> sum / b^L (the boundary B_L rounded to fp32), signed.  The
-// aggregation adds the value into dense_out[key].  Keys are unique within a stream and calls
-// are ordered by the CUDA stream, so the read-modify-write needs no atomics and the result
-// does not depend on the launch shape.
+// aggregation adds the value into dense_out[key].  Keys are unique within a stream, and the
+// streams of one launch are applied to a group in their given order by the same warp or block,
+// so the read-modify-write needs no atomics and the result equals that of one call per stream.
 //
-// Work split: a group with few keys is decoded by one warp, a group with many keys by the
+// Work split: a group whose streams all hold few keys is decoded by one warp, any other by the
 // whole block; either way a thread owns a run of consecutive keys, so that the scans are one
-// shuffle scan (plus one shared-memory step for the block) per group instead of one per 32 keys,
-// and a group is validated in full before any of it is applied.
+// shuffle scan (plus one shared-memory step for the block) per group, and a group is validated
+// in full before any of it is applied.  The blobs of all streams of a group are first copied
+// into shared memory with coalesced loads (one memory round trip for all of them), then parsed
+// from there.
 #pragma once
+
+#include <cstddef>
 
 #include "common.cuh"
 #include "encode.cuh"
+#include "compress.cuh"     // mbarrier / bulk-copy primitives
 
 namespace fsg {
 
-constexpr int      kDecThreads   = 256;
-constexpr int      kDecWarps     = kDecThreads / 32;
-constexpr uint32_t kDecWarpMax   = 128;     // groups with more keys go to the whole block
-constexpr int      kDecListMax   = 512;     // groups one block may own
+constexpr int      kDecThreads     = 256;
+constexpr int      kDecWarps       = kDecThreads / 32;
+constexpr int      kDecMaxStreams  = 8;       // streams per launch
+constexpr uint32_t kDecWarpMax     = 128;     // groups with more keys (in any stream) go to the whole block
+constexpr int      kDecListMax     = 512;     // groups one block may own
+constexpr uint32_t kWarpStageWords = 1088;    // >= kDecMaxStreams * ceil(128 * (8 + 5 + 20) / 32)
+constexpr uint32_t kBlockStageWords = 10240;  // blobs larger than this in total are parsed from global memory
+constexpr uint32_t kDecSpinLimit   = 1u << 20;
 
 struct DecArgs {
-    const uint8_t*      stream;
-    uint64_t            bytes;
+    const uint8_t*      stream[kDecMaxStreams];
+    uint64_t            bytes[kDecMaxStreams];
     uint64_t            n;
     float*              dense;
     unsigned long long* status;     // sticky minimum of (group << 32 | key index << 8 | status)
+    unsigned int*       q_ctl;      // {pushed, taken, done, exited, reserved}: queue of groups for whole blocks, shared by the grid
+    unsigned int*       q_list;     // its G slots
+    unsigned long long* trace;      // per-block stamps (profiling aid)
     double              base;
+    uint32_t            W;          // streams in this launch
     uint32_t            G;
     uint32_t            tau;
     uint32_t            l;
     uint32_t            group_log2;
 };
 
+__device__ __forceinline__ unsigned long long read_globaltimer_dec() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 __device__ __forceinline__ void dec_fail(const DecArgs& a, uint32_t g, uint32_t j, int st) {
     atomicMin(a.status, ((unsigned long long)g << 32) | ((unsigned long long)(j & 0xFFFFFFu) << 8) | (unsigned)st);
 }
 
-__device__ __forceinline__ int check_header(const DecArgs& a, const uint32_t* w, uint64_t* total_out, double* sum_out) {
+__device__ __forceinline__ int check_header(const DecArgs& a, uint64_t bytes, const uint32_t* w, uint64_t* total_out, double* sum_out) {
     if (w[0] != kMagic) return kStBadMagic;
     if (w[1] != kVersion) return kStBadVersion;
     if (w[2] != (uint32_t)kStOk) return kStBadStatus;
@@ -52,22 +72,45 @@ __device__ __forceinline__ int check_header(const DecArgs& a, const uint32_t* w,
         return kStParamMismatch;
     const uint64_t total = (uint64_t)w[8] | ((uint64_t)w[9] << 32);
     const uint64_t fixed = (uint64_t)kHeaderBytes + 8ull * a.G;
-    if (total > a.bytes || total < fixed || (total & 3ull)) return kStTruncated;
+    if (total > bytes || total < fixed || (total & 3ull)) return kStTruncated;
     *total_out = total;
     *sum_out = __longlong_as_double((long long)((unsigned long long)w[10] | ((unsigned long long)w[11] << 32)));
     return kStOk;
 }
 
 struct DecShared {
-    float              val[132];
+    float              val[kDecMaxStreams][132];
+    double             sum[kDecMaxStreams];
+    uint32_t           total_words[kDecMaxStreams];
+    uint32_t           ok[kDecMaxStreams];
     uint32_t           scan[kDecWarps];
     uint32_t           big[kDecListMax];
     unsigned long long first_bad;     // min over threads of (key index << 8 | status), block path
     uint32_t           big_count;
-    int                status;
-    unsigned long long total;
-    double             sum;
+    uint32_t           pad;
+    unsigned long long tile_bar;      // mbarrier of the bulk copy that loads the tile
+    // per stream, for the group the block works on
+    uint32_t           g_count[kDecMaxStreams], g_M[kDecMaxStreams], g_off[kDecMaxStreams], g_nwords[kDecMaxStreams],
+                       g_base[kDecMaxStreams], g_valid[kDecMaxStreams];
+    uint32_t           bstage[kBlockStageWords];
+    union alignas(128) {               // (bulk copies need 16-byte aligned shared addresses)
+        uint32_t       wstage[kDecWarps][kWarpStageWords];   // warp path: the streams' blobs of a small group
+        float          tile[1u << 14];                       // block path: the group's slice of dense_out
+    } u;
 };
+static_assert(sizeof(DecShared) <= 113 * 1024, "two blocks per SM");
+static_assert(offsetof(DecShared, u) % 128 == 0, "tile alignment");
+
+// bits [pos, pos+nb) of a most-significant-bit-first sequence held as little-endian 32-bit words
+// (shared or global memory); nb <= 32
+__device__ __forceinline__ uint32_t get_bits(const uint32_t* words, uint32_t nwords, uint32_t pos, uint32_t nb) {
+    const uint32_t wi = pos >> 5, sh = pos & 31u;
+    const uint32_t w0 = wi < nwords ? bswap32(words[wi]) : 0u;
+    const uint32_t w1 = (wi + 1u) < nwords ? bswap32(words[wi + 1u]) : 0u;
+    const unsigned long long both = ((unsigned long long)w0 << 32) | w1;
+    if (nb == 0) return 0u;
+    return (uint32_t)((both >> (64u - sh - nb)) & ((nb >= 32u) ? 0xFFFFFFFFull : ((1ull << nb) - 1ull)));
+}
 
 // exclusive scan of one value per thread over the warp (BLOCK = false) or the block; also returns the total
 template <bool BLOCK>
@@ -91,38 +134,51 @@ __device__ __forceinline__ uint32_t excl_scan(uint32_t v, uint32_t* total, DecSh
     return before + incl - v;
 }
 
-// One group, decoded by a warp (BLOCK = false, `t` = lane, `nthreads` = 32) or by the block.
-template <bool BLOCK>
-__device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* __restrict__ sw,
-                                             uint32_t g, uint32_t total_words, uint32_t fixed_words,
-                                             int t, int nthreads, int lane, int warp) {
+// Directory entry of group g in one stream, checked.  Returns false (and records the status) if
+// it is inconsistent.  count = 0 for an empty group.
+__device__ __forceinline__ bool read_dir(const DecArgs& a, const uint32_t* sw, uint32_t g, uint32_t total_words,
+                                         uint32_t* count, uint32_t* M, uint32_t* off, uint32_t* nwords) {
+    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
     const uint32_t* dir = sw + (kHeaderBytes >> 2);
-    const uint32_t e0 = __ldg(dir + 2 * g), off = __ldg(dir + 2 * g + 1);
+    const uint32_t e0 = __ldg(dir + 2 * g), o = __ldg(dir + 2 * g + 1);
     const uint32_t next_off = (g + 1 < a.G) ? __ldg(dir + 2 * g + 3) : total_words;
-    const uint32_t count = e0 & 0xFFFFFFu, M = e0 >> 24;
+    const uint32_t c = e0 & 0xFFFFFFu, m = e0 >> 24;
+    *count = 0; *M = m; *off = o; *nwords = 0;
+    if ((g == 0 && o != fixed_words) || next_off < o || next_off > total_words || o < fixed_words) {
+        dec_fail(a, g, 0u, kStBadDirectory);
+        return false;
+    }
+    if (c == 0) {
+        if (e0 != 0u || next_off != o) { dec_fail(a, g, 0u, kStBadDirectory); return false; }
+        return true;
+    }
     const uint64_t lo64 = (uint64_t)g << a.group_log2;
-    const uint32_t lo = (uint32_t)lo64;
     const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+    const uint32_t span = (uint32_t)((hi64 < a.n ? hi64 : a.n) - lo64);
+    const uint32_t nw = next_off - o;
+    // (a blob is never longer than count * (8 + l + M) bits rounded up to words: also bounds the staging copy)
+    if (c > span || m < 1u || m > a.group_log2 || (uint64_t)(8u + a.l) * c > 32ull * nw ||
+        (uint64_t)nw > ((uint64_t)c * (8u + a.l + m) + 31ull) / 32ull) {
+        dec_fail(a, g, 0u, kStBadDirectory);
+        return false;
+    }
+    *count = c; *nwords = nw;
+    return true;
+}
+
+// One group of one stream, decoded by a warp (BLOCK = false, `t` = lane, `nthreads` = 32) or by the
+// block from `blob` (shared memory copy, or global memory for very large blobs).
+template <bool BLOCK>
+__device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* blob, uint32_t nwords,
+                                             uint32_t g, uint32_t count, uint32_t M, const float* val, float* tile,
+                                             int t, int nthreads, int lane, int warp) {
+    const uint64_t lo64 = (uint64_t)g << a.group_log2;
+    const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+    const uint32_t lo = (uint32_t)lo64;
     const uint32_t hi = (uint32_t)(hi64 < a.n ? hi64 : a.n);
     const bool lead = (t == 0);
-    if ((g == 0 && off != fixed_words) || next_off < off || next_off > total_words || off < fixed_words) {
-        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
-        return;
-    }
-    if (count == 0) {
-        if ((e0 != 0u || next_off != off) && lead) dec_fail(a, g, 0u, kStBadDirectory);
-        return;
-    }
-    const uint32_t nwords = next_off - off;
-    const uint64_t avail_bits = 32ull * nwords;
     const uint32_t flag_pos0 = 8u * count;
-    const uint64_t delta_pos0_64 = (uint64_t)flag_pos0 + (uint64_t)a.l * count;
-    if (count > hi - lo || M < 1u || M > a.group_log2 || delta_pos0_64 > avail_bits) {
-        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
-        return;
-    }
-    const uint32_t delta_pos0 = (uint32_t)delta_pos0_64;
-    const uint32_t* blob = sw + off;
+    const uint32_t delta_pos0 = flag_pos0 + a.l * count;
     const uint32_t levels_m1 = (1u << a.l) - 1u;
 
     // this thread's run of consecutive keys [jb, je)
@@ -132,7 +188,7 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     // phase 1: widths from the flags; their sum fixes the blob's length, which must be the directory's
     uint32_t wsum = 0;
     for (uint32_t j = jb; j < je; ++j) {
-        const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+        const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
         wsum += ((f + 1u) * M + levels_m1) >> a.l;
     }
     uint32_t wtotal;
@@ -147,9 +203,9 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     {
         uint32_t pos = pos0;
         for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
             const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            dsum = min(dsum + get_bits_be(blob, nwords, pos, w), 1u << 21);   // saturates only when already invalid
+            dsum = min(dsum + get_bits(blob, nwords, pos, w), 1u << 21);   // saturates only when already invalid
             pos += w;
         }
     }
@@ -162,12 +218,12 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     {
         uint32_t pos = pos0, key = key0;
         for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * j, a.l);
+            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
             const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            const uint32_t delta = get_bits_be(blob, nwords, pos, w);
+            const uint32_t delta = get_bits(blob, nwords, pos, w);
             pos += w;
             key += delta;
-            const uint32_t code = (__ldg(blob + (j >> 2)) >> (8u * (j & 3u))) & 0xFFu;
+            const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
             if ((j > 0 && delta == 0u) || key >= hi) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey; break; }
             if ((code & 0x7Fu) + 1u > a.tau) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode; break; }
         }
@@ -188,7 +244,22 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
         return;
     }
 
-    // phases 3-4 and the aggregation, four keys at a time (distinct keys: no aliasing)
+    // phases 3-4 and the aggregation
+    if (BLOCK && tile != nullptr) {
+        // into the group's slice of dense_out held in shared memory (the caller loads and stores it)
+        uint32_t pos = pos0, key = key0;
+        for (uint32_t j = jb; j < je; ++j) {
+            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
+            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
+            key += get_bits(blob, nwords, pos, w);
+            pos += w;
+            const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+            const float mag = val[(code & 0x7Fu) + 1u];
+            tile[key - lo] = __fadd_rn(tile[key - lo], (code & 0x80u) ? -mag : mag);
+        }
+        return;
+    }
+    // straight into dense_out, four keys at a time (distinct keys: no aliasing)
     {
         uint32_t pos = pos0, key = key0;
         for (uint32_t j = jb; j < je; j += 4) {
@@ -197,12 +268,12 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
             for (int i = 0; i < 4; ++i) {
                 kk[i] = 0xFFFFFFFFu; vv[i] = 0.f;
                 if (j + i < je) {
-                    const uint32_t f = get_bits_be(blob, nwords, flag_pos0 + a.l * (j + i), a.l);
+                    const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * (j + i), a.l);
                     const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-                    key += get_bits_be(blob, nwords, pos, w);
+                    key += get_bits(blob, nwords, pos, w);
                     pos += w;
-                    const uint32_t code = (__ldg(blob + ((j + i) >> 2)) >> (8u * ((j + i) & 3u))) & 0xFFu;
-                    const float mag = s.val[(code & 0x7Fu) + 1u];
+                    const uint32_t code = (blob[(j + i) >> 2] >> (8u * ((j + i) & 3u))) & 0xFFu;
+                    const float mag = val[(code & 0x7Fu) + 1u];
                     kk[i] = key; vv[i] = (code & 0x80u) ? -mag : mag;
                 }
             }
@@ -216,43 +287,178 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
 
 __global__ void __launch_bounds__(kDecThreads)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
-    __shared__ DecShared s;
+    extern __shared__ __align__(128) unsigned char dec_smem_raw[];
+    DecShared& s = *reinterpret_cast<DecShared*>(dec_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t* sw = reinterpret_cast<const uint32_t*>(a.stream);
+    const uint32_t W = a.W;
+    // per-block %globaltimer stamps (profiling aid): start, tables ready, own groups done, end; groups taken from the queue
+    unsigned long long T0 = 0, T1 = 0, T2 = 0; unsigned int taken = 0;
+    if (tid == 0) T0 = read_globaltimer_dec();
 
     if (tid == 0) {
+        mbar_init(&s.tile_bar, 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    uint32_t tile_parity = 0;
+    // ---- headers: thread w checks stream w
+    if (tid < (int)W) {
+        const uint32_t* sw = reinterpret_cast<const uint32_t*>(a.stream[tid]);
         uint32_t h[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) h[i] = __ldg(sw + i);
         uint64_t total = 0; double S = 0.0;
-        const int st = check_header(a, h, &total, &S);
-        s.status = st; s.total = total; s.sum = S; s.big_count = 0u;
+        const int st = check_header(a, a.bytes[tid], h, &total, &S);
+        s.ok[tid] = st == kStOk ? 1u : 0u;
+        s.total_words[tid] = (uint32_t)(total >> 2);
+        s.sum[tid] = S;
         if (st != kStOk && blockIdx.x == 0) dec_fail(a, 0u, 0u, st);
     }
     __syncthreads();
-    if (s.status != kStOk) return;
-    // phases 3-4 as a table: value[L] = (float)(sum / b^L)
-    if (tid <= (int)a.tau) s.val[tid] = __double2float_rn(__ddiv_rn(s.sum, pw.P[tid]));
-    __syncthreads();
-
-    const uint32_t total_words = (uint32_t)(s.total >> 2);
-    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
-    const uint32_t* dir = sw + (kHeaderBytes >> 2);
-
-    // this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
-    uint32_t i = warp;
-    for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += kDecWarps * gridDim.x, i += kDecWarps) {
-        const uint32_t count = __ldg(dir + 2 * g) & 0xFFFFFFu;
-        if (count > kDecWarpMax) {
-            if (lane == 0) { const uint32_t slot = atomicAdd(&s.big_count, 1u); if (slot < kDecListMax) s.big[slot] = g; }
-            continue;
-        }
-        decode_group<false>(a, s, sw, g, total_words, fixed_words, lane, 32, lane, warp);
+    // phases 3-4 as a table per stream: value[L] = (float)(sum / b^L)
+    for (uint32_t idx = tid; idx < W * 132u; idx += kDecThreads) {
+        const uint32_t w = idx / 132u, k = idx % 132u;
+        if (k <= a.tau && s.ok[w]) s.val[w][k] = __double2float_rn(__ddiv_rn(s.sum[w], pw.P[k]));
     }
     __syncthreads();
-    const uint32_t nbig = min(s.big_count, (uint32_t)kDecListMax);
-    for (uint32_t b = 0; b < nbig; ++b)
-        decode_group<true>(a, s, sw, s.big[b], total_words, fixed_words, tid, kDecThreads, lane, warp);
+
+    if (tid == 0) T1 = read_globaltimer_dec();
+    // ---- this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
+    for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += kDecWarps * gridDim.x) {
+        // lane w reads and checks stream w's directory entry
+        uint32_t count = 0, M = 0, off = 0, nwords = 0;
+        if (lane < (int)W && s.ok[lane])
+            read_dir(a, reinterpret_cast<const uint32_t*>(a.stream[lane]), g, s.total_words[lane], &count, &M, &off, &nwords);
+        if (!__any_sync(kFullMask, count != 0u)) continue;
+        if (__any_sync(kFullMask, count > kDecWarpMax)) {
+            if (lane == 0) {                 // hand it to the grid-wide queue: reserve a slot, then fill it (g + 1: 0 = empty)
+                const uint32_t slot = atomicAdd(a.q_ctl + 4, 1u);
+                __threadfence();
+                *reinterpret_cast<volatile unsigned int*>(a.q_list + slot) = g + 1u;
+            }
+            continue;
+        }
+        // copy the streams' blobs for this group into the warp's staging area
+        if (count == 0u) nwords = 0u;
+        const uint32_t nw_incl = warp_incl_scan(nwords, lane);
+        const uint32_t base = nw_incl - nwords;
+        uint32_t* stage = s.u.wstage[warp];
+        for (uint32_t w = 0; w < W; ++w) {
+            const uint32_t nw = __shfl_sync(kFullMask, nwords, w), b = __shfl_sync(kFullMask, base, w), o = __shfl_sync(kFullMask, off, w);
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(a.stream[w]) + o;
+            for (uint32_t i = lane; i < nw; i += 32) stage[b + i] = __ldg(src + i);
+        }
+        __syncwarp();
+        for (uint32_t w = 0; w < W; ++w) {
+            const uint32_t c = __shfl_sync(kFullMask, count, w);
+            const uint32_t b = __shfl_sync(kFullMask, base, w), nw = __shfl_sync(kFullMask, nwords, w), m = __shfl_sync(kFullMask, M, w);
+            if (c == 0u) continue;
+            decode_group<false>(a, s, stage + b, nw, g, c, m, s.val[w], nullptr, lane, 32, lane, warp);
+            __syncwarp();          // this stream's stores before the next stream's loads of the same keys
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+
+    if (tid == 0) T2 = read_globaltimer_dec();
+    // ---- groups with many keys sit in a queue shared by all blocks, so that a block that found
+    //      several of them does not hold the others up.  Slots are filled as the groups are found;
+    //      a taker waits (bounded) for its slot, or leaves once every block is past its own groups
+    //      and the slot lies beyond the last reservation.
+    unsigned int* q_taken = a.q_ctl + 1, *q_done = a.q_ctl + 2, *q_exited = a.q_ctl + 3, *q_reserved = a.q_ctl + 4;
+    if (tid == 0) { __threadfence(); atomicAdd(q_done, 1u); }
+    for (;;) {
+        if (tid == 0) {
+            uint32_t got = 0xFFFFFFFFu;
+            const uint32_t i = atomicAdd(q_taken, 1u);
+            uint32_t spin = 0;
+            for (;;) {
+                if (i < a.G) {
+                    const uint32_t e = *reinterpret_cast<volatile unsigned int*>(a.q_list + i);
+                    if (e != 0u) { got = e - 1u; *reinterpret_cast<volatile unsigned int*>(a.q_list + i) = 0u; break; }
+                }
+                if (*reinterpret_cast<volatile unsigned int*>(q_done) >= gridDim.x &&
+                    i >= *reinterpret_cast<volatile unsigned int*>(q_reserved)) break;      // nothing will fill it
+                if (i >= a.G || ++spin > kDecSpinLimit) break;
+                __nanosleep(100);
+            }
+            s.big[0] = got;
+        }
+        __syncthreads();
+        const uint32_t g = s.big[0];
+        if (g == 0xFFFFFFFFu) break;
+        ++taken;
+        const uint64_t lo64 = (uint64_t)g << a.group_log2;
+        const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+        const uint32_t lo = (uint32_t)lo64, span = (uint32_t)((hi64 < a.n ? hi64 : a.n) - lo64);
+        // The group's slice of dense_out is brought into shared memory by one bulk copy, updated there by
+        // every stream in turn, and written back by one bulk copy (needs 16-byte alignment and size).
+        const bool use_tile = a.group_log2 <= 14u && ((reinterpret_cast<uintptr_t>(a.dense) & 15u) == 0u) && ((span & 3u) == 0u);
+        if (use_tile && tid == 0) {
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the last write-back has read the tile
+            mbar_expect_tx(&s.tile_bar, span * 4u);
+            bulk_load(s.u.tile, a.dense + lo, span * 4u, &s.tile_bar);
+        }
+        if (tid < (int)W) {
+            uint32_t count = 0, M = 0, off = 0, nwords = 0;
+            if (s.ok[tid])
+                read_dir(a, reinterpret_cast<const uint32_t*>(a.stream[tid]), g, s.total_words[tid], &count, &M, &off, &nwords);
+            s.g_count[tid] = count; s.g_M[tid] = M; s.g_off[tid] = off; s.g_nwords[tid] = nwords;
+        }
+        __syncthreads();
+        // staging offsets; a blob that does not fit is parsed from global memory
+        uint32_t used = 0;
+        for (uint32_t w = 0; w < W; ++w) {
+            const uint32_t nw = s.g_count[w] ? s.g_nwords[w] : 0u;
+            const bool fits = used + nw <= kBlockStageWords;
+            if (tid == 0) { s.g_base[w] = used; s.g_valid[w] = fits ? 1u : 0u; }
+            if (fits) {
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(a.stream[w]) + s.g_off[w];
+                for (uint32_t i = tid; i < nw; i += kDecThreads) s.bstage[used + i] = __ldg(src + i);
+                used += nw;
+            }
+        }
+        __syncthreads();
+        if (use_tile) {
+            if (tid == 0) s.big[1] = mbar_wait(&s.tile_bar, tile_parity) ? 1u : 0u;     // bounded wait, one thread
+            __syncthreads();
+            tile_parity ^= 1u;
+            if (s.big[1] == 0u) {                                 // ran out: the group is skipped
+                if (tid == 0) dec_fail(a, g, 0u, kStTimeout);
+                __syncthreads();
+                continue;
+            }
+        }
+        for (uint32_t w = 0; w < W; ++w) {
+            const uint32_t c = s.g_count[w];
+            if (c == 0u) continue;
+            const uint32_t* blob = s.g_valid[w] ? s.bstage + s.g_base[w]
+                                                : reinterpret_cast<const uint32_t*>(a.stream[w]) + s.g_off[w];
+            decode_group<true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                               tid, kDecThreads, lane, warp);
+            __syncthreads();       // this stream's updates before the next stream's
+        }
+        if (use_tile && tid == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // the updates above, before the copy reads them
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(__cvta_generic_to_global(a.dense + lo)), "r"(smem_u32(s.u.tile)), "r"(span * 4u) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        __syncthreads();
+    }
+    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // write-backs complete before the block leaves
+    if (tid == 0 && blockIdx.x < 480u) {
+        a.trace[8u * blockIdx.x + 0] = T0; a.trace[8u * blockIdx.x + 1] = T1; a.trace[8u * blockIdx.x + 2] = T2;
+        a.trace[8u * blockIdx.x + 3] = read_globaltimer_dec(); a.trace[8u * blockIdx.x + 4] = taken;
+    }
+    // the last block to leave clears the counters for the next launch (the slots were cleared as they were taken)
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(q_exited, 1u) == gridDim.x - 1u) {
+            a.q_ctl[0] = 0u; *q_taken = 0u; *q_done = 0u; *q_reserved = 0u;
+            __threadfence();
+            *q_exited = 0u;
+        }
+    }
 }
 
 }  // namespace fsg

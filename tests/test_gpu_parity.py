@@ -258,3 +258,42 @@ def test_host_buffer_calls():
     oracle.decompress_accumulate(ostream, n, po, odense)
     oracle.decompress_accumulate(ostream, n, po, odense)
     assert rc == 0 and st == 0 and np.array_equal(dense.numpy(), odense)
+
+
+@pytest.mark.parametrize("nstreams", [1, 3, 8, 10])
+def test_batched_decode_equals_one_call_per_stream(nstreams):
+    # several workers' streams in one launch: same result, bit for bit, as sequential calls and as
+    # the oracle applied in the same order; the streams share many keys (same layer layout) and two
+    # of them are identical, so the per-group ordering matters
+    import torch
+    import gpu_util as G
+    n = 6 * 16384 + 321
+    rng = np.random.default_rng(nstreams)
+    dense0 = rng.standard_normal(n).astype(np.float32)
+    odense = dense0.copy()
+    streams, sizes, pg, po = [], [], None, None
+    base = None
+    for w in range(nstreams):
+        v = workloads.student_t_layers(n, seed=min(w, nstreams - 2) if nstreams > 1 else 0, blocks=5, lo=1e-3, hi=1e-1)
+        if base is None:
+            base = workloads.base_for_keep(v, n // 30)
+            pg, po = _params(base)
+        orc, ostream = oracle.compress(v, po)
+        rc, status, gstream, intact = G.gpu_compress(v, pg)
+        assert rc == 0 and status == 0 and np.array_equal(gstream, ostream)
+        assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+        pad = (-gstream.size) % 16
+        streams.append(G.to_dev(np.concatenate([gstream, np.zeros(pad + 16, np.uint8)])))
+        sizes.append(gstream.size)
+    binding.ensure_workspace(n, pg)
+    buf = G.Guarded(4 * n)
+    dense = buf.view.view(torch.float32)
+    dense.copy_(torch.from_numpy(dense0))
+    assert binding.decompress_accumulate_batch(streams, sizes, n, pg, dense) == 0
+    assert binding.decode_status() == 0 and buf.intact()
+    got = dense.cpu().numpy()
+    assert np.allclose(got, odense, rtol=RTOL, atol=ATOL) and np.array_equal(got, odense)
+    seq = torch.from_numpy(dense0).cuda()
+    for s, b in zip(streams, sizes):
+        assert binding.decompress_accumulate(s, b, n, pg, seq) == 0
+    assert np.array_equal(seq.cpu().numpy(), got)
