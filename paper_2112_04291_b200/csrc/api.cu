@@ -263,6 +263,10 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
     if (grid > kMaxCtas) grid = kMaxCtas;
     if (grid > G) grid = G;
+    {   // equal shares: every block gets the same number of tiles in the sum pass (+-0 when G divides)
+        const uint64_t rounds = (G + grid - 1) / grid;
+        grid = (G + rounds - 1) / rounds;
+    }
     CmpArgs ca;
     ca.grad = grad; ca.n = n; ca.out = static_cast<uint8_t*>(out); ca.out_bytes = out_bytes;
     ca.ctl = w.ctl; ca.partials = w.partials; ca.desc = w.desc;

@@ -38,6 +38,7 @@ constexpr uint32_t kArenaWords   = 4608;                      // packed blobs wa
 constexpr int      kPendMax      = 32;                        // tiles that may wait in the arena
 constexpr uint32_t kMaxCtas      = 320;                       // scratch slots for the dense path
 constexpr uint32_t kWaitLimit    = 1u << 22;                  // polls before a wait gives up
+constexpr int      kDrainChunks  = 4;                         // descriptors read at once when draining: 4 x 512
 constexpr uint32_t kDenseMark    = 0xFFFFFFFFu;               // arena offset of a blob that sits in global scratch
 // dense path scratch per block: values / blob u32[T] | keys u16[T] | codes u8[T]
 constexpr uint64_t kDenseScratchBytes = (uint64_t)kTile * 4u + (uint64_t)kTile * 2u + kTile;
@@ -50,7 +51,7 @@ struct CmpSmem {
     unsigned long long mbar[kStages];
     double   s_warp[2][kCmpWarps];
     double   s_tree[kCmpWarps];
-    unsigned long long scan64[kCmpWarps];
+    unsigned long long scan64[kDrainChunks][kCmpWarps];
     float    thr[132];
     // per-slab summaries, by tile parity (an empty tile has no second barrier)
     uint32_t sum_count[2][kCmpWarps];        // kept entries of the slab; bit 31: more than kSlabCap
@@ -68,6 +69,8 @@ struct CmpSmem {
     uint32_t abort_flag;
     uint32_t poison_seen;
     uint32_t pad;
+    uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
+    uint32_t pad2[2];
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
     uint16_t wkeys[kCmpWarps][kSlabCap];     // per warp: kept keys (tile-local), in index order
@@ -179,8 +182,19 @@ __device__ __forceinline__ double block_tree(double x, double* s_tree, int lane,
 __device__ __forceinline__ double reduce_partials(const double* partials, uint32_t chunks, double* s_tree,
                                                   double* s_nodes, int tid, int lane, int warp) {
     const uint32_t passes = (chunks + kCmpThreads - 1) / kCmpThreads;       // <= 256 for n < 2^31
-    if (passes == 1) {
-        const double x = (uint32_t)tid < chunks ? __ldcg(partials + tid) : 0.0;
+    if (passes <= 8) {
+        // thread t folds the aligned run of R = 1, 2, 4 or 8 partials that starts at R*t (all loads in
+        // flight at once), then one tree over the threads: the same tree, one barrier pair
+        const uint32_t R = passes <= 1 ? 1u : (passes <= 2 ? 2u : (passes <= 4 ? 4u : 8u));
+        double v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint64_t idx = (uint64_t)tid * R + k;
+            v[k] = ((uint32_t)k < R && idx < chunks) ? __ldcg(partials + idx) : 0.0;
+        }
+        // with R < 8 the unused slots are zero and x + 0 = x, so the full 8-leaf tree is still exact
+        const double x = __dadd_rn(__dadd_rn(__dadd_rn(v[0], v[1]), __dadd_rn(v[2], v[3])),
+                                   __dadd_rn(__dadd_rn(v[4], v[5]), __dadd_rn(v[6], v[7])));
         return block_tree(x, s_tree, lane, warp);
     }
     double next = (uint32_t)tid < chunks ? __ldcg(partials + tid) : 0.0;
@@ -220,7 +234,7 @@ __device__ __forceinline__ uint32_t code_byte_of(const float* thr, uint32_t tau,
 // Phase 2 for a tile too dense for the per-warp lists: block-wide compaction, quantisation,
 // deltas, M, flags, width scan and packing in the block's slot of global scratch (the blob reuses
 // the values' words).  `m` is the kept mask of this thread's 32 entries, `tile` the tile's entries
-// (shared memory).
+// (global memory: kept entries lie below n).
 __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, uint32_t count,
                                              uint32_t warp_base, uint32_t m, const float* tile,
                                              uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
@@ -320,55 +334,77 @@ struct ScanState {
 };
 
 // Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
-// group numbers ascend in steps of gridDim.x.  Returns false if a poisoned descriptor or a
+// group numbers ascend.  Returns false if a poisoned descriptor or a
 // timeout was met (the caller aborts).
 __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, ScanState& sc,
                                       double S, uint32_t skip, int tid, int lane, int warp) {
     if (npend == 0) return true;
-    const uint32_t g_first = s.pend_g[0], g_last = s.pend_g[npend - 1], grid = gridDim.x;
+    const uint32_t g_last = s.pend_g[npend - 1];
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
-    // ---- advance the scan over descriptors [sc.pos, g_last], 512 at a time
+    // ---- advance the scan over descriptors [sc.pos, g_last]: batches of kDrainChunks x 512, all loads
+    //      of a batch in flight at once, one shuffle scan per chunk, two barriers per batch
     while (sc.pos <= g_last) {
-        const uint32_t idx = sc.pos + tid;
-        unsigned long long d = 0ull;
-        if (idx <= g_last) {
+        unsigned long long own[kDrainChunks], excl[kDrainChunks];
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            const uint32_t idx = sc.pos + (uint32_t)j * kCmpThreads + tid;
+            own[j] = idx <= g_last ? ld_relaxed_u64(a.desc + idx) : desc_pack(kDescValid, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            const uint32_t idx = sc.pos + (uint32_t)j * kCmpThreads + tid;
             uint32_t spin = 0;
-            d = ld_relaxed_u64(a.desc + idx);
-            while ((d >> 62) == kDescInvalid) {             // not published yet: bounded poll
-                if (++spin > kWaitLimit) { s.poison_seen = 2u; d = 0ull; break; }
+            while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
+                if (++spin > kWaitLimit) { s.poison_seen = 2u; own[j] = 0ull; break; }
                 __nanosleep(64);
-                d = ld_relaxed_u64(a.desc + idx);
+                own[j] = ld_relaxed_u64(a.desc + idx);
             }
-            if ((d >> 62) == kDescPoison) { s.poison_seen = 1u; d = 0ull; }
-        }
-        const unsigned long long own = ((unsigned long long)desc_count(d) << 32) | desc_words(d);
-        unsigned long long incl = own;
+            if ((own[j] >> 62) == kDescPoison) { s.poison_seen = 1u; own[j] = 0ull; }
+            own[j] = ((unsigned long long)desc_count(own[j]) << 32) | desc_words(own[j]);
+            unsigned long long incl = own[j];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long t = __shfl_up_sync(kFullMask, incl, o);
-            if (lane >= o) incl += t;
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(kFullMask, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) s.scan64[j][warp] = incl;
+            excl[j] = incl - own[j];
         }
-        if (lane == 31) s.scan64[warp] = incl;
         __syncthreads();
-        unsigned long long before = ((unsigned long long)sc.count << 32) | sc.words, all = 0ull;
+        unsigned long long running = ((unsigned long long)sc.count << 32) | sc.words;
 #pragma unroll
-        for (int w = 0; w < kCmpWarps; ++w) {
-            const unsigned long long t = s.scan64[w];
-            if (w < warp) before += t;
-            all += t;
+        for (int j = 0; j < kDrainChunks; ++j) {
+            unsigned long long before = running, all = 0ull;
+#pragma unroll
+            for (int w = 0; w < kCmpWarps; ++w) {
+                const unsigned long long t = s.scan64[j][w];
+                if (w < warp) before += t;
+                all += t;
+            }
+            excl[j] += before;                               // exclusive prefix of descriptor sc.pos + 512 j + tid
+            running += all;
         }
         // the thread that holds one of this block's pending tiles records that tile's exclusive prefix
-        if (idx >= g_first && idx <= g_last && (idx - g_first) % grid == 0u)
-            s.pend_prefix[(idx - g_first) / grid] = before + incl - own;
-        sc.count += (uint32_t)(all >> 32);
-        sc.words += (uint32_t)all;
-        sc.pos += kCmpThreads;
+        for (int p = 0; p < npend; ++p) {
+            const uint32_t idx = s.pend_g[p];
+            if (idx < sc.pos || idx >= sc.pos + (uint32_t)kDrainChunks * kCmpThreads) continue;
+            const uint32_t rel = idx - sc.pos;
+            if ((rel % kCmpThreads) != (uint32_t)tid) continue;
+            const int jj = (int)(rel / kCmpThreads);
+            unsigned long long e = 0ull;
+#pragma unroll
+            for (int j = 0; j < kDrainChunks; ++j) if (j == jj) e = excl[j];
+            s.pend_prefix[p] = e;
+        }
+        sc.count = (uint32_t)(running >> 32);
+        sc.words = (uint32_t)running;
+        sc.pos += (uint32_t)kDrainChunks * kCmpThreads;
         const uint32_t poison_now = s.poison_seen;      // read between the barriers: same value in every thread
         __syncthreads();
         if (poison_now) return false;
     }
-    // the scan ran past g_last by whole steps of 512: pull it back to g_last + 1
+    // the scan ran past g_last by whole steps: pull it back to g_last + 1
     // (descriptors beyond g_last were read as zero, so only the position needs correcting)
     sc.pos = g_last + 1u;
 
@@ -449,6 +485,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         const int st = (int)(q % kStages);
         const uint32_t tile = c + (k - 1 - q) * grid;
         if (tid == 0) a.desc[tile] = 0ull;    // descriptors of phase 2 (ordered by the grid barrier)
+        if (tid == 0 && c == 0 && q == 0) a.ctl->ticket = grid;       // tiles below `grid` are taken: see phase 2
         if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
         parity ^= 1u << st;
         pending &= ~(1u << st);
@@ -496,6 +533,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
     }
     __syncthreads();
     bool aborted = s.abort_flag != 0u;
+    uint32_t held_now = 0xFFFFFFFFu, held_next = 0xFFFFFFFFu;     // thread 0: tiles taken and not yet published
 
     if (!aborted) {
         if (tracer) a.ctl->trace[2] = read_globaltimer();
@@ -527,9 +565,16 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         int npend = 0;
         uint32_t arena_used = 0;
         const uint32_t round_up = (1u << a.l) - 1u;
-        for (uint32_t i = 0; i < k && !aborted; ++i) {
-            const uint32_t g = c + i * grid;
-            const int st = (int)((k - 1 - (i % kStages)) % kStages);
+        // The block's first tile is the one it summed last (still in shared memory); every further tile
+        // is handed out by a ticket counter, so that blocks that met dense tiles take fewer.  Thread 0
+        // holds the ticket of the tile after the one at hand, taken a whole iteration before it is used.
+        static_assert(kStages == 1, "the encode pass keeps one tile in flight per block");
+        uint32_t g = c;
+        bool have = k > 0;
+        unsigned int ticket_ahead = 0u;
+        if (tid == 0 && have) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
+        for (uint32_t i = 0; have && !aborted; ++i) {
+            const int st = 0;
             const uint32_t par = i & 1u;
             if (i >= (uint32_t)kStages) {
                 const unsigned long long tw0 = tid == 0 ? read_globaltimer() : 0ull;
@@ -617,25 +662,36 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                     slab_last = wk[slab_count - 1];
                 }
             }
+            if (tid == 0) { s.next_tile[par] = ticket_ahead; held_now = g; held_next = ticket_ahead; }
             if (lane == 0) {
                 s.sum_count[par][warp] = slab_count | (slab_count > kSlabCap ? 0x80000000u : 0u);
                 s.sum_first[par][warp] = slab_first;
                 s.sum_last[par][warp] = slab_last;
                 s.sum_maxd[par][warp] = slab_maxd;
             }
-            __syncthreads();                       // summaries written; every thread has read its part of the stage
+            // barrier 1: summaries written, every thread has read its part of the stage; it also tells
+            // whether the tile holds any kept entry at all
+            const int any_kept = __syncthreads_or(m != 0u);
             if (s.abort_flag) { aborted = true; break; }
-            // ---- every warp combines the 16 summaries (lane w <-> slab w)
-            const uint32_t sc_raw = lane < kCmpWarps ? s.sum_count[par][lane] : 0u;
-            const uint32_t cnt_l = sc_raw & 0x7FFFFFFFu;
-            const uint32_t count = __reduce_add_sync(kFullMask, cnt_l);
-            const bool overflow = __any_sync(kFullMask, (sc_raw >> 31) != 0u);
-            const uint32_t cnt_incl = warp_incl_scan(cnt_l, lane);
-            const uint32_t warp_base = __shfl_sync(kFullMask, cnt_incl - cnt_l, warp);      // kept entries in the slabs before mine
-            const bool refill = i + kStages < k;
-            if (refill && !overflow) {             // every thread has read its part of the stage (a dense tile
-                issue_tile(s, a, st, c + (i + kStages) * grid, tid);      // still needs its values: refilled below)
+            // the stage is free: start the copy of the next tile at once (thread 0 knows its number
+            // already), then take the ticket for the one after
+            const uint32_t g_next = s.next_tile[par];
+            const bool refill = g_next < a.G;
+            if (refill) {
+                issue_tile(s, a, st, g_next, tid);
                 pending |= 1u << st;
+                if (tid == 0) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
+            }
+            // ---- every warp combines the 16 summaries (lane w <-> slab w)
+            uint32_t count = 0, warp_base = 0, cnt_l = 0;
+            bool overflow = false;
+            if (any_kept) {
+                const uint32_t sc_raw = lane < kCmpWarps ? s.sum_count[par][lane] : 0u;
+                cnt_l = sc_raw & 0x7FFFFFFFu;
+                count = __reduce_add_sync(kFullMask, cnt_l);
+                overflow = __any_sync(kFullMask, (sc_raw >> 31) != 0u);
+                const uint32_t cnt_incl = warp_incl_scan(cnt_l, lane);
+                warp_base = __shfl_sync(kFullMask, cnt_incl - cnt_l, warp);      // kept entries in the slabs before mine
             }
 
             uint32_t words = 0, M = 0, aoff = 0;
@@ -712,11 +768,8 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 aoff = kDenseMark;
-                pack_tile_dense(s, a, count, warp_base, m, tile, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
-                if (refill) {
-                    issue_tile(s, a, st, c + (i + kStages) * grid, tid);
-                    pending |= 1u << st;
-                }
+                pack_tile_dense(s, a, count, warp_base, m, a.grad + ((uint64_t)g << kGroupLog2), ex0, ex1, tot0, tot1,
+                                &words, &M, tid, lane, warp);      // (the stage is being refilled: values come from global memory)
             }
             if (tid == 0) {
                 t_pack += read_globaltimer() - tp0;
@@ -732,6 +785,8 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
             }
+            g = g_next;
+            have = refill;
         }
         if (tid == 0) btrace[4] = read_globaltimer();
         if (!aborted) {
@@ -748,7 +803,12 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         __syncthreads();
         if (tid == 0) {
             atomicExch(&a.ctl->error, (unsigned)kStTimeout);
-            for (uint32_t i = 0; i < k; ++i) st_relaxed_u64(a.desc + c + i * grid, desc_pack(kDescPoison, 0, 0));
+            if (held_now == 0xFFFFFFFFu) {            // still in the sum pass: nobody waits for descriptors yet
+                for (uint32_t i = 0; i < k; ++i) st_relaxed_u64(a.desc + c + i * grid, desc_pack(kDescPoison, 0, 0));
+            } else {
+                if (held_now < a.G) st_relaxed_u64(a.desc + held_now, desc_pack(kDescPoison, 0, 0));
+                if (held_next < a.G) st_relaxed_u64(a.desc + held_next, desc_pack(kDescPoison, 0, 0));
+            }
             for (int st = 0; st < kStages; ++st)
                 if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
             if (k > 0 && c + (k - 1) * grid == a.G - 1) {
