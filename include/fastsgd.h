@@ -67,6 +67,7 @@ typedef struct fastsgd_params {
 #define FASTSGD_E_NOT_IMPLEMENTED (-7)   /* valid parameters this build has no kernel for                    */
 #define FASTSGD_E_CUDA            (-8)   /* a CUDA runtime call failed                                       */
 #define FASTSGD_E_TRUNCATED       (-9)   /* decompress: fewer than 64 bytes given                            */
+#define FASTSGD_E_TOO_LARGE       (-10)  /* fastsgd_abs_sum_noalloc: n above FASTSGD_NOALLOC_MAX_N           */
 
 /* device-visible status words */
 #define FASTSGD_ST_OK              0
@@ -163,6 +164,36 @@ int fastsgd_decode_status(void* stream, int* status);
 /* Step 1 of Algorithm 1 alone: *sum_out (device, one double) = sum|v_i| on the
  * same fp64 pairwise tree fastsgd_compress uses.  Uses the workspace. */
 int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream);
+
+/*
+ * The same sum for callers that cannot hand the library any scratch memory.
+ * (The paper has no counterpart: this is a packaging variant of step 1 of
+ * Algorithm 1, bit-identical to fastsgd_abs_sum.)
+ *
+ * Who needs it: code that runs where device memory cannot be obtained at call
+ * time -- a plug-in inside a host application that owns the whole device heap,
+ * a latency-critical loop that must not hit cudaMalloc's implicit device-wide
+ * synchronisation or its failure under memory pressure, a component that is
+ * only ever given its input and output buffers.  Such a caller cannot register
+ * a workspace either, so the per-tile partial sums and the block counter live
+ * in a fixed array inside the library's own device image instead
+ * (about 129 KiB, held by every GPU that loads the library until the process
+ * exits).  The price is a size limit: n <= FASTSGD_NOALLOC_MAX_N, otherwise
+ * FASTSGD_E_TOO_LARGE is returned and nothing is launched.
+ *
+ *   grad     device, n floats, 16-byte aligned
+ *   sum_out  device, one double, 8-byte aligned
+ * The call allocates nothing and frees nothing, neither through the CUDA
+ * runtime nor through any library.  The first call on a device looks the
+ * array's device address up and queries launch limits (once per device, with
+ * that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps what the previous
+ * call left: the call clears the part that must start at zero itself, but two
+ * calls that overlap on the GPU (different streams, no ordering) race on it --
+ * issue them on one stream or order them yourself.
+ */
+#define FASTSGD_NOALLOC_MAX_N (1ull << 28)
+int fastsgd_abs_sum_noalloc(const float* grad, uint64_t n, double* sum_out, void* stream);
 
 /*
  * Host-buffer forms of the two calls, for callers whose gradients live in host

@@ -16,6 +16,8 @@ LIB_PATH = os.path.join(_PKG, "libfastsgd_b200.so")
 
 OK = 0
 E_NULL, E_ALIGN, E_BAD_PARAM, E_BAD_N, E_CAPACITY, E_NO_WORKSPACE, E_NOT_IMPLEMENTED, E_CUDA, E_TRUNCATED = range(-1, -10, -1)
+E_TOO_LARGE = -10
+NOALLOC_MAX_N = 1 << 28
 ST_OK, ST_NONFINITE, ST_CAPACITY, ST_TIMEOUT = 0, 1, 2, 3
 ST_BAD_MAGIC, ST_BAD_VERSION, ST_BAD_STATUS, ST_N_MISMATCH, ST_PARAM_MISMATCH = 16, 17, 18, 19, 20
 ST_TRUNCATED, ST_BAD_DIRECTORY, ST_BAD_KEY, ST_BAD_CODE = 21, 22, 23, 24
@@ -25,7 +27,7 @@ EXPORTS = [
     "fastsgd_workspace_bytes", "fastsgd_set_workspace", "fastsgd_stream_info",
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
-    "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read",
+    "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
 ]
 
 
@@ -88,6 +90,8 @@ def lib():
         L.fastsgd_strerror.argtypes = [C.c_int]
         L.fastsgd_version.restype = C.c_int
         L.fastsgd_version.argtypes = []
+        L.fastsgd_abs_sum_noalloc.restype = C.c_int
+        L.fastsgd_abs_sum_noalloc.argtypes = [vp, u64, vp, vp]
         L.fastsgd_kernel_timing_enable.restype = C.c_int
         L.fastsgd_kernel_timing_enable.argtypes = [C.c_int]
         L.fastsgd_kernel_timing_read.restype = C.c_int
@@ -183,6 +187,12 @@ def decode_status(stream=None) -> int:
 def abs_sum(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int:
     assert grad.is_cuda and grad.dtype == torch.float32 and out.is_cuda and out.dtype == torch.float64
     return lib().fastsgd_abs_sum(grad.data_ptr(), grad.numel(), out.data_ptr(), _stream_handle(stream))
+
+
+def abs_sum_noalloc(grad: torch.Tensor, out: torch.Tensor, stream=None) -> int:
+    """fastsgd_abs_sum_noalloc: the same sum, with the library's built-in scratch (no workspace needed)."""
+    assert grad.is_cuda and grad.dtype == torch.float32 and out.is_cuda and out.dtype == torch.float64
+    return lib().fastsgd_abs_sum_noalloc(grad.data_ptr(), grad.numel(), out.data_ptr(), _stream_handle(stream))
 
 
 def host_scratch_bytes(n: int, p: Params) -> int:

@@ -182,6 +182,7 @@ const char* fastsgd_strerror(int code) {
         case FASTSGD_E_NOT_IMPLEMENTED: return "parameter combination not implemented in this build";
         case FASTSGD_E_CUDA: return "CUDA runtime error";
         case FASTSGD_E_TRUNCATED: return "stream shorter than its header";
+        case FASTSGD_E_TOO_LARGE: return "n exceeds the built-in scratch of fastsgd_abs_sum_noalloc (2^28 entries)";
         case FASTSGD_ST_NONFINITE: return "sum of |v| is not finite";
         case FASTSGD_ST_CAPACITY: return "stream does not fit in the output buffer";
         case FASTSGD_ST_TIMEOUT: return "bounded wait between thread blocks ran out";
@@ -443,3 +444,86 @@ int fastsgd_decompress_accumulate_host(const void* const* streams_host, const ui
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// fastsgd_abs_sum_noalloc: the sum kernel with its scratch inside the library image.
+//
+// Some callers have no way to give the library scratch memory: they may not call cudaMalloc
+// (it synchronises the whole device and can fail when memory is tight), they do not own a
+// framework allocator, they only receive an input and an output pointer.  For them the
+// per-tile partials and the block counter of the sum kernel live in the array below: part of
+// the loaded module on every GPU, 256-byte aligned, never allocated and never freed.
+//
+// In host code the name `g_noalloc_scratch` is only a handle for the symbol, not a device
+// address; the address the kernel may use comes from cudaGetSymbolAddress, looked up once
+// per device with that device current.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint64_t kNoAllocMaxN      = FASTSGD_NOALLOC_MAX_N;                  // 2^28 entries = 1 GiB of fp32
+constexpr uint64_t kNoAllocPartials  = kNoAllocMaxN >> fsg::kChunkLog2;        // 16384 fp64 partials
+constexpr uint64_t kNoAllocCtlBytes  = 1024;                                   // control block + boundary table
+constexpr uint64_t kNoAllocBytes     = kNoAllocCtlBytes + 8ull * kNoAllocPartials;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+struct NoAllocDevice {
+    unsigned char* scratch = nullptr;     // device address of g_noalloc_scratch on this GPU
+    int            grid_cap = 0;          // blocks that fit the GPU at once
+};
+std::mutex     g_noalloc_mu;
+NoAllocDevice  g_noalloc_dev[kNoAllocMaxDevices];
+
+// once per device, with that device current; allocates nothing
+int noalloc_setup(int dev, NoAllocDevice** out) {
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return FASTSGD_E_CUDA;
+    NoAllocDevice& d = g_noalloc_dev[dev];
+    if (!d.scratch) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return FASTSGD_E_CUDA; }
+        int sms = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fsg::k_abs_sum, fsg::kSumThreads, 0) != cudaSuccess)
+            return FASTSGD_E_CUDA;
+        d.grid_cap = sms * (per_sm > 0 ? per_sm : 1);
+        d.scratch = static_cast<unsigned char*>(p);
+    }
+    *out = &d;
+    return FASTSGD_OK;
+}
+
+}  // namespace
+
+extern "C" int fastsgd_abs_sum_noalloc(const float* grad, uint64_t n, double* sum_out, void* stream) {
+    if (!grad || !sum_out) return FASTSGD_E_NULL;
+    if (!aligned(grad, 16) || !aligned(sum_out, 8)) return FASTSGD_E_ALIGN;
+    if (n == 0) return FASTSGD_E_BAD_N;
+    if (n > kNoAllocMaxN) return FASTSGD_E_TOO_LARGE;              // would not fit the built-in scratch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FASTSGD_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    NoAllocDevice* d = nullptr;
+    int rc = noalloc_setup(dev, &d);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps the previous call's contents.  Only the block counter has to start at zero
+    // (the kernel leaves it at zero, but a call that was cut short might not have): clear the
+    // control block on the stream.  Every partial that is read is written first by this call.
+    if (cudaMemsetAsync(d->scratch, 0, sizeof(fsg::Control), st) != cudaSuccess) return FASTSGD_E_CUDA;
+    fsg::SumArgs sa;
+    sa.grad = grad; sa.n = n; sa.chunks = (uint32_t)((n + fsg::kChunk - 1) >> fsg::kChunkLog2);
+    sa.groups = 0u; sa.tau = 0u;
+    sa.ctl = reinterpret_cast<fsg::Control*>(d->scratch);
+    sa.thr = reinterpret_cast<float*>(d->scratch + fsg::kThrOffset);
+    sa.partials = reinterpret_cast<double*>(d->scratch + kNoAllocCtlBytes);
+    sa.desc = nullptr;
+    sa.sum_out = sum_out;
+    fsg::PowTable pw;
+    for (int k = 0; k <= fsg::kMaxTau; ++k) pw.P[k] = 1.0;
+    unsigned grid = (unsigned)d->grid_cap;
+    if (grid > sa.chunks) grid = sa.chunks;
+    fsg::k_abs_sum<<<grid, fsg::kSumThreads, 0, st>>>(sa, pw);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? FASTSGD_OK : FASTSGD_E_CUDA;
+}
