@@ -35,10 +35,12 @@ constexpr int      kStages       = 1;
 constexpr uint32_t kTile         = 1u << kGroupLog2;          // entries per tile = per group
 constexpr uint32_t kSlabCap      = 192;                       // kept entries a warp's 1024-entry slab may have on the shared-memory path
 constexpr uint32_t kArenaWords   = 4608;                      // packed blobs waiting for their offsets
-constexpr int      kPendMax      = 32;                        // tiles that may wait in the arena
+constexpr int      kPendMax      = 128;                       // tiles that may wait in the arena
+constexpr uint32_t kArenaReserve = 1024;                      // drain ahead of time when less than this would be left
 constexpr uint32_t kMaxCtas      = 320;                       // scratch slots for the dense path
 constexpr uint32_t kWaitLimit    = 1u << 22;                  // polls before a wait gives up
 constexpr int      kDrainChunks  = 4;                         // descriptors read at once when draining: 4 x 512
+constexpr uint32_t kNoTicket     = 0xFFFFFFFEu;               // "no tile reserved": the block drains before it takes one
 constexpr uint32_t kDenseMark    = 0xFFFFFFFFu;               // arena offset of a blob that sits in global scratch
 // dense path scratch per block: values / blob u32[T] | keys u16[T] | codes u8[T]
 constexpr uint64_t kDenseScratchBytes = (uint64_t)kTile * 4u + (uint64_t)kTile * 2u + kTile;
@@ -673,15 +675,6 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
             // whether the tile holds any kept entry at all
             const int any_kept = __syncthreads_or(m != 0u);
             if (s.abort_flag) { aborted = true; break; }
-            // the stage is free: start the copy of the next tile at once (thread 0 knows its number
-            // already), then take the ticket for the one after
-            const uint32_t g_next = s.next_tile[par];
-            const bool refill = g_next < a.G;
-            if (refill) {
-                issue_tile(s, a, st, g_next, tid);
-                pending |= 1u << st;
-                if (tid == 0) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
-            }
             // ---- every warp combines the 16 summaries (lane w <-> slab w)
             uint32_t count = 0, warp_base = 0, cnt_l = 0;
             bool overflow = false;
@@ -692,6 +685,25 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 overflow = __any_sync(kFullMask, (sc_raw >> 31) != 0u);
                 const uint32_t cnt_incl = warp_incl_scan(cnt_l, lane);
                 warp_base = __shfl_sync(kFullMask, cnt_incl - cnt_l, warp);      // kept entries in the slabs before mine
+            }
+            // The stage is free: start the copy of the next tile (reserved one iteration ago) and reserve
+            // the one after -- unless the arena or the pending list will soon be full.  A block that
+            // drains must not sit on a reserved tile: nobody else can publish it, so the others'
+            // drains would queue up behind this one, one after the other.  Hence a block that expects
+            // to drain stops reserving, finishes what it holds, drains while it holds nothing, and only
+            // then takes its next ticket.
+            const uint32_t worst_now = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
+            const uint32_t g_next = s.next_tile[par];
+            const bool more = g_next < a.G;                  // (false for kNoTicket too)
+            if (more) {
+                issue_tile(s, a, st, g_next, tid);
+                pending |= 1u << st;
+                if (tid == 0) {
+                    // (tiles too dense for the arena drain at once whatever is done: keep their copies overlapped)
+                    const bool stop_reserving = !overflow && worst_now <= kArenaWords / 4u &&
+                        (npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords);
+                    ticket_ahead = stop_reserving ? kNoTicket : atomicAdd(&a.ctl->ticket, 1u);
+                }
             }
 
             uint32_t words = 0, M = 0, aoff = 0;
@@ -785,8 +797,25 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
             }
-            g = g_next;
-            have = refill;
+            if (g_next == kNoTicket) {
+                // nothing reserved: drain now, then take the next ticket and start its copy
+                __syncthreads();
+                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                npend = 0; arena_used = 0;
+                if (tid == 0) s.next_tile[par] = atomicAdd(&a.ctl->ticket, 1u);
+                __syncthreads();
+                g = s.next_tile[par];
+                have = g < a.G;
+                if (have) {
+                    issue_tile(s, a, st, g, tid);
+                    pending |= 1u << st;
+                    if (tid == 0) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
+                }
+                __syncthreads();                   // next_tile[par] is rewritten two iterations from now at the earliest
+            } else {
+                g = g_next;
+                have = more;
+            }
         }
         if (tid == 0) btrace[4] = read_globaltimer();
         if (!aborted) {
