@@ -192,10 +192,10 @@ def main():
     torch.cuda.synchronize()
 
     def compress_all():
-        for w in range(W):
-            rc = binding.compress(grads[w], pg, outs[w])
-            if rc:
-                raise binding.FastSGDError(rc, "fastsgd_compress")
+        # all workers' gradients in one launch (per 8 gradients); same streams as one call per gradient
+        rc = binding.compress_batch(grads, pg, outs)
+        if rc:
+            raise binding.FastSGDError(rc, "fastsgd_compress_batch")
 
     def decompress_all():
         # all workers' streams in one launch (per 8 streams); same result as one call per stream
@@ -299,7 +299,7 @@ def main():
 
     per_launch_bytes = {
         "k_abs_sum": 4.0 * n + 8.0 * ((n + 16383) // 16384),
-        "k_compress": 8.0 * n + float(sum(stream_bytes)) / W,
+        "k_compress": (8.0 * n * W + float(sum(stream_bytes))) / max(1, (W + 7) // 8),
         "k_decode_accumulate": (float(sum(stream_bytes)) + 8.0 * float(sum(kept))) / max(1, (W + 7) // 8),
     }
     kernels = {}

@@ -107,6 +107,20 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
                      void* out, uint64_t out_bytes, void* stream);
 
 /*
+ * The same encoder for the gradients of several workers (Sec. 2.1: W workers
+ * each hold a gradient of the same model), all of length n and compressed with
+ * the same parameters, each into its own stream.
+ *   grads   host array of num_grads device pointers (each 16-byte aligned)
+ *   outs    host array of num_grads device pointers (each 16-byte aligned),
+ *           every one with room for out_bytes bytes
+ * Every stream is byte for byte what fastsgd_compress produces for that
+ * gradient.  Up to 8 gradients share one kernel launch: thread blocks that are
+ * done with one gradient start on the next while the others finish.
+ */
+int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_params* params,
+                           void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream);
+
+/*
  * Decoder and aggregation (Sec. 3.1 decoder phases 1-4; Sec. 2.1 aggregation).
  *   stream_in  device, 16-byte aligned, a stream made by fastsgd_compress
  *   bytes      number of valid bytes at stream_in (>= header.total_bytes)

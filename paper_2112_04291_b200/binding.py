@@ -23,7 +23,7 @@ ST_BAD_MAGIC, ST_BAD_VERSION, ST_BAD_STATUS, ST_N_MISMATCH, ST_PARAM_MISMATCH = 
 ST_TRUNCATED, ST_BAD_DIRECTORY, ST_BAD_KEY, ST_BAD_CODE = 21, 22, 23, 24
 
 EXPORTS = [
-    "fastsgd_compress", "fastsgd_decompress_accumulate", "fastsgd_decompress_accumulate_batch", "fastsgd_compress_bound",
+    "fastsgd_compress", "fastsgd_compress_batch", "fastsgd_decompress_accumulate", "fastsgd_decompress_accumulate_batch", "fastsgd_compress_bound",
     "fastsgd_workspace_bytes", "fastsgd_set_workspace", "fastsgd_stream_info",
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
@@ -64,6 +64,8 @@ def lib():
         L.fastsgd_compress.argtypes = [vp, u64, PP, vp, u64, vp]
         L.fastsgd_decompress_accumulate.restype = C.c_int
         L.fastsgd_decompress_accumulate.argtypes = [vp, u64, u64, PP, vp, vp]
+        L.fastsgd_compress_batch.restype = C.c_int
+        L.fastsgd_compress_batch.argtypes = [C.POINTER(vp), u64, PP, C.POINTER(vp), u64, C.c_uint32, vp]
         L.fastsgd_decompress_accumulate_batch.restype = C.c_int
         L.fastsgd_decompress_accumulate_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, vp]
         L.fastsgd_compress_bound.restype = u64
@@ -149,6 +151,19 @@ def compress(grad: torch.Tensor, p: Params, out: torch.Tensor, stream=None) -> i
     assert out.is_cuda and out.dtype == torch.uint8 and out.is_contiguous()
     return lib().fastsgd_compress(grad.data_ptr(), grad.numel(), C.byref(p), out.data_ptr(), out.numel(),
                                   _stream_handle(stream))
+
+
+def compress_batch(grads, p: Params, outs, stream=None) -> int:
+    """fastsgd_compress_batch: several workers' gradients (same length) in one launch per 8."""
+    k = len(grads)
+    assert k == len(outs) and k > 0
+    n = grads[0].numel()
+    assert all(g.is_cuda and g.dtype == torch.float32 and g.is_contiguous() and g.numel() == n for g in grads)
+    cap = outs[0].numel()
+    assert all(o.is_cuda and o.dtype == torch.uint8 and o.is_contiguous() and o.numel() == cap for o in outs)
+    gp = (C.c_void_p * k)(*[int(g.data_ptr()) for g in grads])
+    op = (C.c_void_p * k)(*[int(o.data_ptr()) for o in outs])
+    return lib().fastsgd_compress_batch(gp, n, C.byref(p), op, cap, k, _stream_handle(stream))
 
 
 def decompress_accumulate(stream_in: torch.Tensor, nbytes: int, n: int, p: Params, dense: torch.Tensor,

@@ -83,7 +83,8 @@ uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
 }
 
 uint64_t ws_dense_offset(uint64_t n, uint32_t group_log2) {
-    const uint64_t b = kPartialsOffset + 8ull * chunks_of(n) + 8ull * groups_of(n, group_log2);
+    // partials and descriptors for every gradient one launch can take
+    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 8ull * groups_of(n, group_log2));
     return (b + 255ull) & ~255ull;
 }
 
@@ -97,7 +98,7 @@ WorkspaceView view(void* ws, uint64_t n) {
     v.ctl = reinterpret_cast<Control*>(base);
     v.thr = reinterpret_cast<float*>(base + kThrOffset);
     v.partials = reinterpret_cast<double*>(base + kPartialsOffset);
-    v.desc = reinterpret_cast<unsigned long long*>(base + kPartialsOffset + 8ull * chunks_of(n));
+    v.desc = reinterpret_cast<unsigned long long*>(base + kPartialsOffset + (uint64_t)kCmpMaxJobs * 8ull * chunks_of(n));
     return v;
 }
 
@@ -241,10 +242,13 @@ int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream
     return launch_sum(grad, n, 0u, 0u, pw, view(g_state.ws, n), sum_out, static_cast<cudaStream_t>(stream));
 }
 
-int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
-                     void* out, uint64_t out_bytes, void* stream) {
-    if (!grad || !out || !params) return FASTSGD_E_NULL;
-    if (!aligned(grad, 16) || !aligned(out, 16)) return FASTSGD_E_ALIGN;
+int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_params* params,
+                           void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream) {
+    if (!grads || !outs || !params) return FASTSGD_E_NULL;
+    for (uint32_t i = 0; i < num_grads; ++i) {
+        if (!grads[i] || !outs[i]) return FASTSGD_E_NULL;
+        if (!aligned(grads[i], 16) || !aligned(outs[i], 16)) return FASTSGD_E_ALIGN;
+    }
     PowTable pw;
     int rc = check_params(params, &pw);
     if (rc) return rc;
@@ -252,14 +256,13 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     if (rc) return rc;
     const uint64_t G = groups_of(n, params->group_log2);
     if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
-    if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;   // look-back fields are 31 bits
+    if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;   // descriptor fields are 31 bits
     std::lock_guard<std::mutex> lock(g_state.mu);
     if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     WorkspaceView w = view(g_state.ws, n);
-
     if (g_state.cmp_blocks_per_sm < 1) return FASTSGD_E_CUDA;
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
     if (grid > kMaxCtas) grid = kMaxCtas;
@@ -268,22 +271,36 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
         const uint64_t rounds = (G + grid - 1) / grid;
         grid = (G + rounds - 1) / rounds;
     }
-    CmpArgs ca;
-    ca.grad = grad; ca.n = n; ca.out = static_cast<uint8_t*>(out); ca.out_bytes = out_bytes;
-    ca.ctl = w.ctl; ca.partials = w.partials; ca.desc = w.desc;
-    ca.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
-    ca.base = params->base;
-    ca.G = (uint32_t)G; ca.tau = params->tau; ca.l = params->flag_bits;
-    void* kargs[] = {&ca, &pw};
-    cudaError_t err;
-    {
-        LaunchTimer lt(1, st);
-        err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)grid), dim3(kCmpThreads), kargs,
-                                          sizeof(CmpSmem), st);
+    for (uint32_t first = 0; first < num_grads; first += kCmpMaxJobs) {
+        CmpBatch cb;
+        std::memset(&cb, 0, sizeof(cb));
+        cb.jobs = num_grads - first < (uint32_t)kCmpMaxJobs ? num_grads - first : (uint32_t)kCmpMaxJobs;
+        for (uint32_t i = 0; i < cb.jobs; ++i) {
+            cb.grad[i] = grads[first + i];
+            cb.out[i] = static_cast<uint8_t*>(outs[first + i]);
+        }
+        cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc;
+        cb.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
+        cb.base = params->base; cb.G = (uint32_t)G; cb.tau = params->tau; cb.l = params->flag_bits;
+        void* kargs[] = {&cb, &pw};
+        cudaError_t err;
+        {
+            LaunchTimer lt(1, st);
+            err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)grid), dim3(kCmpThreads), kargs,
+                                              sizeof(CmpSmem), st);
+        }
+        if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
+        g_launches.fetch_add(1, std::memory_order_relaxed);
     }
-    if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
-    g_launches.fetch_add(1, std::memory_order_relaxed);
     return FASTSGD_OK;
+}
+
+int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
+                     void* out, uint64_t out_bytes, void* stream) {
+    if (!grad || !out) return FASTSGD_E_NULL;
+    const float* g1[1] = {grad};
+    void* o1[1] = {out};
+    return fastsgd_compress_batch(g1, n, params, o1, out_bytes, 1u, stream);
 }
 
 int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uint64_t* bytes,

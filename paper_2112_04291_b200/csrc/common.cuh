@@ -39,7 +39,8 @@ struct Control {
     unsigned int       bar_gen;        // bumped by the last block to arrive (sense of the barrier)
     unsigned long long trace[8];       // %globaltimer of block 0 at its phase boundaries (profiling aid)
     unsigned int       dq[6];          // decoder work queue: pushed, taken, done, exited, reserved (zero between launches)
-    unsigned int       pad[32];
+    unsigned int       tickets[8];     // encode pass: next tile of each gradient of the launch
+    unsigned int       pad[24];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 

@@ -79,12 +79,16 @@ struct CmpSmem {
 };
 static_assert(sizeof(CmpSmem) <= 232448, "shared memory of one block on sm_100");
 
+constexpr int kCmpMaxJobs = 8;             // gradients (simulated workers) one launch can take
+
+// One gradient's view of the launch arguments.
 struct CmpArgs {
     const float*        grad;
     uint64_t            n;
     uint8_t*            out;
     uint64_t            out_bytes;
     Control*            ctl;
+    unsigned int*       ticket;          // this gradient's tile counter of the encode pass
     double*             partials;
     unsigned long long* desc;
     unsigned char*      dense_scratch;
@@ -93,6 +97,35 @@ struct CmpArgs {
     uint32_t            tau;
     uint32_t            l;
 };
+
+// The launch arguments: up to kCmpMaxJobs gradients of the same length and parameters, compressed
+// one after the other by the same resident grid (a block that is done with one gradient's encode
+// pass starts summing the next while the others finish).
+struct CmpBatch {
+    const float*        grad[kCmpMaxJobs];
+    uint8_t*            out[kCmpMaxJobs];
+    uint64_t            out_bytes;
+    uint64_t            n;
+    Control*            ctl;
+    double*             partials;        // [jobs][G]
+    unsigned long long* desc;            // [jobs][G]
+    unsigned char*      dense_scratch;
+    double              base;
+    uint32_t            jobs;
+    uint32_t            G;
+    uint32_t            tau;
+    uint32_t            l;
+};
+
+__device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
+    CmpArgs a;
+    a.grad = b.grad[w]; a.n = b.n; a.out = b.out[w]; a.out_bytes = b.out_bytes; a.ctl = b.ctl;
+    a.ticket = b.ctl->tickets + w;
+    a.partials = b.partials + (uint64_t)w * b.G;
+    a.desc = b.desc + (uint64_t)w * b.G;
+    a.dense_scratch = b.dense_scratch; a.base = b.base; a.G = b.G; a.tau = b.tau; a.l = b.l;
+    return a;
+}
 
 // ---- mbarrier / bulk-copy primitives (sm_90+ PTX) -------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -454,21 +487,19 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, S
 }
 
 __global__ void __launch_bounds__(kCmpThreads, 2)
-k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
+k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
     CmpSmem& s = *reinterpret_cast<CmpSmem*>(cmp_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t c = blockIdx.x, grid = gridDim.x;
-    const uint32_t k = c < a.G ? (a.G - c + grid - 1) / grid : 0u;      // tiles of this block: c + i * grid
+    const uint32_t k = c < b.G ? (b.G - c + grid - 1) / grid : 0u;      // tiles of this block in a sum pass: c + i * grid
     const bool tracer = (c == 0 && tid == 0);
-    if (tracer) a.ctl->trace[0] = read_globaltimer();
-    unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(a.ctl) + kTraceOffset) + 8u * c;
+    unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kTraceOffset) + 8u * c;
     unsigned long long t_wait = 0ull, t_pack = 0ull;
-    if (tid == 0) btrace[0] = read_globaltimer();
 
     unsigned int my_gen = 0u;
     if (tid == 0) {
-        my_gen = ld_acquire_u32(&a.ctl->bar_gen);      // before this block can arrive at the barrier
+        my_gen = ld_acquire_u32(&b.ctl->bar_gen);      // before this block can arrive at the barrier
         for (int st = 0; st < kStages; ++st) mbar_init(&s.mbar[st], 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s.abort_flag = 0u;
@@ -476,6 +507,22 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
     __syncthreads();
     uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects
     uint32_t pending = 0;                     // bit st: a copy into stage st has been started and not waited for
+    bool aborted = false;
+    uint32_t held_now = 0xFFFFFFFFu, held_next = 0xFFFFFFFFu;     // thread 0: tiles taken and not yet published
+    // the pending tiles of the gradient before the one at hand: drained after the next sum pass, when
+    // (almost) every block has published its last tiles of that gradient
+    bool prev_valid = false;
+    int prev_npend = 0;
+    ScanState prev_sc; prev_sc.pos = 0u; prev_sc.count = 0u; prev_sc.words = 0u;
+    double prev_S = 0.0;
+    uint32_t prev_skip = 0u;
+    CmpArgs a = job_view(b, 0u);
+
+    for (uint32_t job = 0; job < b.jobs && !aborted; ++job) {
+    a = job_view(b, job);
+    held_now = 0xFFFFFFFFu; held_next = 0xFFFFFFFFu;
+    if (tracer) a.ctl->trace[0] = read_globaltimer();
+    if (tid == 0) btrace[0] = read_globaltimer();
 
     // =============================== phase 1: partial sums ===============================
     // load sequence q = 0..k-1 visits the tiles from the block's last to its first
@@ -487,7 +534,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         const int st = (int)(q % kStages);
         const uint32_t tile = c + (k - 1 - q) * grid;
         if (tid == 0) a.desc[tile] = 0ull;    // descriptors of phase 2 (ordered by the grid barrier)
-        if (tid == 0 && c == 0 && q == 0) a.ctl->ticket = grid;       // tiles below `grid` are taken: see phase 2
+        if (tid == 0 && c == 0 && q == 0) *a.ticket = grid;       // tiles below `grid` are taken: see phase 2
         if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
         parity ^= 1u << st;
         pending &= ~(1u << st);
@@ -513,6 +560,14 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
     if (tracer) a.ctl->trace[1] = read_globaltimer();
     if (tid == 0) btrace[1] = read_globaltimer();
 
+    // the previous gradient's last pending tiles (their blobs still sit in the arena)
+    if (prev_valid && !s.abort_flag) {
+        const CmpArgs ap = job_view(b, job - 1u);
+        __syncthreads();
+        if (!drain(s, ap, prev_npend, prev_sc, prev_S, prev_skip, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
+        prev_valid = false;
+    }
+
     // =============================== grid barrier ===============================
     __threadfence();
     __syncthreads();
@@ -534,8 +589,8 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         __threadfence();
     }
     __syncthreads();
-    bool aborted = s.abort_flag != 0u;
-    uint32_t held_now = 0xFFFFFFFFu, held_next = 0xFFFFFFFFu;     // thread 0: tiles taken and not yet published
+    aborted = s.abort_flag != 0u;
+    if (tid == 0) ++my_gen;                   // the next barrier of this launch waits for the next generation
 
     if (!aborted) {
         if (tracer) a.ctl->trace[2] = read_globaltimer();
@@ -574,7 +629,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
         uint32_t g = c;
         bool have = k > 0;
         unsigned int ticket_ahead = 0u;
-        if (tid == 0 && have) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
+        if (tid == 0 && have) ticket_ahead = atomicAdd(a.ticket, 1u);
         for (uint32_t i = 0; have && !aborted; ++i) {
             const int st = 0;
             const uint32_t par = i & 1u;
@@ -702,7 +757,7 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                     // (tiles too dense for the arena drain at once whatever is done: keep their copies overlapped)
                     const bool stop_reserving = !overflow && worst_now <= kArenaWords / 4u &&
                         (npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords);
-                    ticket_ahead = stop_reserving ? kNoTicket : atomicAdd(&a.ctl->ticket, 1u);
+                    ticket_ahead = stop_reserving ? kNoTicket : atomicAdd(a.ticket, 1u);
                 }
             }
 
@@ -802,14 +857,14 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
                 __syncthreads();
                 if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
-                if (tid == 0) s.next_tile[par] = atomicAdd(&a.ctl->ticket, 1u);
+                if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
                 g = s.next_tile[par];
                 have = g < a.G;
                 if (have) {
                     issue_tile(s, a, st, g, tid);
                     pending |= 1u << st;
-                    if (tid == 0) ticket_ahead = atomicAdd(&a.ctl->ticket, 1u);
+                    if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
                 __syncthreads();                   // next_tile[par] is rewritten two iterations from now at the earliest
             } else {
@@ -818,13 +873,17 @@ k_compress(const CmpArgs a, const __grid_constant__ PowTable pw) {
             }
         }
         if (tid == 0) btrace[4] = read_globaltimer();
-        if (!aborted) {
-            __syncthreads();                       // pending list written by thread 0
-            if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) aborted = true;
-        }
-        if (tracer) a.ctl->trace[4] = read_globaltimer();
-        if (tid == 0) { btrace[5] = read_globaltimer(); btrace[6] = t_wait; btrace[7] = t_pack; }
+        // what is still pending is drained after the next gradient's sum pass (or below, after the last)
+        prev_valid = !aborted; prev_npend = npend; prev_sc = sc; prev_S = S; prev_skip = skip;
     }
+    }   // jobs
+
+    if (!aborted && prev_valid) {
+        __syncthreads();                           // pending list written by thread 0
+        if (!drain(s, a, prev_npend, prev_sc, prev_S, prev_skip, tid, lane, warp)) aborted = true;
+    }
+    if (tracer) a.ctl->trace[4] = read_globaltimer();
+    if (tid == 0) { btrace[5] = read_globaltimer(); btrace[6] = t_wait; btrace[7] = t_pack; }
 
     if (aborted) {
         // give up: record it, unblock the others, drain this block's copies, return.  The header

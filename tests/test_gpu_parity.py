@@ -297,3 +297,32 @@ def test_batched_decode_equals_one_call_per_stream(nstreams):
     for s, b in zip(streams, sizes):
         assert binding.decompress_accumulate(s, b, n, pg, seq) == 0
     assert np.array_equal(seq.cpu().numpy(), got)
+
+
+@pytest.mark.parametrize("ngrads", [2, 4, 9])
+def test_batched_compress_equals_one_call_per_gradient(ngrads):
+    # several workers' gradients in one launch: every stream byte-equal to the oracle's (hence to
+    # what one call per gradient gives), including a tile-ragged length and an all-zero gradient
+    import torch
+    import gpu_util as G
+    n = 7 * 16384 + 4097
+    grads = [workloads.student_t_layers(n, seed=w, blocks=6, lo=1e-3, hi=1e-1) for w in range(ngrads)]
+    grads[1] = np.zeros(n, np.float32)
+    base = workloads.base_for_keep(grads[0], n // 40)
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    dg = [G.to_dev(v) for v in grads]
+    bufs = [G.Guarded(cap, fill=0x5A) for _ in range(ngrads)]
+    assert binding.compress_batch(dg, pg, [b.view for b in bufs]) == 0
+    for w in range(ngrads):
+        total, d, status = binding.stream_info(bufs[w].view)
+        orc, ostream = oracle.compress(grads[w], po)
+        assert status == orc == 0 and total == ostream.size and bufs[w].intact()
+        assert np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream), f"gradient {w}"
+    # and a second launch right after reuses the workspace cleanly
+    assert binding.compress_batch(dg[::-1], pg, [b.view for b in bufs]) == 0
+    for w in range(ngrads):
+        total, d, status = binding.stream_info(bufs[w].view)
+        orc, ostream = oracle.compress(grads[ngrads - 1 - w], po)
+        assert status == 0 and np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream)
