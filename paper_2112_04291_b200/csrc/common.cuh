@@ -40,7 +40,8 @@ struct Control {
     unsigned long long trace[8];       // %globaltimer of block 0 at its phase boundaries (profiling aid)
     unsigned int       dq[6];          // decoder work queue: pushed, taken, done, exited, reserved (zero between launches)
     unsigned int       tickets[8];     // encode pass: next tile of each gradient of the launch
-    unsigned int       pad[24];
+    unsigned int       tickets1[8];    // sum pass: the same (zero between launches)
+    unsigned int       pad[16];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 

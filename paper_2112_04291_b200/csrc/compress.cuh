@@ -72,7 +72,7 @@ struct CmpSmem {
     uint32_t poison_seen;
     uint32_t pad;
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
-    uint32_t pad2[2];
+    uint32_t p1_next[2];                     // the same for the sum pass
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
     uint16_t wkeys[kCmpWarps][kSlabCap];     // per warp: kept keys (tile-local), in index order
@@ -446,21 +446,24 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, S
     // ---- copy-out, directory entries, header
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
     uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
-    for (int p = 0; p < npend; ++p) {
-        const uint32_t g = s.pend_g[p], cm = s.pend_cm[p], words = s.pend_words[p], aoff = s.pend_off[p];
-        const unsigned long long pre = s.pend_prefix[p];
+    // one warp per pending tile (a dense tile's blob, in global scratch, is copied by the whole block)
+    for (int p0 = 0; p0 < npend; p0 += kCmpWarps) {
+        const int p = p0 + warp;
+        const bool mine = p < npend;
+        const uint32_t g = mine ? s.pend_g[p] : 0u, cm = mine ? s.pend_cm[p] : 0u, words = mine ? s.pend_words[p] : 0u,
+                       aoff = mine ? s.pend_off[p] : 0u;
+        const unsigned long long pre = mine ? s.pend_prefix[p] : 0ull;
         const uint32_t off = fixed_words + (uint32_t)pre;
         const uint64_t end_bytes = ((uint64_t)off + words) << 2;
-        const uint32_t* blob = aoff == kDenseMark
-            ? reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes)
-            : s.arena + aoff;
-        if (end_bytes <= a.out_bytes)
-            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
-        if (tid == 0) {
+        if (mine && aoff != kDenseMark && end_bytes <= a.out_bytes) {
+            const uint32_t* blob = s.arena + aoff;
+            for (uint32_t i = lane; i < words; i += 32) outw[off + i] = bswap32(blob[i]);
+        }
+        if (mine && lane == 0) {
             outw[(kHeaderBytes >> 2) + 2 * g]     = cm;
             outw[(kHeaderBytes >> 2) + 2 * g + 1] = off;
         }
-        if (g == a.G - 1 && tid == 0) {
+        if (mine && g == a.G - 1 && lane == 0) {
             int status = kStOk;
             if (skip == 2u) status = kStNonfinite;
             else if (end_bytes > a.out_bytes) status = kStCapacity;
@@ -482,6 +485,16 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, S
             outw[15] = a.G;
         }
     }
+    // a dense tile is always the only pending one when it is drained
+    if (npend >= 1 && s.pend_off[npend - 1] == kDenseMark) {
+        const int p = npend - 1;
+        const uint32_t words = s.pend_words[p];
+        const uint32_t off = fixed_words + (uint32_t)s.pend_prefix[p];
+        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
+        const uint32_t* blob = reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
+        if (end_bytes <= a.out_bytes)
+            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
+    }
     __syncthreads();       // the arena and the pending list are free again
     return true;
 }
@@ -492,7 +505,6 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     CmpSmem& s = *reinterpret_cast<CmpSmem*>(cmp_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t c = blockIdx.x, grid = gridDim.x;
-    const uint32_t k = c < b.G ? (b.G - c + grid - 1) / grid : 0u;      // tiles of this block in a sum pass: c + i * grid
     const bool tracer = (c == 0 && tid == 0);
     unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kTraceOffset) + 8u * c;
     unsigned long long t_wait = 0ull, t_pack = 0ull;
@@ -525,36 +537,47 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     if (tid == 0) btrace[0] = read_globaltimer();
 
     // =============================== phase 1: partial sums ===============================
-    // load sequence q = 0..k-1 visits the tiles from the block's last to its first
-    for (uint32_t q = 0; q < min(k, (uint32_t)kStages); ++q) {
-        issue_tile(s, a, (int)(q % kStages), c + (k - 1 - q) * grid, tid);
-        pending |= 1u << (q % kStages);
-    }
-    for (uint32_t q = 0; q < k; ++q) {
-        const int st = (int)(q % kStages);
-        const uint32_t tile = c + (k - 1 - q) * grid;
-        if (tid == 0) a.desc[tile] = 0ull;    // descriptors of phase 2 (ordered by the grid barrier)
-        if (tid == 0 && c == 0 && q == 0) *a.ticket = grid;       // tiles below `grid` are taken: see phase 2
-        if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
-        parity ^= 1u << st;
-        pending &= ~(1u << st);
-        double x[8];
-        const float4* row = reinterpret_cast<const float4*>(&s.stage[st][warp * 1024]) + lane;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
-        const double u = warp_slab_tree(x, lane);
-        if (lane == 0) s.s_warp[q & 1][warp] = u;
-        __syncthreads();
-        if (s.abort_flag) break;
-        if (warp == 0) {
-            double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
-            t = warp_tree(t, kCmpWarps);
-            if (lane == 0) a.partials[tile] = t;
+    // Tiles grid..G-1 are handed out by a ticket counter (so that the blocks finish together); the
+    // block's own tile c comes last and stays in shared memory for phase 2.  Thread 0 holds the
+    // ticket of the tile after the one at hand, taken one iteration before it is used.
+    {
+        unsigned int tk = 0u;
+        if (tid == 0) {
+            tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+            s.p1_next[0] = grid + tk < a.G ? grid + tk : c;
+            if (c == 0) *a.ticket = grid;                 // phase 2: tiles below `grid` are taken
         }
-        // the last kStages tiles stay in shared memory for phase 2
-        if (q + kStages < k) {
-            issue_tile(s, a, st, c + (k - 1 - (q + kStages)) * grid, tid);
-            pending |= 1u << st;
+        __syncthreads();
+        uint32_t tile = s.p1_next[0];
+        issue_tile(s, a, 0, tile, tid);
+        pending |= 1u;
+        if (tid == 0 && tile != c) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+        for (uint32_t q = 0;; ++q) {
+            if (tid == 0) a.desc[tile] = 0ull;            // descriptors of phase 2 (ordered by the grid barrier)
+            if (!mbar_wait(&s.mbar[0], parity & 1u)) s.abort_flag = 1u;
+            parity ^= 1u;
+            pending &= ~1u;
+            double x[8];
+            const float4* row = reinterpret_cast<const float4*>(&s.stage[0][warp * 1024]) + lane;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
+            const double u = warp_slab_tree(x, lane);
+            if (lane == 0) s.s_warp[q & 1][warp] = u;
+            if (tid == 0)                                 // the tile after this one: a ticketed tile, then c, then none
+                s.p1_next[(q + 1) & 1] = tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c);
+            __syncthreads();
+            if (s.abort_flag) break;
+            if (warp == 0) {
+                double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
+                t = warp_tree(t, kCmpWarps);
+                if (lane == 0) a.partials[tile] = t;
+            }
+            const uint32_t nxt = s.p1_next[(q + 1) & 1];
+            if (nxt == kNoTicket) break;                  // tile c was the last: it stays in the stage
+            issue_tile(s, a, 0, nxt, tid);
+            pending |= 1u;
+            if (tid == 0 && nxt != c) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+            tile = nxt;
         }
     }
     if (tracer) a.ctl->trace[1] = read_globaltimer();
@@ -590,6 +613,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     }
     __syncthreads();
     aborted = s.abort_flag != 0u;
+    if (tid == 0 && c == 0) a.ctl->tickets1[job] = 0u;       // every block is past its sum pass: ready for the next launch
     if (tid == 0) ++my_gen;                   // the next barrier of this launch waits for the next generation
 
     if (!aborted) {
@@ -627,7 +651,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // holds the ticket of the tile after the one at hand, taken a whole iteration before it is used.
         static_assert(kStages == 1, "the encode pass keeps one tile in flight per block");
         uint32_t g = c;
-        bool have = k > 0;
+        bool have = true;
         unsigned int ticket_ahead = 0u;
         if (tid == 0 && have) ticket_ahead = atomicAdd(a.ticket, 1u);
         for (uint32_t i = 0; have && !aborted; ++i) {
@@ -887,19 +911,16 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
     if (aborted) {
         // give up: record it, unblock the others, drain this block's copies, return.  The header
-        // is written here by the owner of the last group so that the caller sees the status.
+        // is written here by block 0 so that the caller sees the status.
         __syncthreads();
         if (tid == 0) {
             atomicExch(&a.ctl->error, (unsigned)kStTimeout);
-            if (held_now == 0xFFFFFFFFu) {            // still in the sum pass: nobody waits for descriptors yet
-                for (uint32_t i = 0; i < k; ++i) st_relaxed_u64(a.desc + c + i * grid, desc_pack(kDescPoison, 0, 0));
-            } else {
-                if (held_now < a.G) st_relaxed_u64(a.desc + held_now, desc_pack(kDescPoison, 0, 0));
-                if (held_next < a.G) st_relaxed_u64(a.desc + held_next, desc_pack(kDescPoison, 0, 0));
-            }
+            // (in the sum pass nobody waits for descriptors yet)
+            if (held_now < a.G) st_relaxed_u64(a.desc + held_now, desc_pack(kDescPoison, 0, 0));
+            if (held_next < a.G) st_relaxed_u64(a.desc + held_next, desc_pack(kDescPoison, 0, 0));
             for (int st = 0; st < kStages; ++st)
                 if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
-            if (k > 0 && c + (k - 1) * grid == a.G - 1) {
+            if (c == 0) {
                 uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
                 outw[0] = kMagic; outw[1] = kVersion; outw[2] = (uint32_t)kStTimeout; outw[3] = a.tau;
                 outw[4] = (uint32_t)a.n; outw[5] = (uint32_t)(a.n >> 32);
