@@ -323,8 +323,13 @@ int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uin
     rc = ensure_device_setup();
     if (rc) return rc;
     const uint64_t G = groups_of(n, params->group_log2);
+    // a warp per group at least; for few groups a block per group (up to two per SM), since groups
+    // with many keys are decoded by whole blocks taken from a shared queue
     const int warps_per_block = kDecThreads / 32;
     uint64_t grid = (G + warps_per_block - 1) / warps_per_block;
+    const uint64_t want = 2ull * (uint64_t)g_state.sm_count;
+    const uint64_t per_group = G < want ? G : want;
+    if (grid < per_group) grid = per_group;
     const uint64_t cap = (uint64_t)g_state.sm_count * g_state.dec_blocks_per_sm;
     if (grid > cap) grid = cap;
     const uint64_t min_grid = (G + kDecListMax - 1) / kDecListMax;     // a block owns at most kDecListMax groups

@@ -83,7 +83,7 @@ struct DecShared {
     double             sum[kDecMaxStreams];
     uint32_t           total_words[kDecMaxStreams];
     uint32_t           ok[kDecMaxStreams];
-    uint32_t           scan[kDecWarps];
+    uint32_t           scan[2][kDecWarps];
     uint32_t           big[kDecListMax];
     unsigned long long first_bad;     // min over threads of (key index << 8 | status), block path
     uint32_t           big_count;
@@ -112,21 +112,21 @@ __device__ __forceinline__ uint32_t get_bits(const uint32_t* words, uint32_t nwo
     return (uint32_t)((both >> (64u - sh - nb)) & ((nb >= 32u) ? 0xFFFFFFFFull : ((1ull << nb) - 1ull)));
 }
 
-// exclusive scan of one value per thread over the warp (BLOCK = false) or the block; also returns the total
+// exclusive scan of one value per thread over the warp (BLOCK = false) or the block; also returns the
+// total.  `which` alternates between the two shared arrays so that one barrier per scan is enough.
 template <bool BLOCK>
-__device__ __forceinline__ uint32_t excl_scan(uint32_t v, uint32_t* total, DecShared& s, int lane, int warp) {
+__device__ __forceinline__ uint32_t excl_scan(uint32_t v, uint32_t* total, DecShared& s, int lane, int warp, int which) {
     const uint32_t incl = warp_incl_scan(v, lane);
     if (!BLOCK) {
         *total = __shfl_sync(kFullMask, incl, 31);
         return incl - v;
     }
-    __syncthreads();                       // s.scan may still be read from the previous scan
-    if (lane == 31) s.scan[warp] = incl;
+    if (lane == 31) s.scan[which][warp] = incl;
     __syncthreads();
     uint32_t before = 0, all = 0;
 #pragma unroll
     for (int w = 0; w < kDecWarps; ++w) {
-        const uint32_t t = s.scan[w];
+        const uint32_t t = s.scan[which][w];
         if (w < warp) before += t;
         all += t;
     }
@@ -167,7 +167,10 @@ __device__ __forceinline__ bool read_dir(const DecArgs& a, const uint32_t* sw, u
 }
 
 // One group of one stream, decoded by a warp (BLOCK = false, `t` = lane, `nthreads` = 32) or by the
-// block from `blob` (shared memory copy, or global memory for very large blobs).
+// block from `blob` (shared memory copy, or global memory for very large blobs).  A thread owns a
+// run of K consecutive keys; for K <= 8 (up to 2048 keys per block) everything it parses stays in
+// registers between the passes.  With `tile` the values go into the group's slice of dense_out held
+// in shared memory (block path), else straight into dense_out.
 template <bool BLOCK>
 __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* blob, uint32_t nwords,
                                              uint32_t g, uint32_t count, uint32_t M, const float* val, float* tile,
@@ -184,38 +187,72 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     // this thread's run of consecutive keys [jb, je)
     const uint32_t K = (count + nthreads - 1) / nthreads;
     const uint32_t jb = min(count, (uint32_t)t * K), je = min(count, jb + K);
+    const bool small = K <= 8u;                       // uniform over the group
+    uint32_t wv[8], dv[8];
 
     // phase 1: widths from the flags; their sum fixes the blob's length, which must be the directory's
     uint32_t wsum = 0;
-    for (uint32_t j = jb; j < je; ++j) {
-        const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-        wsum += ((f + 1u) * M + levels_m1) >> a.l;
+    if (small) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            wv[k] = 0u;
+            if (jb + k < je) {
+                const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * (jb + k), a.l);
+                wv[k] = ((f + 1u) * M + levels_m1) >> a.l;
+            }
+            wsum += wv[k];
+        }
+    } else {
+        for (uint32_t j = jb; j < je; ++j) {
+            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
+            wsum += ((f + 1u) * M + levels_m1) >> a.l;
+        }
     }
     uint32_t wtotal;
-    const uint32_t pos0 = delta_pos0 + excl_scan<BLOCK>(wsum, &wtotal, s, lane, warp);
+    const uint32_t pos0 = delta_pos0 + excl_scan<BLOCK>(wsum, &wtotal, s, lane, warp, 0);
     if ((((uint64_t)delta_pos0 + wtotal + 31ull) >> 5) != nwords) {
         if (lead) dec_fail(a, g, 0u, kStBadDirectory);
         return;
     }
 
-    // phase 2: sum of this thread's deltas, then the key before its first one
+    // phase 2: this thread's deltas and their sum, then the key before its first one
     uint32_t dsum = 0;
-    {
+    if (small) {
+        uint32_t pos = pos0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            dv[k] = get_bits(blob, nwords, pos, wv[k]);       // width 0 beyond the run: reads as 0
+            pos += wv[k];
+            dsum = min(dsum + dv[k], 1u << 21);                // saturates only when already invalid
+        }
+    } else {
         uint32_t pos = pos0;
         for (uint32_t j = jb; j < je; ++j) {
             const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
             const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            dsum = min(dsum + get_bits(blob, nwords, pos, w), 1u << 21);   // saturates only when already invalid
+            dsum = min(dsum + get_bits(blob, nwords, pos, w), 1u << 21);
             pos += w;
         }
     }
     uint32_t dtotal;
-    const uint32_t key0 = lo + excl_scan<BLOCK>(dsum, &dtotal, s, lane, warp);
+    const uint32_t key0 = lo + excl_scan<BLOCK>(dsum, &dtotal, s, lane, warp, 1);
 
     // validation of the whole group before anything is applied: first key index that repeats,
     // leaves the group, or carries a code beyond tau
     unsigned long long bad = ~0ull;
-    {
+    if (small) {
+        uint32_t key = key0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t j = jb + k;
+            if (j < je && bad == ~0ull) {
+                key += dv[k];
+                const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+                if ((j > 0 && dv[k] == 0u) || key >= hi) bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
+                else if ((code & 0x7Fu) + 1u > a.tau) bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode;
+            }
+        }
+    } else {
         uint32_t pos = pos0, key = key0;
         for (uint32_t j = jb; j < je; ++j) {
             const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
@@ -229,12 +266,14 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
         }
     }
     if (BLOCK) {
-        __syncthreads();
-        if (t == 0) s.first_bad = ~0ull;
-        __syncthreads();
-        if (bad != ~0ull) atomicMin(&s.first_bad, bad);
-        __syncthreads();
-        bad = s.first_bad;
+        if (__syncthreads_or(bad != ~0ull)) {             // one barrier when the group is sound
+            if (t == 0) s.first_bad = ~0ull;
+            __syncthreads();
+            if (bad != ~0ull) atomicMin(&s.first_bad, bad);
+            __syncthreads();
+            bad = s.first_bad;
+            __syncthreads();
+        }
     } else {
         const uint32_t blo = __reduce_min_sync(kFullMask, (uint32_t)(bad < 0xFFFFFFFFull ? bad : 0xFFFFFFFFull));
         bad = blo == 0xFFFFFFFFu ? ~0ull : (unsigned long long)blo;
@@ -245,8 +284,34 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     }
 
     // phases 3-4 and the aggregation
-    if (BLOCK && tile != nullptr) {
-        // into the group's slice of dense_out held in shared memory (the caller loads and stores it)
+    if (small) {
+        uint32_t key = key0;
+        uint32_t kk[8]; float vv[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t j = jb + k;
+            kk[k] = 0xFFFFFFFFu; vv[k] = 0.f;
+            if (j < je) {
+                key += dv[k];
+                const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+                const float mag = val[(code & 0x7Fu) + 1u];
+                kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
+            }
+        }
+        if (BLOCK && tile != nullptr) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = __fadd_rn(tile[kk[k] - lo], vv[k]);
+        } else {
+            float dd[8];                                       // distinct keys: all loads, then all stores
+#pragma unroll
+            for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = __fadd_rn(dd[k], vv[k]);
+        }
+        return;
+    }
+    {
         uint32_t pos = pos0, key = key0;
         for (uint32_t j = jb; j < je; ++j) {
             const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
@@ -255,32 +320,9 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
             pos += w;
             const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
             const float mag = val[(code & 0x7Fu) + 1u];
-            tile[key - lo] = __fadd_rn(tile[key - lo], (code & 0x80u) ? -mag : mag);
-        }
-        return;
-    }
-    // straight into dense_out, four keys at a time (distinct keys: no aliasing)
-    {
-        uint32_t pos = pos0, key = key0;
-        for (uint32_t j = jb; j < je; j += 4) {
-            uint32_t kk[4]; float vv[4], dd[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                kk[i] = 0xFFFFFFFFu; vv[i] = 0.f;
-                if (j + i < je) {
-                    const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * (j + i), a.l);
-                    const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-                    key += get_bits(blob, nwords, pos, w);
-                    pos += w;
-                    const uint32_t code = (blob[(j + i) >> 2] >> (8u * ((j + i) & 3u))) & 0xFFu;
-                    const float mag = val[(code & 0x7Fu) + 1u];
-                    kk[i] = key; vv[i] = (code & 0x80u) ? -mag : mag;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dd[i] = kk[i] != 0xFFFFFFFFu ? a.dense[kk[i]] : 0.f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) if (kk[i] != 0xFFFFFFFFu) a.dense[kk[i]] = __fadd_rn(dd[i], vv[i]);
+            const float add = (code & 0x80u) ? -mag : mag;
+            if (BLOCK && tile != nullptr) tile[key - lo] = __fadd_rn(tile[key - lo], add);
+            else a.dense[key] = __fadd_rn(a.dense[key], add);
         }
     }
 }
