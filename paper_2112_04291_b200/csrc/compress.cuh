@@ -72,6 +72,12 @@ struct CmpSmem {
     uint32_t poison_seen;
     uint32_t pad;
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
+    uint32_t held[2];                        // tiles this block has taken and not yet published (for the give-up path)
+    uint32_t sc_pos, sc_count, sc_words;     // running exclusive scan of the descriptors: [0, pos) included
+    uint32_t job_skip;                       // 0 encode, 1 sum == 0, 2 sum not finite (of the gradient whose tiles are pending)
+    double   job_sum;                        // its sum
+    int      prev_npend;                     // pending tiles carried over to after the next sum pass
+    uint32_t pad3;
     uint32_t p1_next[2];                     // the same for the sum pass
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
@@ -371,9 +377,11 @@ struct ScanState {
 // Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
 // group numbers ascend.  Returns false if a poisoned descriptor or a
 // timeout was met (the caller aborts).
-__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, ScanState& sc,
-                                      double S, uint32_t skip, int tid, int lane, int warp) {
+__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
     if (npend == 0) return true;
+    ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
+    const double S = s.job_sum;
+    const uint32_t skip = s.job_skip;
     const uint32_t g_last = s.pend_g[npend - 1];
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
@@ -442,6 +450,7 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, S
     // the scan ran past g_last by whole steps: pull it back to g_last + 1
     // (descriptors beyond g_last were read as zero, so only the position needs correcting)
     sc.pos = g_last + 1u;
+    if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after the barrier below)
 
     // ---- copy-out, directory entries, header
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
@@ -507,7 +516,6 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     const uint32_t c = blockIdx.x, grid = gridDim.x;
     const bool tracer = (c == 0 && tid == 0);
     unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kTraceOffset) + 8u * c;
-    unsigned long long t_wait = 0ull, t_pack = 0ull;
 
     unsigned int my_gen = 0u;
     if (tid == 0) {
@@ -520,19 +528,15 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects
     uint32_t pending = 0;                     // bit st: a copy into stage st has been started and not waited for
     bool aborted = false;
-    uint32_t held_now = 0xFFFFFFFFu, held_next = 0xFFFFFFFFu;     // thread 0: tiles taken and not yet published
-    // the pending tiles of the gradient before the one at hand: drained after the next sum pass, when
-    // (almost) every block has published its last tiles of that gradient
+    // the pending tiles of the gradient before the one at hand are drained after the next sum pass,
+    // when (almost) every block has published its last tiles of that gradient; their count, the scan
+    // state and that gradient's sum wait in shared memory
     bool prev_valid = false;
-    int prev_npend = 0;
-    ScanState prev_sc; prev_sc.pos = 0u; prev_sc.count = 0u; prev_sc.words = 0u;
-    double prev_S = 0.0;
-    uint32_t prev_skip = 0u;
     CmpArgs a = job_view(b, 0u);
+    if (tid == 0) { s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu; }
 
     for (uint32_t job = 0; job < b.jobs && !aborted; ++job) {
     a = job_view(b, job);
-    held_now = 0xFFFFFFFFu; held_next = 0xFFFFFFFFu;
     if (tracer) a.ctl->trace[0] = read_globaltimer();
     if (tid == 0) btrace[0] = read_globaltimer();
 
@@ -587,7 +591,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     if (prev_valid && !s.abort_flag) {
         const CmpArgs ap = job_view(b, job - 1u);
         __syncthreads();
-        if (!drain(s, ap, prev_npend, prev_sc, prev_S, prev_skip, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
+        if (!drain(s, ap, s.prev_npend, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
         prev_valid = false;
     }
 
@@ -631,6 +635,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             s.thr[tid] = finite ? fmaxf(__double2float_ru(Bk), __int_as_float(1)) : __int_as_float(0x7f800000);
         }
         if (c == 0 && tid == 0) a.ctl->sum = S;
+        if (tid == 0) { s.job_sum = S; s.job_skip = skip; s.sc_pos = 0u; s.sc_count = 0u; s.sc_words = 0u; s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu; }
         __syncthreads();
         const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
         if (tracer) a.ctl->trace[3] = read_globaltimer();
@@ -642,7 +647,6 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // filters it, compacts its kept entries into its own list, quantises them and forms their
         // deltas without talking to the other warps; two block barriers per non-empty tile exchange
         // the slab summaries (counts, boundary keys, largest delta -> M) and the payload bits.
-        ScanState sc; sc.pos = 0u; sc.count = 0u; sc.words = 0u;
         int npend = 0;
         uint32_t arena_used = 0;
         const uint32_t round_up = (1u << a.l) - 1u;
@@ -658,13 +662,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             const int st = 0;
             const uint32_t par = i & 1u;
             if (i >= (uint32_t)kStages) {
-                const unsigned long long tw0 = tid == 0 ? read_globaltimer() : 0ull;
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
-                if (tid == 0) t_wait += read_globaltimer() - tw0;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
             }
-            const unsigned long long tp0 = tid == 0 ? read_globaltimer() : 0ull;
             // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c.
             // A row (128 consecutive entries, one float4 per lane) is looked at entry by entry only
             // if some lane holds an entry that reaches the threshold.
@@ -743,7 +744,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     slab_last = wk[slab_count - 1];
                 }
             }
-            if (tid == 0) { s.next_tile[par] = ticket_ahead; held_now = g; held_next = ticket_ahead; }
+            if (tid == 0) { s.next_tile[par] = ticket_ahead; s.held[0] = g; s.held[1] = ticket_ahead; }
             if (lane == 0) {
                 s.sum_count[par][warp] = slab_count | (slab_count > kSlabCap ? 0x80000000u : 0u);
                 s.sum_first[par][warp] = slab_first;
@@ -787,11 +788,11 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
             uint32_t words = 0, M = 0, aoff = 0;
             if (count == 0u) {
-                if (npend == kPendMax) { if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
+                if (npend == kPendMax) { if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
             } else if (!overflow) {
                 const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
                 if (npend == kPendMax || arena_used + worst > kArenaWords) {
-                    if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                    if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
                     npend = 0; arena_used = 0;
                 }
                 aoff = arena_used;
@@ -856,14 +857,13 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 arena_used += words;
             } else {
                 // a slab is too dense for its list: block-wide path in global scratch, committed at once
-                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 aoff = kDenseMark;
                 pack_tile_dense(s, a, count, warp_base, m, a.grad + ((uint64_t)g << kGroupLog2), ex0, ex1, tot0, tot1,
                                 &words, &M, tid, lane, warp);      // (the stage is being refilled: values come from global memory)
             }
             if (tid == 0) {
-                t_pack += read_globaltimer() - tp0;
                 st_relaxed_u64(a.desc + g, desc_pack(kDescValid, count, words));
                 s.pend_g[npend] = g;
                 s.pend_cm[npend] = count ? (count | (M << 24)) : 0u;
@@ -873,13 +873,13 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             ++npend;
             if (aoff == kDenseMark) {
                 __syncthreads();
-                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
             }
             if (g_next == kNoTicket) {
                 // nothing reserved: drain now, then take the next ticket and start its copy
                 __syncthreads();
-                if (!drain(s, a, npend, sc, S, skip, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
@@ -898,16 +898,17 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         }
         if (tid == 0) btrace[4] = read_globaltimer();
         // what is still pending is drained after the next gradient's sum pass (or below, after the last)
-        prev_valid = !aborted; prev_npend = npend; prev_sc = sc; prev_S = S; prev_skip = skip;
+        prev_valid = !aborted;
+        if (tid == 0) s.prev_npend = npend;
     }
     }   // jobs
 
     if (!aborted && prev_valid) {
         __syncthreads();                           // pending list written by thread 0
-        if (!drain(s, a, prev_npend, prev_sc, prev_S, prev_skip, tid, lane, warp)) aborted = true;
+        if (!drain(s, a, s.prev_npend, tid, lane, warp)) aborted = true;
     }
     if (tracer) a.ctl->trace[4] = read_globaltimer();
-    if (tid == 0) { btrace[5] = read_globaltimer(); btrace[6] = t_wait; btrace[7] = t_pack; }
+    if (tid == 0) btrace[5] = read_globaltimer();
 
     if (aborted) {
         // give up: record it, unblock the others, drain this block's copies, return.  The header
@@ -916,8 +917,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) {
             atomicExch(&a.ctl->error, (unsigned)kStTimeout);
             // (in the sum pass nobody waits for descriptors yet)
-            if (held_now < a.G) st_relaxed_u64(a.desc + held_now, desc_pack(kDescPoison, 0, 0));
-            if (held_next < a.G) st_relaxed_u64(a.desc + held_next, desc_pack(kDescPoison, 0, 0));
+            if (s.held[0] < a.G) st_relaxed_u64(a.desc + s.held[0], desc_pack(kDescPoison, 0, 0));
+            if (s.held[1] < a.G) st_relaxed_u64(a.desc + s.held[1], desc_pack(kDescPoison, 0, 0));
             for (int st = 0; st < kStages; ++st)
                 if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
             if (c == 0) {
