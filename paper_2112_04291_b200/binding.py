@@ -271,11 +271,13 @@ def debug_trace():
 
 
 def debug_trace_blocks(blocks: int = 148):
-    """Per-block stamps of the last fastsgd_compress call, one row per block: start, end of the sum
-    pass, barrier passed, table ready, end of the encode loop, end; then the nanoseconds thread 0
-    spent waiting for tiles and packing in the encode pass.  Profiling aid; synchronises."""
+    """Per-block stamps (ns, %globaltimer) of the last compress launch, shape (blocks, 8, 8): for
+    each block and each gradient of the launch: start, end of the sum pass, previous gradient's
+    pending tiles placed, grid barrier passed, table ready, end of the encode loop; slot 6 of
+    gradient 0 holds the end of the launch's last drain.  Profiling aid; synchronises."""
     ws = _workspace_keepalive
     if ws is None:
         return None
     torch.cuda.synchronize()
-    return ws[1024:1024 + 64 * blocks].cpu().numpy().view("<u8").reshape(blocks, 8).astype("int64")
+    off = 32768 + (4 << 17)
+    return ws[off:off + 512 * blocks].cpu().numpy().view("<u8").reshape(blocks, 8, 8).astype("int64")

@@ -41,7 +41,8 @@ struct Control {
     unsigned int       dq[6];          // decoder work queue: pushed, taken, done, exited, reserved (zero between launches)
     unsigned int       tickets[8];     // encode pass: next tile of each gradient of the launch
     unsigned int       tickets1[8];    // sum pass: the same (zero between launches)
-    unsigned int       pad[16];
+    unsigned int       enc_done[8];    // encode pass: blocks that have published all their tiles of each gradient (self-resetting)
+    unsigned int       pad[8];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -49,13 +50,16 @@ constexpr uint64_t kThrOffset      = 256;    // float thr[132]: RU32(B_k)
 constexpr uint64_t kTraceOffset    = 1024;   // u64 trace[<=496][8]: per-block %globaltimer stamps (profiling aid)
 constexpr uint64_t kQueueOffset    = 32768;  // u32 queue[2^17]: decoder's grid-wide queue of groups (zero between launches)
 constexpr uint64_t kQueueBytes     = 4ull << 17;
-constexpr uint64_t kPartialsOffset = kQueueOffset + kQueueBytes;  // double partial[chunks], then u64 desc[G]
+constexpr uint64_t kJobTraceOffset = kQueueOffset + kQueueBytes;  // u64 [320 blocks][8 gradients][8]: k_compress stamps (profiling aid)
+constexpr uint64_t kJobTraceBytes  = 320ull * 8ull * 8ull * 8ull;
+constexpr uint64_t kPartialsOffset = kJobTraceOffset + kJobTraceBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]
 
 struct WorkspaceView {
     Control*            ctl;
     float*              thr;
     double*             partials;
     unsigned long long* desc;
+    unsigned long long* prefix;
 };
 
 __host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }

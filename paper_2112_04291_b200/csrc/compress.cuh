@@ -77,7 +77,7 @@ struct CmpSmem {
     uint32_t job_skip;                       // 0 encode, 1 sum == 0, 2 sum not finite (of the gradient whose tiles are pending)
     double   job_sum;                        // its sum
     int      prev_npend;                     // pending tiles carried over to after the next sum pass
-    uint32_t pad3;
+    uint32_t publisher;                      // this block was the last to finish the gradient's encode pass
     uint32_t p1_next[2];                     // the same for the sum pass
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
@@ -97,6 +97,8 @@ struct CmpArgs {
     unsigned int*       ticket;          // this gradient's tile counter of the encode pass
     double*             partials;
     unsigned long long* desc;
+    unsigned long long* prefix;          // exclusive scan of desc, written by the last block to finish the encode pass
+    unsigned int*       enc_done;        // blocks that have finished this gradient's encode pass
     unsigned char*      dense_scratch;
     double              base;
     uint32_t            G;
@@ -115,6 +117,7 @@ struct CmpBatch {
     Control*            ctl;
     double*             partials;        // [jobs][G]
     unsigned long long* desc;            // [jobs][G]
+    unsigned long long* prefix;          // [jobs][G]
     unsigned char*      dense_scratch;
     double              base;
     uint32_t            jobs;
@@ -129,6 +132,8 @@ __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
     a.ticket = b.ctl->tickets + w;
     a.partials = b.partials + (uint64_t)w * b.G;
     a.desc = b.desc + (uint64_t)w * b.G;
+    a.prefix = b.prefix + (uint64_t)w * b.G;
+    a.enc_done = b.ctl->enc_done + w;
     a.dense_scratch = b.dense_scratch; a.base = b.base; a.G = b.G; a.tau = b.tau; a.l = b.l;
     return a;
 }
@@ -374,14 +379,72 @@ struct ScanState {
     uint32_t words;        // blob words of groups [0, pos)
 };
 
+// Copies the pending tiles' blobs to their places in the stream (pend_prefix holds each tile's
+// exclusive prefix), writes their directory entries and, for the last group, the header.
+__device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
+    const double S = s.job_sum;
+    const uint32_t skip = s.job_skip;
+    // ---- copy-out, directory entries, header
+    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
+    uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
+    // one warp per pending tile (a dense tile's blob, in global scratch, is copied by the whole block)
+    for (int p0 = 0; p0 < npend; p0 += kCmpWarps) {
+        const int p = p0 + warp;
+        const bool mine = p < npend;
+        const uint32_t g = mine ? s.pend_g[p] : 0u, cm = mine ? s.pend_cm[p] : 0u, words = mine ? s.pend_words[p] : 0u,
+                       aoff = mine ? s.pend_off[p] : 0u;
+        const unsigned long long pre = mine ? s.pend_prefix[p] : 0ull;
+        const uint32_t off = fixed_words + (uint32_t)pre;
+        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
+        if (mine && aoff != kDenseMark && end_bytes <= a.out_bytes) {
+            const uint32_t* blob = s.arena + aoff;
+            for (uint32_t i = lane; i < words; i += 32) outw[off + i] = bswap32(blob[i]);
+        }
+        if (mine && lane == 0) {
+            outw[(kHeaderBytes >> 2) + 2 * g]     = cm;
+            outw[(kHeaderBytes >> 2) + 2 * g + 1] = off;
+        }
+        if (mine && g == a.G - 1 && lane == 0) {
+            int status = kStOk;
+            if (skip == 2u) status = kStNonfinite;
+            else if (end_bytes > a.out_bytes) status = kStCapacity;
+            const uint64_t d_total = status == kStOk ? (pre >> 32) + (cm & 0xFFFFFFu) : 0ull;
+            const uint64_t total = status == kStOk ? end_bytes : (uint64_t)kHeaderBytes;
+            const double Sh = status == kStNonfinite ? 0.0 : S;
+            outw[0] = kMagic;
+            outw[1] = kVersion;
+            outw[2] = (uint32_t)status;
+            outw[3] = a.tau;
+            outw[4] = (uint32_t)a.n;            outw[5] = (uint32_t)(a.n >> 32);
+            outw[6] = (uint32_t)d_total;        outw[7] = (uint32_t)(d_total >> 32);
+            outw[8] = (uint32_t)total;          outw[9] = (uint32_t)(total >> 32);
+            const unsigned long long sb = (unsigned long long)__double_as_longlong(Sh);
+            const unsigned long long bb = (unsigned long long)__double_as_longlong(a.base);
+            outw[10] = (uint32_t)sb;            outw[11] = (uint32_t)(sb >> 32);
+            outw[12] = (uint32_t)bb;            outw[13] = (uint32_t)(bb >> 32);
+            outw[14] = a.l | ((uint32_t)kGroupLog2 << 8);
+            outw[15] = a.G;
+        }
+    }
+    // a dense tile is always the only pending one when it is drained
+    if (npend >= 1 && s.pend_off[npend - 1] == kDenseMark) {
+        const int p = npend - 1;
+        const uint32_t words = s.pend_words[p];
+        const uint32_t off = fixed_words + (uint32_t)s.pend_prefix[p];
+        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
+        const uint32_t* blob = reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
+        if (end_bytes <= a.out_bytes)
+            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
+    }
+    __syncthreads();       // the arena and the pending list are free again
+}
+
 // Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
 // group numbers ascend.  Returns false if a poisoned descriptor or a
 // timeout was met (the caller aborts).
 __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
     if (npend == 0) return true;
     ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
-    const double S = s.job_sum;
-    const uint32_t skip = s.job_skip;
     const uint32_t g_last = s.pend_g[npend - 1];
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
@@ -452,60 +515,81 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, i
     sc.pos = g_last + 1u;
     if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after the barrier below)
 
-    // ---- copy-out, directory entries, header
-    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
-    uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
-    // one warp per pending tile (a dense tile's blob, in global scratch, is copied by the whole block)
-    for (int p0 = 0; p0 < npend; p0 += kCmpWarps) {
-        const int p = p0 + warp;
-        const bool mine = p < npend;
-        const uint32_t g = mine ? s.pend_g[p] : 0u, cm = mine ? s.pend_cm[p] : 0u, words = mine ? s.pend_words[p] : 0u,
-                       aoff = mine ? s.pend_off[p] : 0u;
-        const unsigned long long pre = mine ? s.pend_prefix[p] : 0ull;
-        const uint32_t off = fixed_words + (uint32_t)pre;
-        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
-        if (mine && aoff != kDenseMark && end_bytes <= a.out_bytes) {
-            const uint32_t* blob = s.arena + aoff;
-            for (uint32_t i = lane; i < words; i += 32) outw[off + i] = bswap32(blob[i]);
-        }
-        if (mine && lane == 0) {
-            outw[(kHeaderBytes >> 2) + 2 * g]     = cm;
-            outw[(kHeaderBytes >> 2) + 2 * g + 1] = off;
-        }
-        if (mine && g == a.G - 1 && lane == 0) {
-            int status = kStOk;
-            if (skip == 2u) status = kStNonfinite;
-            else if (end_bytes > a.out_bytes) status = kStCapacity;
-            const uint64_t d_total = status == kStOk ? (pre >> 32) + (cm & 0xFFFFFFu) : 0ull;
-            const uint64_t total = status == kStOk ? end_bytes : (uint64_t)kHeaderBytes;
-            const double Sh = status == kStNonfinite ? 0.0 : S;
-            outw[0] = kMagic;
-            outw[1] = kVersion;
-            outw[2] = (uint32_t)status;
-            outw[3] = a.tau;
-            outw[4] = (uint32_t)a.n;            outw[5] = (uint32_t)(a.n >> 32);
-            outw[6] = (uint32_t)d_total;        outw[7] = (uint32_t)(d_total >> 32);
-            outw[8] = (uint32_t)total;          outw[9] = (uint32_t)(total >> 32);
-            const unsigned long long sb = (unsigned long long)__double_as_longlong(Sh);
-            const unsigned long long bb = (unsigned long long)__double_as_longlong(a.base);
-            outw[10] = (uint32_t)sb;            outw[11] = (uint32_t)(sb >> 32);
-            outw[12] = (uint32_t)bb;            outw[13] = (uint32_t)(bb >> 32);
-            outw[14] = a.l | ((uint32_t)kGroupLog2 << 8);
-            outw[15] = a.G;
-        }
-    }
-    // a dense tile is always the only pending one when it is drained
-    if (npend >= 1 && s.pend_off[npend - 1] == kDenseMark) {
-        const int p = npend - 1;
-        const uint32_t words = s.pend_words[p];
-        const uint32_t off = fixed_words + (uint32_t)s.pend_prefix[p];
-        const uint64_t end_bytes = ((uint64_t)off + words) << 2;
-        const uint32_t* blob = reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
-        if (end_bytes <= a.out_bytes)
-            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
-    }
-    __syncthreads();       // the arena and the pending list are free again
+    place_pending(s, a, npend, tid, lane, warp);
     return true;
+}
+
+// The same once a gradient's encode pass is over: the last block to finish it has written the
+// exclusive scan of all descriptors (publish_prefixes); every block fetches the entries of its
+// pending tiles (bounded polls) and places them.
+__device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
+    if (npend == 0) return true;
+    if (tid == 0) s.poison_seen = 0u;
+    __syncthreads();
+    if (tid < npend) {
+        const unsigned long long* p = a.prefix + s.pend_g[tid];
+        unsigned long long v = ld_relaxed_u64(p);
+        uint32_t spin = 0;
+        while ((v >> 62) == kDescInvalid) {
+            if (++spin > kWaitLimit) { s.poison_seen = 2u; break; }
+            __nanosleep(64);
+            v = ld_relaxed_u64(p);
+        }
+        if ((v >> 62) == kDescPoison) s.poison_seen = 1u;
+        s.pend_prefix[tid] = ((unsigned long long)desc_count(v) << 32) | desc_words(v);
+    }
+    __syncthreads();
+    if (s.poison_seen) return false;       // (rewritten only at the start of the next drain, behind a barrier)
+    place_pending(s, a, npend, tid, lane, warp);
+    return true;
+}
+
+// Run by the last block to finish a gradient's encode pass (every descriptor is published by then):
+// exclusive scan of all descriptors into a.prefix, kDrainChunks x 512 at a time.  A descriptor that
+// is not valid poisons its own and every later prefix.
+__device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, int tid, int lane, int warp) {
+    unsigned long long running = 0ull;
+    bool bad = false;
+    for (uint32_t pos = 0; pos < a.G; pos += (uint32_t)kDrainChunks * kCmpThreads) {
+        unsigned long long own[kDrainChunks], excl[kDrainChunks];
+        bool bad_here = false;
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+            own[j] = idx < a.G ? ld_relaxed_u64(a.desc + idx) : desc_pack(kDescValid, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            if ((own[j] >> 62) != kDescValid) { bad_here = true; own[j] = 0ull; }
+            own[j] = ((unsigned long long)desc_count(own[j]) << 32) | desc_words(own[j]);
+            unsigned long long incl = own[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(kFullMask, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) s.scan64[j][warp] = incl;
+            excl[j] = incl - own[j];
+        }
+        if (__syncthreads_or(bad_here ? 1 : 0)) bad = true;
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            unsigned long long before = running, all = 0ull;
+#pragma unroll
+            for (int w = 0; w < kCmpWarps; ++w) {
+                const unsigned long long t = s.scan64[j][w];
+                if (w < warp) before += t;
+                all += t;
+            }
+            excl[j] += before;
+            running += all;
+            const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+            if (idx < a.G)
+                st_relaxed_u64(a.prefix + idx, bad ? desc_pack(kDescPoison, 0, 0)
+                                                   : desc_pack(kDescValid, (uint32_t)(excl[j] >> 32), (uint32_t)excl[j]));
+        }
+        __syncthreads();
+    }
 }
 
 __global__ void __launch_bounds__(kCmpThreads, 2)
@@ -515,7 +599,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t c = blockIdx.x, grid = gridDim.x;
     const bool tracer = (c == 0 && tid == 0);
-    unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kTraceOffset) + 8u * c;
+    unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kJobTraceOffset) + 64u * c;
 
     unsigned int my_gen = 0u;
     if (tid == 0) {
@@ -538,7 +622,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     for (uint32_t job = 0; job < b.jobs && !aborted; ++job) {
     a = job_view(b, job);
     if (tracer) a.ctl->trace[0] = read_globaltimer();
-    if (tid == 0) btrace[0] = read_globaltimer();
+    if (tid == 0) btrace[8u * job + 0] = read_globaltimer();
 
     // =============================== phase 1: partial sums ===============================
     // Tiles grid..G-1 are handed out by a ticket counter (so that the blocks finish together); the
@@ -557,7 +641,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         pending |= 1u;
         if (tid == 0 && tile != c) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
         for (uint32_t q = 0;; ++q) {
-            if (tid == 0) a.desc[tile] = 0ull;            // descriptors of phase 2 (ordered by the grid barrier)
+            if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }   // phase 2's descriptors and prefixes (ordered by the grid barrier)
             if (!mbar_wait(&s.mbar[0], parity & 1u)) s.abort_flag = 1u;
             parity ^= 1u;
             pending &= ~1u;
@@ -585,28 +669,37 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         }
     }
     if (tracer) a.ctl->trace[1] = read_globaltimer();
-    if (tid == 0) btrace[1] = read_globaltimer();
+    if (tid == 0) btrace[8u * job + 1] = read_globaltimer();
 
-    // the previous gradient's last pending tiles (their blobs still sit in the arena)
-    if (prev_valid && !s.abort_flag) {
-        const CmpArgs ap = job_view(b, job - 1u);
-        __syncthreads();
-        if (!drain(s, ap, s.prev_npend, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
-        prev_valid = false;
-    }
-
-    // =============================== grid barrier ===============================
+    // =============================== grid barrier, first half: arrive ===============================
+    // Sense-reversing barrier: the last block to arrive clears the count and bumps the generation
+    // every block read when it started (no state outside the workspace, so a launch can be replayed).
+    // Between arriving and waiting the block places the previous gradient's last pending tiles.
     __threadfence();
     __syncthreads();
+    bool last_arrival = false;
     if (tid == 0 && !s.abort_flag) {
-        // sense-reversing barrier: the last block to arrive clears the count and bumps the generation
-        // every block read when it started (no state outside the workspace, so a launch can be replayed)
         const unsigned int old = atomicAdd(&a.ctl->bar_count, 1u);
         if (old == grid - 1u) {
             a.ctl->bar_count = 0u;
             __threadfence();
             atomicAdd(&a.ctl->bar_gen, 1u);
-        } else {
+            last_arrival = true;
+        }
+    }
+
+    // the previous gradient's last pending tiles (their blobs still sit in the arena)
+    if (prev_valid && !s.abort_flag) {
+        const CmpArgs ap = job_view(b, job - 1u);
+        __syncthreads();
+        if (!drain_final(s, ap, s.prev_npend, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
+        prev_valid = false;
+    }
+    if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
+
+    // =============================== grid barrier, second half: wait ===============================
+    if (tid == 0 && !s.abort_flag) {
+        if (!last_arrival) {
             uint32_t spin = 0;
             while (ld_acquire_u32(&a.ctl->bar_gen) == my_gen) {
                 if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
@@ -622,7 +715,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
     if (!aborted) {
         if (tracer) a.ctl->trace[2] = read_globaltimer();
-        if (tid == 0) btrace[2] = read_globaltimer();
+        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
 
         // =============================== sum, boundary table ===============================
         const double S = reduce_partials(a.partials, a.G, s.s_tree, reinterpret_cast<double*>(s.arena), tid, lane, warp);
@@ -639,7 +732,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         __syncthreads();
         const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
         if (tracer) a.ctl->trace[3] = read_globaltimer();
-        if (tid == 0) btrace[3] = read_globaltimer();
+        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
 
         // =============================== phase 2: encode ===============================
         // Tile i of this block sits in stage (k-1-(i%kStages))%kStages; the last ones of phase 1 are
@@ -896,23 +989,34 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 have = more;
             }
         }
-        if (tid == 0) btrace[4] = read_globaltimer();
-        // what is still pending is drained after the next gradient's sum pass (or below, after the last)
+        if (tid == 0) btrace[8u * job + 5] = read_globaltimer();
+        // what is still pending is placed after the next gradient's sum pass (or below, after the last),
+        // with the prefixes that the last block to get here computes for everybody
         prev_valid = !aborted;
-        if (tid == 0) s.prev_npend = npend;
+        if (tid == 0) {
+            s.prev_npend = npend;
+            s.publisher = 0u;
+            if (!aborted) {
+                __threadfence();                            // this block's descriptors before its count
+                const unsigned int old = atomicAdd(a.enc_done, 1u);
+                if (old == grid - 1u) { *a.enc_done = 0u; s.publisher = 1u; __threadfence(); }
+            }
+        }
+        __syncthreads();
+        if (s.publisher) publish_prefixes(s, a, tid, lane, warp);
     }
     }   // jobs
 
     if (!aborted && prev_valid) {
         __syncthreads();                           // pending list written by thread 0
-        if (!drain(s, a, s.prev_npend, tid, lane, warp)) aborted = true;
+        if (!drain_final(s, a, s.prev_npend, tid, lane, warp)) aborted = true;
     }
     if (tracer) a.ctl->trace[4] = read_globaltimer();
-    if (tid == 0) btrace[5] = read_globaltimer();
+    if (tid == 0) btrace[6] = read_globaltimer();   // (slot 6 of the first gradient: end of the launch's last drain)
 
     if (aborted) {
-        // give up: record it, unblock the others, drain this block's copies, return.  The header
-        // is written here by block 0 so that the caller sees the status.
+        // give up: record it, unblock the others, wait for this block's copies, mark every stream of
+        // the launch as timed out, return.
         __syncthreads();
         if (tid == 0) {
             atomicExch(&a.ctl->error, (unsigned)kStTimeout);
@@ -921,8 +1025,9 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             if (s.held[1] < a.G) st_relaxed_u64(a.desc + s.held[1], desc_pack(kDescPoison, 0, 0));
             for (int st = 0; st < kStages; ++st)
                 if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
-            if (c == 0) {
-                uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
+            // every stream of the launch reports the timeout (identical words from every block that gives up)
+            for (uint32_t w = 0; w < b.jobs; ++w) {
+                uint32_t* outw = reinterpret_cast<uint32_t*>(b.out[w]);
                 outw[0] = kMagic; outw[1] = kVersion; outw[2] = (uint32_t)kStTimeout; outw[3] = a.tau;
                 outw[4] = (uint32_t)a.n; outw[5] = (uint32_t)(a.n >> 32);
                 outw[6] = 0u; outw[7] = 0u; outw[8] = kHeaderBytes; outw[9] = 0u;
