@@ -259,15 +259,14 @@ def kernel_timing_read():
 
 
 def debug_trace():
-    """Block 0's %globaltimer stamps (ns) of the last fastsgd_compress call: start, end of the
-    sum pass, grid barrier passed, boundary table ready, end of the encode pass.  Profiling aid
-    read straight from the registered workspace tensor; synchronises."""
-    ws = _workspace_keepalive
-    if ws is None:
+    """Block 0's %globaltimer stamps (ns) for the first gradient of the last compress launch: start,
+    end of the sum pass, grid barrier passed, boundary table ready, end of the encode pass.
+    Profiling aid read straight from the registered workspace tensor; synchronises."""
+    t = debug_trace_blocks(1)
+    if t is None:
         return None
-    torch.cuda.synchronize()
-    raw = ws[40:40 + 64].cpu().numpy().view("<u8")
-    return [int(x) for x in raw]
+    r = t[0, 0]
+    return [int(r[0]), int(r[1]), int(r[3]), int(r[4]), int(r[5])]
 
 
 def debug_trace_blocks(blocks: int = 148):

@@ -267,11 +267,8 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
     if (g_state.cmp_blocks_per_sm < 1) return FASTSGD_E_CUDA;
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
     if (grid > kMaxCtas) grid = kMaxCtas;
+    const uint64_t grid_full = grid;
     if (grid > G) grid = G;
-    {   // equal shares: every block gets the same number of tiles in the sum pass (+-0 when G divides)
-        const uint64_t rounds = (G + grid - 1) / grid;
-        grid = (G + rounds - 1) / rounds;
-    }
     for (uint32_t first = 0; first < num_grads; first += kCmpMaxJobs) {
         CmpBatch cb;
         std::memset(&cb, 0, sizeof(cb));
@@ -281,13 +278,27 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
             cb.out[i] = static_cast<uint8_t*>(outs[first + i]);
         }
         cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc; cb.prefix = w.prefix;
+        cb.sm_slots = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kSmSlotOffset);
         cb.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
         cb.base = params->base; cb.G = (uint32_t)G; cb.tau = params->tau; cb.l = params->flag_bits;
+        // Two or more gradients, two resident blocks per SM and enough tiles: the two blocks of an SM
+        // form two teams that work on different gradients.  One gradient: the tiles below the grid
+        // size are assigned statically, so every block gets an equal share.
+        uint64_t launch_grid = grid;
+        cb.teams = 1u;
+        if (cb.jobs >= 2u && g_state.cmp_blocks_per_sm >= 2 && grid_full == 2ull * (uint64_t)g_state.sm_count &&
+            g_state.sm_count <= 256 && G >= grid_full) {
+            cb.teams = 2u;
+            launch_grid = grid_full;
+        } else if (cb.jobs == 1u) {
+            const uint64_t rounds = (G + grid - 1) / grid;
+            launch_grid = (G + rounds - 1) / rounds;
+        }
         void* kargs[] = {&cb, &pw};
         cudaError_t err;
         {
             LaunchTimer lt(1, st);
-            err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)grid), dim3(kCmpThreads), kargs,
+            err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
                                               sizeof(CmpSmem), st);
         }
         if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }

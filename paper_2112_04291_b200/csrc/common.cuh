@@ -35,13 +35,14 @@ struct Control {
     unsigned int       skip;           // 0 encode normally, 1 sum == 0, 2 sum not finite
     unsigned long long decode_status;  // min over failures of (group << 32 | key index << 8 | status)
     double             sum;            // S
-    unsigned int       bar_count;      // blocks that have reached the grid barrier of the running call
-    unsigned int       bar_gen;        // bumped by the last block to arrive (sense of the barrier)
-    unsigned long long trace[8];       // %globaltimer of block 0 at its phase boundaries (profiling aid)
+    unsigned int       bar_gen;        // launches of k_compress that have finished
+    unsigned int       exit_count;     // blocks of the running k_compress launch that have finished (self-resetting)
     unsigned int       dq[6];          // decoder work queue: pushed, taken, done, exited, reserved (zero between launches)
     unsigned int       tickets[8];     // encode pass: next tile of each gradient of the launch
     unsigned int       tickets1[8];    // sum pass: the same (zero between launches)
     unsigned int       enc_done[8];    // encode pass: blocks that have published all their tiles of each gradient (self-resetting)
+    unsigned int       bar_count[8];   // blocks that have finished each gradient's sum pass (self-resetting)
+    unsigned int       bar_flag[8];    // set to bar_gen + 1 by the last of them: that gradient's partial sums are complete
     unsigned int       pad[8];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
@@ -52,7 +53,9 @@ constexpr uint64_t kQueueOffset    = 32768;  // u32 queue[2^17]: decoder's grid-
 constexpr uint64_t kQueueBytes     = 4ull << 17;
 constexpr uint64_t kJobTraceOffset = kQueueOffset + kQueueBytes;  // u64 [320 blocks][8 gradients][8]: k_compress stamps (profiling aid)
 constexpr uint64_t kJobTraceBytes  = 320ull * 8ull * 8ull * 8ull;
-constexpr uint64_t kPartialsOffset = kJobTraceOffset + kJobTraceBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]
+constexpr uint64_t kSmSlotOffset   = kJobTraceOffset + kJobTraceBytes;  // u32 [256]: blocks of the running launch seen on each SM (zero between launches)
+constexpr uint64_t kSmSlotBytes    = 1024;
+constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]
 
 struct WorkspaceView {
     Control*            ctl;

@@ -74,10 +74,13 @@ struct CmpSmem {
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
     uint32_t held[2];                        // tiles this block has taken and not yet published (for the give-up path)
     uint32_t sc_pos, sc_count, sc_words;     // running exclusive scan of the descriptors: [0, pos) included
-    uint32_t job_skip;                       // 0 encode, 1 sum == 0, 2 sum not finite (of the gradient whose tiles are pending)
-    double   job_sum;                        // its sum
+    uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
+    double   job_sum[2];                     // by gradient parity: its sum
+    double   s_nodes[256];                   // nodes of the final sum tree when a thread holds more than 8 partials
     int      prev_npend;                     // pending tiles carried over to after the next sum pass
     uint32_t publisher;                      // this block was the last to finish the gradient's encode pass
+    uint32_t team;                           // 0: sums the next gradient before it encodes this one; 1: after
+    uint32_t pad4;
     uint32_t p1_next[2];                     // the same for the sum pass
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
@@ -118,12 +121,15 @@ struct CmpBatch {
     double*             partials;        // [jobs][G]
     unsigned long long* desc;            // [jobs][G]
     unsigned long long* prefix;          // [jobs][G]
+    unsigned int*       sm_slots;        // [256] blocks of this launch per SM
     unsigned char*      dense_scratch;
     double              base;
     uint32_t            jobs;
     uint32_t            G;
     uint32_t            tau;
     uint32_t            l;
+    uint32_t            teams;           // 1, or 2: the two blocks of every SM work on different gradients
+    uint32_t            pad;
 };
 
 __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
@@ -176,6 +182,9 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 }
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned int v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
     unsigned int v;
@@ -381,9 +390,9 @@ struct ScanState {
 
 // Copies the pending tiles' blobs to their places in the stream (pend_prefix holds each tile's
 // exclusive prefix), writes their directory entries and, for the last group, the header.
-__device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
-    const double S = s.job_sum;
-    const uint32_t skip = s.job_skip;
+__device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
+    const double S = s.job_sum[jp];
+    const uint32_t skip = s.job_skip[jp];
     // ---- copy-out, directory entries, header
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
     uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
@@ -442,7 +451,7 @@ __device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, int 
 // Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
 // group numbers ascend.  Returns false if a poisoned descriptor or a
 // timeout was met (the caller aborts).
-__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
+__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
     if (npend == 0) return true;
     ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
     const uint32_t g_last = s.pend_g[npend - 1];
@@ -515,14 +524,14 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, int npend, i
     sc.pos = g_last + 1u;
     if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after the barrier below)
 
-    place_pending(s, a, npend, tid, lane, warp);
+    place_pending(s, a, jp, npend, tid, lane, warp);
     return true;
 }
 
 // The same once a gradient's encode pass is over: the last block to finish it has written the
 // exclusive scan of all descriptors (publish_prefixes); every block fetches the entries of its
 // pending tiles (bounded polls) and places them.
-__device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, int npend, int tid, int lane, int warp) {
+__device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
     if (npend == 0) return true;
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
@@ -540,7 +549,7 @@ __device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, int np
     }
     __syncthreads();
     if (s.poison_seen) return false;       // (rewritten only at the start of the next drain, behind a barrier)
-    place_pending(s, a, npend, tid, lane, warp);
+    place_pending(s, a, jp, npend, tid, lane, warp);
     return true;
 }
 
@@ -592,147 +601,228 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
     }
 }
 
+// Phase 1 for one gradient: fp64 partial sum of every 2^14-entry tile.  Tiles grid..G-1 are handed
+// out by a ticket counter (so that the blocks finish together); the block's own tile c comes last
+// (and stays in the stage afterwards).  Thread 0 holds the ticket of the tile after the one at
+// hand, taken one iteration before it is used.  sum_begin starts the copy of the first tile and
+// returns; sum_rest does the rest (the caller has something else to do while that copy flies).
+struct SumCursor {
+    unsigned int tk;       // thread 0: the look-ahead ticket
+    uint32_t     tile;     // the tile whose copy is in flight
+};
+
+__device__ __forceinline__ SumCursor sum_begin(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t c, uint32_t grid,
+                                               uint32_t& pending, int tid) {
+    SumCursor cur; cur.tk = 0u;
+    if (tid == 0) {
+        cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+        s.p1_next[0] = full ? (cur.tk < a.G ? cur.tk : kNoTicket) : (grid + cur.tk < a.G ? grid + cur.tk : c);
+    }
+    __syncthreads();
+    cur.tile = s.p1_next[0];
+    if (cur.tile != kNoTicket) {
+        issue_tile(s, a, 0, cur.tile, tid);
+        pending |= 1u;
+        if (tid == 0 && (full || cur.tile != c)) cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+    }
+    return cur;
+}
+
+__device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t c, uint32_t grid,
+                                         SumCursor cur, uint32_t& parity, uint32_t& pending, int tid, int lane, int warp) {
+    unsigned int tk = cur.tk;
+    uint32_t tile = cur.tile;
+    if (tile == kNoTicket) return;                    // (several gradients, fewer tiles than blocks)
+    for (uint32_t q = 0;; ++q) {
+        if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }   // phase 2's descriptors and prefixes (ordered by the grid barrier)
+        if (!mbar_wait(&s.mbar[0], parity & 1u)) s.abort_flag = 1u;
+        parity ^= 1u;
+        pending &= ~1u;
+        double x[8];
+        const float4* row = reinterpret_cast<const float4*>(&s.stage[0][warp * 1024]) + lane;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
+        const double u = warp_slab_tree(x, lane);
+        if (lane == 0) s.s_warp[q & 1][warp] = u;
+        if (tid == 0)                                 // the tile after this one: a ticketed tile, then (one gradient) c, then none
+            s.p1_next[(q + 1) & 1] = full ? (tk < a.G ? tk : kNoTicket)
+                                          : (tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c));
+        __syncthreads();
+        if (s.abort_flag) break;
+        if (warp == 0) {
+            double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
+            t = warp_tree(t, kCmpWarps);
+            if (lane == 0) a.partials[tile] = t;
+        }
+        const uint32_t nxt = s.p1_next[(q + 1) & 1];
+        if (nxt == kNoTicket) break;
+        issue_tile(s, a, 0, nxt, tid);
+        pending |= 1u;
+        if (tid == 0 && (full || nxt != c)) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+        tile = nxt;
+    }
+}
+
+// Grid barrier of gradient `job` among the `tgrid` blocks that work on it, first half: this
+// block's partial sums are written.  The last block to arrive clears the count, readies the
+// gradient's ticket counters (encode pass: with one gradient the tiles below `tgrid` are taken;
+// sum pass: zero for the next launch) and sets the gradient's flag to the launch's generation
+// (read by every block when it started, bumped by the last block to leave the kernel: no state
+// outside the workspace, so a launch can be replayed).
+__device__ __forceinline__ void barrier_arrive(CmpSmem& s, Control* ctl, uint32_t job, bool full, uint32_t tgrid,
+                                               unsigned int gen_next, int tid) {
+    if (tid == 0 && !s.abort_flag) {                  // (thread 0 wrote the partials and cleared the descriptors itself)
+        __threadfence();
+        const unsigned int old = atomicAdd(&ctl->bar_count[job], 1u);
+        if (old == tgrid - 1u) {
+            ctl->bar_count[job] = 0u;
+            ctl->tickets[job] = full ? 0u : tgrid;
+            ctl->tickets1[job] = 0u;
+            __threadfence();
+            st_release_u32(&ctl->bar_flag[job], gen_next);
+        }
+    }
+}
+
+// Second half: wait (bounded) until every block has arrived.
+__device__ __forceinline__ void barrier_wait(CmpSmem& s, Control* ctl, uint32_t job, unsigned int gen_next, int tid) {
+    if (tid == 0 && !s.abort_flag) {
+        uint32_t spin = 0;
+        while (ld_acquire_u32(&ctl->bar_flag[job]) != gen_next) {
+            if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
+            if (spin > 8u) __nanosleep(64);
+        }
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+// After the grid barrier of gradient `job`: every block reduces the partials itself (same tree),
+// S -> boundary table RU32(B_k) in shared memory; resets the block's per-gradient scan state.
+__device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const PowTable& pw, uint32_t jp,
+                                           int tid, int lane, int warp) {
+    const double S = reduce_partials(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
+    const bool finite = isfinite(S);
+    const uint32_t skip = !finite ? 2u : (S == 0.0 ? 1u : 0u);
+    if (tid <= (int)a.tau) {
+        // |v| >= B_k on an fp32 |v| equals |v| >= RU32(B_k); never below the smallest denormal,
+        // because an entry must also be non-zero to be kept
+        const double Bk = __ddiv_rn(S, pw.P[tid]);
+        s.thr[tid] = finite ? fmaxf(__double2float_ru(Bk), __int_as_float(1)) : __int_as_float(0x7f800000);
+    }
+    if (tid == 0) {
+        s.job_sum[jp] = S; s.job_skip[jp] = skip;
+        s.sc_pos = 0u; s.sc_count = 0u; s.sc_words = 0u;
+        s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
+    }
+    __syncthreads();
+}
+
+// Schedule of one launch.  With teams == 2 the two blocks of every SM belong to different teams;
+// team t compresses gradients t, t+2, ... by itself (own barriers, tickets and prefixes), so that
+// one team streams while the other sits in a control step.  A team's gradients j0 < j1 < ...:
+//   sum(j0) | sum(j1) with table(j0) inside, encode(j0) | sum(j2) with table(j1) inside, place(j0), encode(j1) | ... | place(last)
+// The sum pass of the next gradient runs before the encode pass of the one at hand: nobody waits at
+// its grid barrier, blocks that fall behind in one pass take fewer tickets in the next, and the
+// latencies of the control steps hide behind tile copies in flight.  place(j) puts the tiles of
+// gradient j that were still pending at the end of its encode pass.  With a single gradient the
+// block's last tile of the sum pass stays in shared memory for the encode pass.
 __global__ void __launch_bounds__(kCmpThreads, 2)
 k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
     CmpSmem& s = *reinterpret_cast<CmpSmem*>(cmp_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t c = blockIdx.x, grid = gridDim.x;
-    const bool tracer = (c == 0 && tid == 0);
+    const uint32_t c = blockIdx.x;
     unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kJobTraceOffset) + 64u * c;
 
-    unsigned int my_gen = 0u;
+    const bool full = b.jobs > 1u;            // several gradients: every tile of every pass is handed out by ticket
+    unsigned int gen_next = 0u;
     if (tid == 0) {
-        my_gen = ld_acquire_u32(&b.ctl->bar_gen);      // before this block can arrive at the barrier
+        gen_next = ld_acquire_u32(&b.ctl->bar_gen) + 1u;      // before this block can arrive at a barrier
         for (int st = 0; st < kStages; ++st) mbar_init(&s.mbar[st], 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s.abort_flag = 0u;
+        s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
+        uint32_t team = 0u;
+        if (b.teams == 2u) {                  // (the host launches exactly two blocks per SM then)
+            unsigned int smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            team = atomicAdd(b.sm_slots + (smid & 255u), 1u) & 1u;
+        }
+        s.team = team;
     }
     __syncthreads();
+    const uint32_t first_job = s.team, step = b.teams;
+    const uint32_t grid = gridDim.x / b.teams;              // blocks that work on a gradient
     uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects
     uint32_t pending = 0;                     // bit st: a copy into stage st has been started and not waited for
     bool aborted = false;
-    // the pending tiles of the gradient before the one at hand are drained after the next sum pass,
-    // when (almost) every block has published its last tiles of that gradient; their count, the scan
-    // state and that gradient's sum wait in shared memory
+    // the tiles of the gradient before the one at hand that were pending at the end of its encode
+    // pass: their count, that gradient's sum and status wait in shared memory
     bool prev_valid = false;
-    CmpArgs a = job_view(b, 0u);
-    if (tid == 0) { s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu; }
+    uint32_t prev_job = 0u;
+    CmpArgs a = job_view(b, first_job < b.jobs ? first_job : 0u);
 
-    for (uint32_t job = 0; job < b.jobs && !aborted; ++job) {
+    if (first_job < b.jobs) {
+        if (tid == 0) btrace[8u * first_job + 0] = read_globaltimer();
+        const SumCursor cur = sum_begin(s, a, first_job, full, c, grid, pending, tid);
+        sum_rest(s, a, first_job, full, c, grid, cur, parity, pending, tid, lane, warp);
+        if (tid == 0) btrace[8u * first_job + 1] = read_globaltimer();
+        barrier_arrive(s, b.ctl, first_job, full, grid, gen_next, tid);
+    }
+
+    uint32_t it = 0u;                         // gradients this block has started to encode
+    for (uint32_t job = first_job; job < b.jobs && !aborted; job += step, ++it) {
+    const uint32_t jp = it & 1u;
     a = job_view(b, job);
-    if (tracer) a.ctl->trace[0] = read_globaltimer();
-    if (tid == 0) btrace[8u * job + 0] = read_globaltimer();
-
-    // =============================== phase 1: partial sums ===============================
-    // Tiles grid..G-1 are handed out by a ticket counter (so that the blocks finish together); the
-    // block's own tile c comes last and stays in shared memory for phase 2.  Thread 0 holds the
-    // ticket of the tile after the one at hand, taken one iteration before it is used.
-    {
-        unsigned int tk = 0u;
-        if (tid == 0) {
-            tk = atomicAdd(a.ctl->tickets1 + job, 1u);
-            s.p1_next[0] = grid + tk < a.G ? grid + tk : c;
-            if (c == 0) *a.ticket = grid;                 // phase 2: tiles below `grid` are taken
-        }
-        __syncthreads();
-        uint32_t tile = s.p1_next[0];
-        issue_tile(s, a, 0, tile, tid);
-        pending |= 1u;
-        if (tid == 0 && tile != c) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
-        for (uint32_t q = 0;; ++q) {
-            if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }   // phase 2's descriptors and prefixes (ordered by the grid barrier)
-            if (!mbar_wait(&s.mbar[0], parity & 1u)) s.abort_flag = 1u;
-            parity ^= 1u;
-            pending &= ~1u;
-            double x[8];
-            const float4* row = reinterpret_cast<const float4*>(&s.stage[0][warp * 1024]) + lane;
-#pragma unroll
-            for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
-            const double u = warp_slab_tree(x, lane);
-            if (lane == 0) s.s_warp[q & 1][warp] = u;
-            if (tid == 0)                                 // the tile after this one: a ticketed tile, then c, then none
-                s.p1_next[(q + 1) & 1] = tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c);
-            __syncthreads();
-            if (s.abort_flag) break;
-            if (warp == 0) {
-                double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
-                t = warp_tree(t, kCmpWarps);
-                if (lane == 0) a.partials[tile] = t;
-            }
-            const uint32_t nxt = s.p1_next[(q + 1) & 1];
-            if (nxt == kNoTicket) break;                  // tile c was the last: it stays in the stage
-            issue_tile(s, a, 0, nxt, tid);
-            pending |= 1u;
-            if (tid == 0 && nxt != c) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
-            tile = nxt;
-        }
-    }
-    if (tracer) a.ctl->trace[1] = read_globaltimer();
-    if (tid == 0) btrace[8u * job + 1] = read_globaltimer();
-
-    // =============================== grid barrier, first half: arrive ===============================
-    // Sense-reversing barrier: the last block to arrive clears the count and bumps the generation
-    // every block read when it started (no state outside the workspace, so a launch can be replayed).
-    // Between arriving and waiting the block places the previous gradient's last pending tiles.
-    __threadfence();
     __syncthreads();
-    bool last_arrival = false;
-    if (tid == 0 && !s.abort_flag) {
-        const unsigned int old = atomicAdd(&a.ctl->bar_count, 1u);
-        if (old == grid - 1u) {
-            a.ctl->bar_count = 0u;
-            __threadfence();
-            atomicAdd(&a.ctl->bar_gen, 1u);
-            last_arrival = true;
-        }
-    }
-
-    // the previous gradient's last pending tiles (their blobs still sit in the arena)
-    if (prev_valid && !s.abort_flag) {
-        const CmpArgs ap = job_view(b, job - 1u);
-        __syncthreads();
-        if (!drain_final(s, ap, s.prev_npend, tid, lane, warp)) { if (tid == 0) s.abort_flag = 1u; }
-        prev_valid = false;
-    }
-    if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
-
-    // =============================== grid barrier, second half: wait ===============================
-    if (tid == 0 && !s.abort_flag) {
-        if (!last_arrival) {
-            uint32_t spin = 0;
-            while (ld_acquire_u32(&a.ctl->bar_gen) == my_gen) {
-                if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
-                __nanosleep(64);
-            }
-        }
-        __threadfence();
+    if (job + step < b.jobs && !s.abort_flag) {
+        // next gradient's sum pass; this gradient's table while the first copy is in flight
+        const uint32_t nj = job + step;
+        const CmpArgs an = job_view(b, nj);
+        if (tid == 0) btrace[8u * nj + 0] = read_globaltimer();
+        const SumCursor cur = sum_begin(s, an, nj, full, c, grid, pending, tid);
+        barrier_wait(s, b.ctl, job, gen_next, tid);
+        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
+        if (!s.abort_flag) make_table(s, a, pw, jp, tid, lane, warp);
+        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
+        sum_rest(s, an, nj, full, c, grid, cur, parity, pending, tid, lane, warp);
+        if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
+        barrier_arrive(s, b.ctl, nj, full, grid, gen_next, tid);
+    } else {
+        barrier_wait(s, b.ctl, job, gen_next, tid);
+        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
+        if (!s.abort_flag) make_table(s, a, pw, jp, tid, lane, warp);
+        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
     }
     __syncthreads();
     aborted = s.abort_flag != 0u;
-    if (tid == 0 && c == 0) a.ctl->tickets1[job] = 0u;       // every block is past its sum pass: ready for the next launch
-    if (tid == 0) ++my_gen;                   // the next barrier of this launch waits for the next generation
 
     if (!aborted) {
-        if (tracer) a.ctl->trace[2] = read_globaltimer();
-        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
-
-        // =============================== sum, boundary table ===============================
-        const double S = reduce_partials(a.partials, a.G, s.s_tree, reinterpret_cast<double*>(s.arena), tid, lane, warp);
-        const bool finite = isfinite(S);
-        const uint32_t skip = !finite ? 2u : (S == 0.0 ? 1u : 0u);
-        if (tid <= (int)a.tau) {
-            // |v| >= B_k on an fp32 |v| equals |v| >= RU32(B_k); never below the smallest denormal,
-            // because an entry must also be non-zero to be kept
-            const double Bk = __ddiv_rn(S, pw.P[tid]);
-            s.thr[tid] = finite ? fmaxf(__double2float_ru(Bk), __int_as_float(1)) : __int_as_float(0x7f800000);
+        // the block's first tile of the encode pass: with one gradient its own tile c, still there from
+        // the sum pass; otherwise the first ticket it gets
+        const bool preloaded = full;
+        uint32_t g = c;
+        bool have = true;
+        if (full) {
+            if (tid == 0) s.next_tile[1] = atomicAdd(a.ticket, 1u);
+            __syncthreads();
+            g = s.next_tile[1];
+            have = g < a.G;
+            if (have) {
+                issue_tile(s, a, 0, g, tid);
+                pending |= 1u;
+            }
         }
-        if (c == 0 && tid == 0) a.ctl->sum = S;
-        if (tid == 0) { s.job_sum = S; s.job_skip = skip; s.sc_pos = 0u; s.sc_count = 0u; s.sc_words = 0u; s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu; }
-        __syncthreads();
+        // the previous gradient's last pending tiles (their blobs still sit in the arena)
+        if (prev_valid) {
+            const CmpArgs ap = job_view(b, prev_job);
+            if (!drain_final(s, ap, jp ^ 1u, s.prev_npend, tid, lane, warp)) { aborted = true; break; }
+            prev_valid = false;
+        }
+        if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
+        const uint32_t skip = s.job_skip[jp];
         const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
-        if (tracer) a.ctl->trace[3] = read_globaltimer();
-        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
 
         // =============================== phase 2: encode ===============================
         // Tile i of this block sits in stage (k-1-(i%kStages))%kStages; the last ones of phase 1 are
@@ -747,14 +837,12 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // is handed out by a ticket counter, so that blocks that met dense tiles take fewer.  Thread 0
         // holds the ticket of the tile after the one at hand, taken a whole iteration before it is used.
         static_assert(kStages == 1, "the encode pass keeps one tile in flight per block");
-        uint32_t g = c;
-        bool have = true;
         unsigned int ticket_ahead = 0u;
         if (tid == 0 && have) ticket_ahead = atomicAdd(a.ticket, 1u);
         for (uint32_t i = 0; have && !aborted; ++i) {
             const int st = 0;
             const uint32_t par = i & 1u;
-            if (i >= (uint32_t)kStages) {
+            if (i > 0u || preloaded) {
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
@@ -881,11 +969,11 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
             uint32_t words = 0, M = 0, aoff = 0;
             if (count == 0u) {
-                if (npend == kPendMax) { if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
+                if (npend == kPendMax) { if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
             } else if (!overflow) {
                 const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
                 if (npend == kPendMax || arena_used + worst > kArenaWords) {
-                    if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
+                    if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
                     npend = 0; arena_used = 0;
                 }
                 aoff = arena_used;
@@ -950,7 +1038,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 arena_used += words;
             } else {
                 // a slab is too dense for its list: block-wide path in global scratch, committed at once
-                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 aoff = kDenseMark;
                 pack_tile_dense(s, a, count, warp_base, m, a.grad + ((uint64_t)g << kGroupLog2), ex0, ex1, tot0, tot1,
@@ -966,13 +1054,13 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             ++npend;
             if (aoff == kDenseMark) {
                 __syncthreads();
-                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
             }
             if (g_next == kNoTicket) {
                 // nothing reserved: drain now, then take the next ticket and start its copy
                 __syncthreads();
-                if (!drain(s, a, npend, tid, lane, warp)) { aborted = true; break; }
+                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
                 npend = 0; arena_used = 0;
                 if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
@@ -993,6 +1081,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // what is still pending is placed after the next gradient's sum pass (or below, after the last),
         // with the prefixes that the last block to get here computes for everybody
         prev_valid = !aborted;
+        prev_job = job;
         if (tid == 0) {
             s.prev_npend = npend;
             s.publisher = 0u;
@@ -1009,9 +1098,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
     if (!aborted && prev_valid) {
         __syncthreads();                           // pending list written by thread 0
-        if (!drain_final(s, a, s.prev_npend, tid, lane, warp)) aborted = true;
+        if (!drain_final(s, a, (it - 1u) & 1u, s.prev_npend, tid, lane, warp)) aborted = true;
     }
-    if (tracer) a.ctl->trace[4] = read_globaltimer();
     if (tid == 0) btrace[6] = read_globaltimer();   // (slot 6 of the first gradient: end of the launch's last drain)
 
     if (aborted) {
@@ -1039,6 +1127,18 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             }
         }
         __syncthreads();
+    }
+
+    // the last block to leave readies the workspace for the next launch
+    if (tid == 0) {
+        __threadfence();
+        const unsigned int old = atomicAdd(&b.ctl->exit_count, 1u);
+        if (old == gridDim.x - 1u) {
+            b.ctl->exit_count = 0u;
+            if (b.teams == 2u) for (int i = 0; i < 256; ++i) b.sm_slots[i] = 0u;
+            __threadfence();
+            st_release_u32(&b.ctl->bar_gen, gen_next);
+        }
     }
 }
 
