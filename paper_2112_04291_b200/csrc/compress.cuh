@@ -62,6 +62,7 @@ struct CmpSmem {
     uint32_t sum_maxd[2][kCmpWarps];         // largest delta between two kept keys of the slab
     uint32_t sum_bits[2][kCmpWarps];         // payload bits of the slab
     uint32_t scan_tot[kCmpWarps];
+    uint32_t scan_tot2[2][kCmpWarps];
     uint32_t pend_g[kPendMax];
     uint32_t pend_cm[kPendMax];              // count | M << 24
     uint32_t pend_words[kPendMax];
@@ -77,7 +78,7 @@ struct CmpSmem {
     uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
     double   job_sum[2];                     // by gradient parity: its sum
     double   s_nodes[256];                   // nodes of the final sum tree when a thread holds more than 8 partials
-    int      prev_npend;                     // pending tiles carried over to after the next sum pass
+    uint32_t pad5;
     uint32_t publisher;                      // this block was the last to finish the gradient's encode pass
     uint32_t team;                           // 0: sums the next gradient before it encodes this one; 1: after
     uint32_t pad4;
@@ -286,19 +287,23 @@ __device__ __forceinline__ uint32_t code_byte_of(const float* thr, uint32_t tau,
     return (val < 0.0f ? 0x80u : 0u) | (L - 1u);
 }
 
-// Phase 2 for a tile too dense for the per-warp lists: block-wide compaction, quantisation,
-// deltas, M, flags, width scan and packing in the block's slot of global scratch (the blob reuses
-// the values' words).  `m` is the kept mask of this thread's 32 entries, `tile` the tile's entries
-// (global memory: kept entries lie below n).
+// Phase 2 for a tile too dense for the per-warp lists.  The kept (key, value) pairs are compacted
+// in index order into the block's slot of global scratch (coalesced, L2-resident); the stage, whose
+// values are dead after that, then holds the blob (at most 16384 x 27 bits): code bytes by plain
+// byte stores, then flags and deltas 512 keys at a time (one block-wide scan of the widths per
+// chunk) with shared-memory ORs.  The caller places the blob from the stage before it refills it.
+// `m` is the kept mask of this thread's 32 entries.
+static_assert((uint64_t)kTile * (8u + 5u + (uint32_t)kGroupLog2) <= (uint64_t)kTile * 32u, "the widest blob fits the stage");
+
 __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, uint32_t count,
-                                             uint32_t warp_base, uint32_t m, const float* tile,
+                                             uint32_t warp_base, uint32_t m,
                                              uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
                                              uint32_t* words_out, uint32_t* M_out, int tid, int lane, int warp) {
     unsigned char* slot = a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
     uint32_t* vals = reinterpret_cast<uint32_t*>(slot);
     uint16_t* keys = reinterpret_cast<uint16_t*>(slot + (uint64_t)kTile * 4u);
-    uint8_t* codes = reinterpret_cast<uint8_t*>(slot + (uint64_t)kTile * 6u);
-    uint32_t* blob = vals;
+    const float* tile = s.stage[0];
+    uint32_t* blob = reinterpret_cast<uint32_t*>(s.stage[0]);
 
     // ---- stream compaction in index order: (key, value) of the kept entries
     if (m != 0u) {
@@ -320,64 +325,64 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
         }
     }
     if (tid == 0) s.max_delta = 0u;
+    __syncthreads();                          // the stage's values are dead from here on
+
+    // ---- zero the words the blob can reach
+    {
+        const uint32_t bound_words = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
+        for (uint32_t i = tid; i < bound_words; i += kCmpThreads) blob[i] = 0u;
+    }
     __syncthreads();
 
-    // ---- logarithm quantisation of the kept entries and delta keys (Eq. 4)
+    // ---- logarithm quantisation (code bytes straight to their place: byte j of the stream is the
+    //      byte 3 - j%4 of big-endian-valued word j/4) and the largest delta (Eq. 4)
     {
+        uint8_t* blob_bytes = reinterpret_cast<uint8_t*>(blob);
         uint32_t local_max = 0;
         for (uint32_t j = tid; j < count; j += kCmpThreads) {
             const uint32_t key = keys[j];
-            codes[j] = (uint8_t)code_byte_of(s.thr, a.tau, __uint_as_float(vals[j]));
-            const uint32_t delta = key - (j ? (uint32_t)keys[j - 1] : 0u);
-            local_max = max(local_max, delta);
+            const uint32_t prev = j ? (uint32_t)keys[j - 1] : 0u;      // (the first delta of a group counts from 0)
+            blob_bytes[(j & ~3u) | (3u - (j & 3u))] = (uint8_t)code_byte_of(s.thr, a.tau, __uint_as_float(vals[j]));
+            local_max = max(local_max, key - prev);
         }
         local_max = __reduce_max_sync(kFullMask, local_max);
         if (lane == 0 && local_max) atomicMax(&s.max_delta, local_max);
     }
     __syncthreads();
 
-    // ---- M, flags and widths; exclusive scan of the widths (a thread owns consecutive keys);
-    //      zero the words the blob can reach (they held the values, dead now)
+    // ---- M; flags and deltas, 512 consecutive keys per round
     const uint32_t maxd = s.max_delta;
     const uint32_t M = maxd ? (32u - __clz(maxd)) : 1u;
     const uint32_t inv_m = (65536u + M - 1u) / M;
     const uint32_t round_up = (1u << a.l) - 1u;
-    const uint32_t ipt = (count + kCmpThreads - 1) / kCmpThreads;
-    const uint32_t j_lo = min(count, tid * ipt), j_hi = min(count, j_lo + ipt);
-    uint32_t my_bits = 0;
-    for (uint32_t j = j_lo; j < j_hi; ++j) {
-        const uint32_t delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
-        my_bits += ((flag_of(delta, a.l, inv_m) + 1u) * M + round_up) >> a.l;
-    }
-    const uint32_t incl = warp_incl_scan(my_bits, lane);
-    if (lane == 31) s.scan_tot[warp] = incl;
-    {
-        const uint32_t bound_words = (count * (8u + a.l + M) + 31u) >> 5;
-        for (uint32_t i = tid; i < bound_words; i += kCmpThreads) blob[i] = 0u;
-    }
-    __syncthreads();
-    uint32_t before = 0, payload_bits = 0;
-#pragma unroll
-    for (int w = 0; w < kCmpWarps; ++w) {
-        const uint32_t t = s.scan_tot[w];
-        if (w < warp) before += t;
-        payload_bits += t;
-    }
     const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a.l * count;
-    {
-        uint32_t dpos = delta_pos0 + before + (incl - my_bits);
-        for (uint32_t j = j_lo; j < j_hi; ++j) {
-            const uint32_t delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
-            const uint32_t f = flag_of(delta, a.l, inv_m);
-            const uint32_t w = ((f + 1u) * M + round_up) >> a.l;
-            put_bits_smem(blob, 8u * j, codes[j], 8u);
-            put_bits_smem(blob, flag_pos0 + a.l * j, f, a.l);
-            put_bits_smem(blob, dpos, delta, w);
-            dpos += w;
+    uint32_t dbase = delta_pos0;
+    for (uint32_t j0 = 0, round = 0; j0 < count; j0 += kCmpThreads, ++round) {
+        const uint32_t j = j0 + (uint32_t)tid;
+        uint32_t delta = 0, f = 0, w = 0;
+        if (j < count) {
+            delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
+            f = flag_of(delta, a.l, inv_m);
+            w = ((f + 1u) * M + round_up) >> a.l;
         }
+        const uint32_t incl = warp_incl_scan(w, lane);
+        if (lane == 31) s.scan_tot2[round & 1u][warp] = incl;
+        __syncthreads();                      // (one barrier per round: the totals are double-buffered)
+        uint32_t before = 0, all = 0;
+#pragma unroll
+        for (int k = 0; k < kCmpWarps; ++k) {
+            const uint32_t t = s.scan_tot2[round & 1u][k];
+            if (k < warp) before += t;
+            all += t;
+        }
+        if (j < count) {
+            put_bits_smem(blob, flag_pos0 + a.l * j, f, a.l);
+            put_bits_smem(blob, dbase + before + (incl - w), delta, w);
+        }
+        dbase += all;
     }
     __syncthreads();      // blob complete
-    *words_out = (delta_pos0 + payload_bits + 31u) >> 5;
+    *words_out = (dbase + 31u) >> 5;
     *M_out = M;
 }
 
@@ -388,16 +393,17 @@ struct ScanState {
     uint32_t words;        // blob words of groups [0, pos)
 };
 
-// Copies the pending tiles' blobs to their places in the stream (pend_prefix holds each tile's
-// exclusive prefix), writes their directory entries and, for the last group, the header.
-__device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
+// Copies the blobs of the pending tiles [pbeg, npend) of one gradient to their places in the stream
+// (pend_prefix holds each tile's exclusive prefix), writes their directory entries and, for the
+// last group, the header.  No barrier inside.
+__device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint32_t jp, int pbeg, int npend, int tid, int lane, int warp) {
     const double S = s.job_sum[jp];
     const uint32_t skip = s.job_skip[jp];
     // ---- copy-out, directory entries, header
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
     uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
     // one warp per pending tile (a dense tile's blob, in global scratch, is copied by the whole block)
-    for (int p0 = 0; p0 < npend; p0 += kCmpWarps) {
+    for (int p0 = pbeg; p0 < npend; p0 += kCmpWarps) {
         const int p = p0 + warp;
         const bool mine = p < npend;
         const uint32_t g = mine ? s.pend_g[p] : 0u, cm = mine ? s.pend_cm[p] : 0u, words = mine ? s.pend_words[p] : 0u,
@@ -435,28 +441,56 @@ __device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint
             outw[15] = a.G;
         }
     }
-    // a dense tile is always the only pending one when it is drained
-    if (npend >= 1 && s.pend_off[npend - 1] == kDenseMark) {
+    // a dense tile is always the last pending one when it is drained
+    if (npend > pbeg && s.pend_off[npend - 1] == kDenseMark) {
         const int p = npend - 1;
         const uint32_t words = s.pend_words[p];
         const uint32_t off = fixed_words + (uint32_t)s.pend_prefix[p];
         const uint64_t end_bytes = ((uint64_t)off + words) << 2;
-        const uint32_t* blob = reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
+        const uint32_t* blob = reinterpret_cast<const uint32_t*>(s.stage[0]);      // (still there: the caller refills the stage afterwards)
         if (end_bytes <= a.out_bytes)
             for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
     }
-    __syncthreads();       // the arena and the pending list are free again
 }
 
-// Gives the pending tiles their places in the stream.  `npend` tiles wait (block-uniform); their
-// group numbers ascend.  Returns false if a poisoned descriptor or a
-// timeout was met (the caller aborts).
-__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
+// Pending tiles [0, n) belong to a gradient whose encode pass is over or nearly so: the last block
+// to finish it writes the exclusive scan of all its descriptors (publish_prefixes).  Fetches the
+// entries of these tiles (bounded polls); a failure shows in s.poison_seen after the next barrier.
+__device__ __forceinline__ void fetch_prefixes(CmpSmem& s, const CmpArgs& a, int n, int tid) {
+    if (tid < n) {
+        const unsigned long long* p = a.prefix + s.pend_g[tid];
+        unsigned long long v = ld_relaxed_u64(p);
+        uint32_t spin = 0;
+        while ((v >> 62) == kDescInvalid) {
+            if (++spin > kWaitLimit) { s.poison_seen = 2u; break; }
+            __nanosleep(64);
+            v = ld_relaxed_u64(p);
+        }
+        if ((v >> 62) == kDescPoison) s.poison_seen = 1u;
+        s.pend_prefix[tid] = ((unsigned long long)desc_count(v) << 32) | desc_words(v);
+    }
+}
+
+// Gives every pending tile its place in the stream and empties the arena.  Tiles [0, nprev) of the
+// list belong to the previous gradient (view ap, slot jp ^ 1): their prefixes come from the
+// published scan.  Tiles [nprev, npend) belong to the gradient being encoded (view a, slot jp;
+// group numbers ascend): the block advances its own scan of the descriptors up to them.  Returns
+// false if a poisoned descriptor or a timeout was met (the caller aborts).
+__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, const CmpArgs& ap, uint32_t jp, int nprev, int npend,
+                                      int tid, int lane, int warp) {
     if (npend == 0) return true;
-    ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
-    const uint32_t g_last = s.pend_g[npend - 1];
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
+    fetch_prefixes(s, ap, nprev, tid);
+    if (npend == nprev) {
+        __syncthreads();
+        if (s.poison_seen) return false;   // (rewritten only at the start of the next drain, behind a barrier)
+        place_pending(s, ap, jp ^ 1u, 0, nprev, tid, lane, warp);
+        __syncthreads();                   // the arena and the pending list are free again
+        return true;
+    }
+    ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
+    const uint32_t g_last = s.pend_g[npend - 1];
     // ---- advance the scan over descriptors [sc.pos, g_last]: batches of kDrainChunks x 512, all loads
     //      of a batch in flight at once, one shuffle scan per chunk, two barriers per batch
     while (sc.pos <= g_last) {
@@ -501,7 +535,7 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, uint32_t jp,
             running += all;
         }
         // the thread that holds one of this block's pending tiles records that tile's exclusive prefix
-        for (int p = 0; p < npend; ++p) {
+        for (int p = nprev; p < npend; ++p) {
             const uint32_t idx = s.pend_g[p];
             if (idx < sc.pos || idx >= sc.pos + (uint32_t)kDrainChunks * kCmpThreads) continue;
             const uint32_t rel = idx - sc.pos;
@@ -524,32 +558,22 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, uint32_t jp,
     sc.pos = g_last + 1u;
     if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after the barrier below)
 
-    place_pending(s, a, jp, npend, tid, lane, warp);
+    place_pending(s, ap, jp ^ 1u, 0, nprev, tid, lane, warp);
+    place_pending(s, a, jp, nprev, npend, tid, lane, warp);
+    __syncthreads();                       // the arena and the pending list are free again
     return true;
 }
 
-// The same once a gradient's encode pass is over: the last block to finish it has written the
-// exclusive scan of all descriptors (publish_prefixes); every block fetches the entries of its
-// pending tiles (bounded polls) and places them.
-__device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32_t jp, int npend, int tid, int lane, int warp) {
-    if (npend == 0) return true;
+// Places tiles [0, n) of the list, all of one gradient whose encode pass is over (slot jp).
+__device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32_t jp, int n, int tid, int lane, int warp) {
+    if (n == 0) return true;
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
-    if (tid < npend) {
-        const unsigned long long* p = a.prefix + s.pend_g[tid];
-        unsigned long long v = ld_relaxed_u64(p);
-        uint32_t spin = 0;
-        while ((v >> 62) == kDescInvalid) {
-            if (++spin > kWaitLimit) { s.poison_seen = 2u; break; }
-            __nanosleep(64);
-            v = ld_relaxed_u64(p);
-        }
-        if ((v >> 62) == kDescPoison) s.poison_seen = 1u;
-        s.pend_prefix[tid] = ((unsigned long long)desc_count(v) << 32) | desc_words(v);
-    }
+    fetch_prefixes(s, a, n, tid);
     __syncthreads();
     if (s.poison_seen) return false;       // (rewritten only at the start of the next drain, behind a barrier)
-    place_pending(s, a, jp, npend, tid, lane, warp);
+    place_pending(s, a, jp, 0, n, tid, lane, warp);
+    __syncthreads();
     return true;
 }
 
@@ -606,13 +630,14 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
 // (and stays in the stage afterwards).  Thread 0 holds the ticket of the tile after the one at
 // hand, taken one iteration before it is used.  sum_begin starts the copy of the first tile and
 // returns; sum_rest does the rest (the caller has something else to do while that copy flies).
+// `limit` bounds the tiles the block takes (a block that only helps with a pass).
 struct SumCursor {
     unsigned int tk;       // thread 0: the look-ahead ticket
     uint32_t     tile;     // the tile whose copy is in flight
 };
 
 __device__ __forceinline__ SumCursor sum_begin(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t c, uint32_t grid,
-                                               uint32_t& pending, int tid) {
+                                               uint32_t limit, uint32_t& pending, int tid) {
     SumCursor cur; cur.tk = 0u;
     if (tid == 0) {
         cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
@@ -623,13 +648,14 @@ __device__ __forceinline__ SumCursor sum_begin(CmpSmem& s, const CmpArgs& a, uin
     if (cur.tile != kNoTicket) {
         issue_tile(s, a, 0, cur.tile, tid);
         pending |= 1u;
-        if (tid == 0 && (full || cur.tile != c)) cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+        if (tid == 0 && limit > 1u && (full || cur.tile != c)) cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
     }
     return cur;
 }
 
 __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t c, uint32_t grid,
-                                         SumCursor cur, uint32_t& parity, uint32_t& pending, int tid, int lane, int warp) {
+                                         uint32_t limit, SumCursor cur, uint32_t& parity, uint32_t& pending,
+                                         int tid, int lane, int warp) {
     unsigned int tk = cur.tk;
     uint32_t tile = cur.tile;
     if (tile == kNoTicket) return;                    // (several gradients, fewer tiles than blocks)
@@ -645,8 +671,9 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         const double u = warp_slab_tree(x, lane);
         if (lane == 0) s.s_warp[q & 1][warp] = u;
         if (tid == 0)                                 // the tile after this one: a ticketed tile, then (one gradient) c, then none
-            s.p1_next[(q + 1) & 1] = full ? (tk < a.G ? tk : kNoTicket)
-                                          : (tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c));
+            s.p1_next[(q + 1) & 1] = q + 1u >= limit ? kNoTicket
+                                     : full ? (tk < a.G ? tk : kNoTicket)
+                                            : (tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c));
         __syncthreads();
         if (s.abort_flag) break;
         if (warp == 0) {
@@ -658,23 +685,23 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         if (nxt == kNoTicket) break;
         issue_tile(s, a, 0, nxt, tid);
         pending |= 1u;
-        if (tid == 0 && (full || nxt != c)) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
+        if (tid == 0 && q + 2u < limit && (full || nxt != c)) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
         tile = nxt;
     }
 }
 
-// Grid barrier of gradient `job` among the `tgrid` blocks that work on it, first half: this
+// Grid barrier of gradient `job` among the `expect` blocks that sum it, first half: this
 // block's partial sums are written.  The last block to arrive clears the count, readies the
 // gradient's ticket counters (encode pass: with one gradient the tiles below `tgrid` are taken;
 // sum pass: zero for the next launch) and sets the gradient's flag to the launch's generation
 // (read by every block when it started, bumped by the last block to leave the kernel: no state
 // outside the workspace, so a launch can be replayed).
 __device__ __forceinline__ void barrier_arrive(CmpSmem& s, Control* ctl, uint32_t job, bool full, uint32_t tgrid,
-                                               unsigned int gen_next, int tid) {
+                                               uint32_t expect, unsigned int gen_next, int tid) {
     if (tid == 0 && !s.abort_flag) {                  // (thread 0 wrote the partials and cleared the descriptors itself)
         __threadfence();
         const unsigned int old = atomicAdd(&ctl->bar_count[job], 1u);
-        if (old == tgrid - 1u) {
+        if (old == expect - 1u) {
             ctl->bar_count[job] = 0u;
             ctl->tickets[job] = full ? 0u : tgrid;
             ctl->tickets1[job] = 0u;
@@ -752,43 +779,64 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         s.team = team;
     }
     __syncthreads();
-    const uint32_t first_job = s.team, step = b.teams;
-    const uint32_t grid = gridDim.x / b.teams;              // blocks that work on a gradient
+    const uint32_t team = s.team, step = b.teams;
+    const uint32_t grid = gridDim.x / b.teams;              // blocks of a team
+    // The team's own gradients: team, team + step, ...  With two teams, to keep their control steps
+    // apart and their ends together: the blocks of team 1 first take up to two tiles each of
+    // gradient 0's sum pass (so team 0 runs ahead), and the team that does not own the last
+    // gradient H joins H's encode pass when it is done with its own.
+    const uint32_t nown = b.jobs > team ? (b.jobs - team + step - 1u) / step : 0u;
+    const uint32_t H = b.jobs - 1u;
+    const bool helper = step == 2u && (H & 1u) != team;
+    const uint32_t niter = nown + (helper ? 1u : 0u);
     uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects
     uint32_t pending = 0;                     // bit st: a copy into stage st has been started and not waited for
     bool aborted = false;
     // the tiles of the gradient before the one at hand that were pending at the end of its encode
     // pass: their count, that gradient's sum and status wait in shared memory
-    bool prev_valid = false;
     uint32_t prev_job = 0u;
-    CmpArgs a = job_view(b, first_job < b.jobs ? first_job : 0u);
+    // The pending list and the arena live across gradients: tiles [0, nprev) of the list are what
+    // the previous gradient's encode pass left behind (placed after this gradient's encode pass,
+    // when their prefixes have long been published), tiles [nprev, npend) belong to this gradient.
+    int nprev = 0, npend = 0;
+    uint32_t arena_used = 0;
+    CmpArgs a = job_view(b, 0u);
 
-    if (first_job < b.jobs) {
-        if (tid == 0) btrace[8u * first_job + 0] = read_globaltimer();
-        const SumCursor cur = sum_begin(s, a, first_job, full, c, grid, pending, tid);
-        sum_rest(s, a, first_job, full, c, grid, cur, parity, pending, tid, lane, warp);
-        if (tid == 0) btrace[8u * first_job + 1] = read_globaltimer();
-        barrier_arrive(s, b.ctl, first_job, full, grid, gen_next, tid);
+    if (step == 2u && team == 1u) {
+        if (tid == 0) btrace[8u * 7u + 0] = read_globaltimer();
+        const SumCursor cur = sum_begin(s, a, 0u, full, c, grid, 2u, pending, tid);
+        sum_rest(s, a, 0u, full, c, grid, 2u, cur, parity, pending, tid, lane, warp);
+        barrier_arrive(s, b.ctl, 0u, full, grid, gridDim.x, gen_next, tid);
+        __syncthreads();
+    }
+    if (nown) {
+        a = job_view(b, team);
+        if (tid == 0) btrace[8u * team + 0] = read_globaltimer();
+        const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
+        sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
+        if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
+        barrier_arrive(s, b.ctl, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid);
     }
 
-    uint32_t it = 0u;                         // gradients this block has started to encode
-    for (uint32_t job = first_job; job < b.jobs && !aborted; job += step, ++it) {
+    for (uint32_t it = 0; it < niter && !aborted; ++it) {
     const uint32_t jp = it & 1u;
+    const uint32_t job = it < nown ? team + it * step : H;
+    const uint32_t enc_expect = (step == 2u && job == H) ? gridDim.x : grid;      // blocks that pass through this encode pass
     a = job_view(b, job);
     __syncthreads();
-    if (job + step < b.jobs && !s.abort_flag) {
+    if (it + 1u < nown && !s.abort_flag) {
         // next gradient's sum pass; this gradient's table while the first copy is in flight
         const uint32_t nj = job + step;
         const CmpArgs an = job_view(b, nj);
         if (tid == 0) btrace[8u * nj + 0] = read_globaltimer();
-        const SumCursor cur = sum_begin(s, an, nj, full, c, grid, pending, tid);
+        const SumCursor cur = sum_begin(s, an, nj, full, c, grid, 0xFFFFFFFFu, pending, tid);
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
         if (!s.abort_flag) make_table(s, a, pw, jp, tid, lane, warp);
         if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
-        sum_rest(s, an, nj, full, c, grid, cur, parity, pending, tid, lane, warp);
+        sum_rest(s, an, nj, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
-        barrier_arrive(s, b.ctl, nj, full, grid, gen_next, tid);
+        barrier_arrive(s, b.ctl, nj, full, grid, grid, gen_next, tid);
     } else {
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
@@ -814,12 +862,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 pending |= 1u;
             }
         }
-        // the previous gradient's last pending tiles (their blobs still sit in the arena)
-        if (prev_valid) {
-            const CmpArgs ap = job_view(b, prev_job);
-            if (!drain_final(s, ap, jp ^ 1u, s.prev_npend, tid, lane, warp)) { aborted = true; break; }
-            prev_valid = false;
-        }
+        const CmpArgs ap = job_view(b, prev_job);
         if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
         const uint32_t skip = s.job_skip[jp];
         const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
@@ -830,8 +873,6 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // filters it, compacts its kept entries into its own list, quantises them and forms their
         // deltas without talking to the other warps; two block barriers per non-empty tile exchange
         // the slab summaries (counts, boundary keys, largest delta -> M) and the payload bits.
-        int npend = 0;
-        uint32_t arena_used = 0;
         const uint32_t round_up = (1u << a.l) - 1u;
         // The block's first tile is the one it summed last (still in shared memory); every further tile
         // is handed out by a ticket counter, so that blocks that met dense tiles take fewer.  Thread 0
@@ -957,10 +998,12 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             const uint32_t g_next = s.next_tile[par];
             const bool more = g_next < a.G;                  // (false for kNoTicket too)
             if (more) {
-                issue_tile(s, a, st, g_next, tid);
-                pending |= 1u << st;
+                if (!overflow) {                 // (a tile too dense for the lists packs its blob in the stage first)
+                    issue_tile(s, a, st, g_next, tid);
+                    pending |= 1u << st;
+                }
                 if (tid == 0) {
-                    // (tiles too dense for the arena drain at once whatever is done: keep their copies overlapped)
+                    // (tiles too dense for the arena drain at once whatever is done)
                     const bool stop_reserving = !overflow && worst_now <= kArenaWords / 4u &&
                         (npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords);
                     ticket_ahead = stop_reserving ? kNoTicket : atomicAdd(a.ticket, 1u);
@@ -969,12 +1012,12 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
             uint32_t words = 0, M = 0, aoff = 0;
             if (count == 0u) {
-                if (npend == kPendMax) { if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; } npend = 0; arena_used = 0; }
+                if (npend == kPendMax) { if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; } nprev = 0; npend = 0; arena_used = 0; }
             } else if (!overflow) {
                 const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
                 if (npend == kPendMax || arena_used + worst > kArenaWords) {
-                    if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
-                    npend = 0; arena_used = 0;
+                    if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
+                    nprev = 0; npend = 0; arena_used = 0;
                 }
                 aoff = arena_used;
                 uint32_t* blob = s.arena + aoff;
@@ -1037,12 +1080,13 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 }
                 arena_used += words;
             } else {
-                // a slab is too dense for its list: block-wide path in global scratch, committed at once
-                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
-                npend = 0; arena_used = 0;
+                // a slab is too dense for its list: block-wide path, blob in the stage, placed at once
+                if (npend == kPendMax) {
+                    if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
+                    nprev = 0; npend = 0; arena_used = 0;
+                }
                 aoff = kDenseMark;
-                pack_tile_dense(s, a, count, warp_base, m, a.grad + ((uint64_t)g << kGroupLog2), ex0, ex1, tot0, tot1,
-                                &words, &M, tid, lane, warp);      // (the stage is being refilled: values come from global memory)
+                pack_tile_dense(s, a, count, warp_base, m, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
             }
             if (tid == 0) {
                 st_relaxed_u64(a.desc + g, desc_pack(kDescValid, count, words));
@@ -1054,14 +1098,19 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             ++npend;
             if (aoff == kDenseMark) {
                 __syncthreads();
-                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
-                npend = 0; arena_used = 0;
+                if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
+                nprev = 0; npend = 0; arena_used = 0;
+                if (more) {                      // the stage is free now (generic-proxy writes before an async-proxy one)
+                    if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    issue_tile(s, a, st, g_next, tid);
+                    pending |= 1u << st;
+                }
             }
             if (g_next == kNoTicket) {
                 // nothing reserved: drain now, then take the next ticket and start its copy
                 __syncthreads();
-                if (!drain(s, a, jp, npend, tid, lane, warp)) { aborted = true; break; }
-                npend = 0; arena_used = 0;
+                if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
+                nprev = 0; npend = 0; arena_used = 0;
                 if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
                 g = s.next_tile[par];
@@ -1078,27 +1127,38 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             }
         }
         if (tid == 0) btrace[8u * job + 5] = read_globaltimer();
-        // what is still pending is placed after the next gradient's sum pass (or below, after the last),
-        // with the prefixes that the last block to get here computes for everybody
-        prev_valid = !aborted;
-        prev_job = job;
+        // this block's tiles of the gradient are published: count it; the last block through computes
+        // the prefixes for everybody
         if (tid == 0) {
-            s.prev_npend = npend;
             s.publisher = 0u;
             if (!aborted) {
                 __threadfence();                            // this block's descriptors before its count
                 const unsigned int old = atomicAdd(a.enc_done, 1u);
-                if (old == grid - 1u) { *a.enc_done = 0u; s.publisher = 1u; __threadfence(); }
+                if (old == enc_expect - 1u) { *a.enc_done = 0u; s.publisher = 1u; __threadfence(); }
             }
         }
         __syncthreads();
         if (s.publisher) publish_prefixes(s, a, tid, lane, warp);
+        // place what the previous gradient left behind; what this one leaves waits for the next turn
+        if (!aborted && nprev > 0) {
+            if (!drain_final(s, ap, jp ^ 1u, nprev, tid, lane, warp)) { aborted = true; break; }
+            const int rest = npend - nprev;
+            uint32_t e_g = 0, e_cm = 0, e_w = 0, e_o = 0;
+            if (tid < rest) { e_g = s.pend_g[nprev + tid]; e_cm = s.pend_cm[nprev + tid]; e_w = s.pend_words[nprev + tid]; e_o = s.pend_off[nprev + tid]; }
+            __syncthreads();
+            if (tid < rest) { s.pend_g[tid] = e_g; s.pend_cm[tid] = e_cm; s.pend_words[tid] = e_w; s.pend_off[tid] = e_o; }
+            __syncthreads();
+            npend = rest;
+        }
+        nprev = npend;
+        if (npend == 0) arena_used = 0;
+        prev_job = job;
     }
     }   // jobs
 
-    if (!aborted && prev_valid) {
+    if (!aborted && nprev > 0) {
         __syncthreads();                           // pending list written by thread 0
-        if (!drain_final(s, a, (it - 1u) & 1u, s.prev_npend, tid, lane, warp)) aborted = true;
+        if (!drain_final(s, job_view(b, prev_job), (niter - 1u) & 1u, nprev, tid, lane, warp)) aborted = true;
     }
     if (tid == 0) btrace[6] = read_globaltimer();   // (slot 6 of the first gradient: end of the launch's last drain)
 
