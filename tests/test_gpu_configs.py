@@ -45,6 +45,36 @@ def _run(wl, check_workers=None):
     return kept_total
 
 
+def _run_batched(wl):
+    """The launch configuration bench.py times: all workers' gradients through one
+    fastsgd_compress_batch call, all streams through one fastsgd_decompress_accumulate_batch call."""
+    n, W = wl.n, wl.workers
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg)
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    grads = [torch.from_numpy(g).cuda() for g in wl.grads]
+    outs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(W)]
+    dense = torch.zeros(n, dtype=torch.float32, device="cuda")
+    odense = np.zeros(n, np.float32)
+    for rep in range(2):                       # the second launch reuses the workspace as the first left it
+        for o in outs:
+            o.fill_(0xA5)
+        assert binding.compress_batch(grads, pg, outs) == 0
+        for w in range(W):
+            total, d, status = binding.stream_info(outs[w])
+            orc, ostream = oracle.compress(wl.grads[w], po)
+            assert status == orc == 0 and total == ostream.size, f"worker {w}"
+            assert np.array_equal(outs[w][:total].cpu().numpy(), ostream), f"worker {w}: stream differs (launch {rep})"
+            if rep == 0:
+                assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+    assert binding.decompress_accumulate_batch(outs, [cap] * W, n, pg, dense) == 0
+    assert binding.decode_status() == 0
+    got = dense.cpu().numpy()
+    assert np.allclose(got, odense, rtol=RTOL, atol=ATOL)
+    assert np.array_equal(got, odense)
+
+
 def test_config1_full():
     wl = workloads.make("c1")
     kept = _run(wl)
@@ -56,6 +86,16 @@ def test_config2_full_four_workers():
     assert wl.n == 25_557_032 and wl.workers == 4
     kept = _run(wl)
     assert abs(kept / (4 * wl.n) - 0.005) < 0.002
+
+
+def test_config2_batched_as_benchmarked():
+    _run_batched(workloads.make("c2"))
+
+
+@pytest.mark.parametrize("keep", [1e-3, 1e-2])
+def test_config4_batched_as_benchmarked(keep):
+    # three of the eight workers in one launch (an odd count: the two teams of blocks get unequal shares)
+    _run_batched(workloads.make("c4", workers=3, keep=keep))
 
 
 def test_config3_full_clustered_sparse():

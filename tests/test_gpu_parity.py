@@ -326,3 +326,41 @@ def test_batched_compress_equals_one_call_per_gradient(ngrads):
         total, d, status = binding.stream_info(bufs[w].view)
         orc, ostream = oracle.compress(grads[ngrads - 1 - w], po)
         assert status == 0 and np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream)
+
+
+@pytest.mark.parametrize("ngrads", [2, 3, 5, 8])
+def test_batched_compress_with_two_teams_of_blocks(ngrads):
+    # enough tiles (>= two per SM) for the launch to split its blocks into two teams that work on
+    # different gradients; gradients with tiles too dense for the per-warp lists, an all-zero one,
+    # a ragged last tile; every stream byte-equal to the oracle's, twice in a row
+    import torch
+    import gpu_util as G
+    n = 330 * 16384 + 777
+    grads = []
+    for w in range(ngrads):
+        g = workloads.student_t_layers(n, seed=10 + w, blocks=12, lo=1e-4, hi=1e-1)
+        grads.append(g)
+    if ngrads > 2:
+        grads[2] = np.zeros(n, np.float32)
+    base = workloads.base_for_keep(grads[0], n // 20)
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    dg = [G.to_dev(v) for v in grads]
+    bufs = [G.Guarded(cap, fill=0x3C) for _ in range(ngrads)]
+    expect = [oracle.compress(g, po) for g in grads]
+    dense_tiles = 0
+    for rep in range(2):
+        assert binding.compress_batch(dg, pg, [b.view for b in bufs]) == 0
+        for w in range(ngrads):
+            total, d, status = binding.stream_info(bufs[w].view)
+            orc, ostream = expect[w]
+            assert status == orc == 0 and total == ostream.size and bufs[w].intact()
+            assert np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream), f"gradient {w}, launch {rep}"
+    # the case is only worth its name if some tile took the dense path (a 1024-entry slab with more than 192 kept)
+    for g in grads[:2]:
+        S = np.abs(g.astype(np.float64)).sum()
+        thr = S / base ** 128
+        k = np.abs(np.concatenate([g, np.zeros((-n) % 1024, np.float32)])) >= thr
+        dense_tiles += int((k.reshape(-1, 1024).sum(1) > 192).sum())
+    assert dense_tiles > 0
