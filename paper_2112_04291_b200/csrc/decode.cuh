@@ -86,8 +86,8 @@ struct DecShared {
     uint32_t           scan[2][kDecWarps];
     uint32_t           big[kDecListMax];
     unsigned long long first_bad;     // min over threads of (key index << 8 | status), block path
-    uint32_t           big_count;
-    uint32_t           pad;
+    uint32_t           big_count;     // large groups this block has found among its own
+    uint32_t           local_g;       // the first of them: decoded by this block itself, the others go to the queue
     unsigned long long tile_bar;      // mbarrier of the bulk copy that loads the tile
     // per stream, for the group the block works on
     uint32_t           g_count[kDecMaxStreams], g_M[kDecMaxStreams], g_off[kDecMaxStreams], g_nwords[kDecMaxStreams],
@@ -340,6 +340,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     if (tid == 0) {
         mbar_init(&s.tile_bar, 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s.big_count = 0u;
     }
     uint32_t tile_parity = 0;
     // ---- headers: thread w checks stream w
@@ -372,7 +373,15 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             read_dir(a, reinterpret_cast<const uint32_t*>(a.stream[lane]), g, s.total_words[lane], &count, &M, &off, &nwords);
         if (!__any_sync(kFullMask, count != 0u)) continue;
         if (__any_sync(kFullMask, count > kDecWarpMax)) {
-            if (lane == 0) {                 // hand it to the grid-wide queue: reserve a slot, then fill it (g + 1: 0 = empty)
+            // a large group: the first one the block finds is its own (directory entries kept in shared
+            // memory), any further one goes to the grid-wide queue: reserve a slot, then fill it (g + 1: 0 = empty)
+            uint32_t nth = 0;
+            if (lane == 0) nth = atomicAdd(&s.big_count, 1u);
+            nth = __shfl_sync(kFullMask, nth, 0);
+            if (nth == 0u) {
+                if (lane < (int)W) { s.g_count[lane] = count; s.g_M[lane] = M; s.g_off[lane] = off; s.g_nwords[lane] = nwords; }
+                if (lane == 0) s.local_g = g;
+            } else if (lane == 0) {
                 const uint32_t slot = atomicAdd(a.q_ctl + 4, 1u);
                 __threadfence();
                 *reinterpret_cast<volatile unsigned int*>(a.q_list + slot) = g + 1u;
@@ -408,26 +417,33 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     //      and the slot lies beyond the last reservation.
     unsigned int* q_taken = a.q_ctl + 1, *q_done = a.q_ctl + 2, *q_exited = a.q_ctl + 3, *q_reserved = a.q_ctl + 4;
     if (tid == 0) { __threadfence(); atomicAdd(q_done, 1u); }
-    for (;;) {
-        if (tid == 0) {
-            uint32_t got = 0xFFFFFFFFu;
-            const uint32_t i = atomicAdd(q_taken, 1u);
-            uint32_t spin = 0;
-            for (;;) {
-                if (i < a.G) {
-                    const uint32_t e = *reinterpret_cast<volatile unsigned int*>(a.q_list + i);
-                    if (e != 0u) { got = e - 1u; *reinterpret_cast<volatile unsigned int*>(a.q_list + i) = 0u; break; }
+    const bool local_first = s.big_count > 0u;      // (written before the barrier above)
+    for (uint32_t round = 0;; ++round) {
+        const bool local = round == 0u && local_first;
+        uint32_t g;
+        if (local) {
+            g = s.local_g;
+        } else {
+            if (tid == 0) {
+                uint32_t got = 0xFFFFFFFFu;
+                const uint32_t i = atomicAdd(q_taken, 1u);
+                uint32_t spin = 0;
+                for (;;) {
+                    if (i < a.G) {
+                        const uint32_t e = *reinterpret_cast<volatile unsigned int*>(a.q_list + i);
+                        if (e != 0u) { got = e - 1u; *reinterpret_cast<volatile unsigned int*>(a.q_list + i) = 0u; break; }
+                    }
+                    if (*reinterpret_cast<volatile unsigned int*>(q_done) >= gridDim.x &&
+                        i >= *reinterpret_cast<volatile unsigned int*>(q_reserved)) break;      // nothing will fill it
+                    if (i >= a.G || ++spin > kDecSpinLimit) break;
+                    __nanosleep(100);
                 }
-                if (*reinterpret_cast<volatile unsigned int*>(q_done) >= gridDim.x &&
-                    i >= *reinterpret_cast<volatile unsigned int*>(q_reserved)) break;      // nothing will fill it
-                if (i >= a.G || ++spin > kDecSpinLimit) break;
-                __nanosleep(100);
+                s.big[0] = got;
             }
-            s.big[0] = got;
+            __syncthreads();
+            g = s.big[0];
+            if (g == 0xFFFFFFFFu) break;
         }
-        __syncthreads();
-        const uint32_t g = s.big[0];
-        if (g == 0xFFFFFFFFu) break;
         ++taken;
         const uint64_t lo64 = (uint64_t)g << a.group_log2;
         const uint64_t hi64 = lo64 + (1ull << a.group_log2);
@@ -440,7 +456,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             mbar_expect_tx(&s.tile_bar, span * 4u);
             bulk_load(s.u.tile, a.dense + lo, span * 4u, &s.tile_bar);
         }
-        if (tid < (int)W) {
+        if (!local && tid < (int)W) {
             uint32_t count = 0, M = 0, off = 0, nwords = 0;
             if (s.ok[tid])
                 read_dir(a, reinterpret_cast<const uint32_t*>(a.stream[tid]), g, s.total_words[tid], &count, &M, &off, &nwords);
