@@ -48,6 +48,7 @@ struct Control {
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
 constexpr uint64_t kThrOffset      = 256;    // float thr[132]: RU32(B_k)
+constexpr uint64_t kJobSumOffset   = 800;    // double S[8]: the sum of each gradient of a k_compress launch
 constexpr uint64_t kTraceOffset    = 1024;   // u64 trace[<=496][8]: per-block %globaltimer stamps (profiling aid)
 constexpr uint64_t kQueueOffset    = 32768;  // u32 queue[2^17]: decoder's grid-wide queue of groups (zero between launches)
 constexpr uint64_t kQueueBytes     = 4ull << 17;

@@ -80,8 +80,8 @@ struct CmpSmem {
     double   s_nodes[256];                   // nodes of the final sum tree when a thread holds more than 8 partials
     uint32_t pad5;
     uint32_t publisher;                      // this block was the last to finish the gradient's encode pass
-    uint32_t team;                           // 0: sums the next gradient before it encodes this one; 1: after
-    uint32_t pad4;
+    uint32_t team;                           // which of the two teams of blocks this one belongs to
+    uint32_t last_arrival;                   // this block was the last to arrive at a grid barrier
     uint32_t p1_next[2];                     // the same for the sum pass
     uint32_t arena[kArenaWords];
     uint32_t wvals[kCmpWarps][kSlabCap];     // per warp: kept values (fp32 bits), then their code bytes
@@ -577,9 +577,13 @@ __device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32
     return true;
 }
 
-// Run by the last block to finish a gradient's encode pass (every descriptor is published by then):
-// exclusive scan of all descriptors into a.prefix, kDrainChunks x 512 at a time.  A descriptor that
-// is not valid poisons its own and every later prefix.
+// Exclusive scan of all descriptors of a gradient into a.prefix, kDrainChunks x 512 at a time.
+// POLL = false: run by the last block to finish the gradient's encode pass (every descriptor is
+// published by then).  POLL = true: run by the first block to finish it, which follows the
+// others' descriptors as they appear (bounded polls), so that the prefixes are complete right
+// after the last tile is published -- used for the launch's last gradient, where everybody waits
+// for them.  A descriptor that is not valid (or never comes) poisons its own and every later prefix.
+template <bool POLL>
 __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, int tid, int lane, int warp) {
     unsigned long long running = 0ull;
     bool bad = false;
@@ -593,6 +597,15 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
         }
 #pragma unroll
         for (int j = 0; j < kDrainChunks; ++j) {
+            if (POLL && !bad) {
+                const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+                uint32_t spin = 0;
+                while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
+                    if (++spin > kWaitLimit) break;
+                    __nanosleep(64);
+                    own[j] = ld_relaxed_u64(a.desc + idx);
+                }
+            }
             if ((own[j] >> 62) != kDescValid) { bad_here = true; own[j] = 0ull; }
             own[j] = ((unsigned long long)desc_count(own[j]) << 32) | desc_words(own[j]);
             unsigned long long incl = own[j];
@@ -691,17 +704,29 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
 }
 
 // Grid barrier of gradient `job` among the `expect` blocks that sum it, first half: this
-// block's partial sums are written.  The last block to arrive clears the count, readies the
-// gradient's ticket counters (encode pass: with one gradient the tiles below `tgrid` are taken;
-// sum pass: zero for the next launch) and sets the gradient's flag to the launch's generation
-// (read by every block when it started, bumped by the last block to leave the kernel: no state
-// outside the workspace, so a launch can be replayed).
-__device__ __forceinline__ void barrier_arrive(CmpSmem& s, Control* ctl, uint32_t job, bool full, uint32_t tgrid,
-                                               uint32_t expect, unsigned int gen_next, int tid) {
-    if (tid == 0 && !s.abort_flag) {                  // (thread 0 wrote the partials and cleared the descriptors itself)
-        __threadfence();
-        const unsigned int old = atomicAdd(&ctl->bar_count[job], 1u);
-        if (old == expect - 1u) {
+// block's partial sums are written.  The last block to arrive reduces all partials on the fixed
+// tree (alone: hundreds of blocks reading the same few lines at once queue up in L2), stores S,
+// clears the count, readies the gradient's ticket counters (encode pass: with one gradient the
+// tiles below `tgrid` are taken; sum pass: zero for the next launch) and sets the gradient's flag
+// to the launch's generation (read by every block when it started, bumped by the last block to
+// leave the kernel: no state outside the workspace, so a launch can be replayed).
+__device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t tgrid,
+                                               uint32_t expect, unsigned int gen_next, int tid, int lane, int warp) {
+    Control* ctl = a.ctl;
+    __syncthreads();
+    if (tid == 0) {                                   // (thread 0 wrote the partials and cleared the descriptors itself)
+        s.last_arrival = 0u;
+        if (!s.abort_flag) {
+            __threadfence();
+            const unsigned int old = atomicAdd(&ctl->bar_count[job], 1u);
+            if (old == expect - 1u) { s.last_arrival = 1u; __threadfence(); }
+        }
+    }
+    __syncthreads();
+    if (s.last_arrival) {
+        const double S = reduce_partials(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
+        if (tid == 0) {
+            reinterpret_cast<double*>(reinterpret_cast<unsigned char*>(ctl) + kJobSumOffset)[job] = S;
             ctl->bar_count[job] = 0u;
             ctl->tickets[job] = full ? 0u : tgrid;
             ctl->tickets1[job] = 0u;
@@ -724,11 +749,11 @@ __device__ __forceinline__ void barrier_wait(CmpSmem& s, Control* ctl, uint32_t 
     __syncthreads();
 }
 
-// After the grid barrier of gradient `job`: every block reduces the partials itself (same tree),
-// S -> boundary table RU32(B_k) in shared memory; resets the block's per-gradient scan state.
-__device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const PowTable& pw, uint32_t jp,
+// After the grid barrier of gradient `job`: S (reduced by the last block to arrive) -> boundary
+// table RU32(B_k) in shared memory; resets the block's per-gradient scan state.
+__device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const PowTable& pw, uint32_t job, uint32_t jp,
                                            int tid, int lane, int warp) {
-    const double S = reduce_partials(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
+    const double S = __ldcg(reinterpret_cast<const double*>(reinterpret_cast<const unsigned char*>(a.ctl) + kJobSumOffset) + job);
     const bool finite = isfinite(S);
     const uint32_t skip = !finite ? 2u : (S == 0.0 ? 1u : 0u);
     if (tid <= (int)a.tau) {
@@ -806,7 +831,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[8u * 7u + 0] = read_globaltimer();
         const SumCursor cur = sum_begin(s, a, 0u, full, c, grid, 2u, pending, tid);
         sum_rest(s, a, 0u, full, c, grid, 2u, cur, parity, pending, tid, lane, warp);
-        barrier_arrive(s, b.ctl, 0u, full, grid, gridDim.x, gen_next, tid);
+        barrier_arrive(s, a, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
         __syncthreads();
     }
     if (nown) {
@@ -815,7 +840,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
         sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
-        barrier_arrive(s, b.ctl, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid);
+        barrier_arrive(s, a, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
     }
 
     for (uint32_t it = 0; it < niter && !aborted; ++it) {
@@ -832,15 +857,15 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         const SumCursor cur = sum_begin(s, an, nj, full, c, grid, 0xFFFFFFFFu, pending, tid);
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
-        if (!s.abort_flag) make_table(s, a, pw, jp, tid, lane, warp);
+        if (!s.abort_flag) make_table(s, a, pw, job, jp, tid, lane, warp);
         if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
         sum_rest(s, an, nj, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
-        barrier_arrive(s, b.ctl, nj, full, grid, grid, gen_next, tid);
+        barrier_arrive(s, an, nj, full, grid, grid, gen_next, tid, lane, warp);
     } else {
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
-        if (!s.abort_flag) make_table(s, a, pw, jp, tid, lane, warp);
+        if (!s.abort_flag) make_table(s, a, pw, job, jp, tid, lane, warp);
         if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
     }
     __syncthreads();
@@ -1134,11 +1159,16 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             if (!aborted) {
                 __threadfence();                            // this block's descriptors before its count
                 const unsigned int old = atomicAdd(a.enc_done, 1u);
-                if (old == enc_expect - 1u) { *a.enc_done = 0u; s.publisher = 1u; __threadfence(); }
+                if (old == enc_expect - 1u) { *a.enc_done = 0u; __threadfence(); }
+                // the launch's last gradient: the first block through follows the others; else the last one scans
+                s.publisher = (job == H ? old == 0u : old == enc_expect - 1u) ? 1u : 0u;
             }
         }
         __syncthreads();
-        if (s.publisher) publish_prefixes(s, a, tid, lane, warp);
+        if (s.publisher) {
+            if (job == H) publish_prefixes<true>(s, a, tid, lane, warp);
+            else publish_prefixes<false>(s, a, tid, lane, warp);
+        }
         // place what the previous gradient left behind; what this one leaves waits for the next turn
         if (!aborted && nprev > 0) {
             if (!drain_final(s, ap, jp ^ 1u, nprev, tid, lane, warp)) { aborted = true; break; }
