@@ -84,6 +84,8 @@ struct DecShared {
     uint32_t           total_words[kDecMaxStreams];
     uint32_t           ok[kDecMaxStreams];
     uint32_t           scan[2][kDecWarps];
+    uint32_t           scanm[2][4][kDecWarps];   // the same for up to four streams scanned together
+    unsigned long long first_bad_m[4];
     uint32_t           big[kDecListMax];
     unsigned long long first_bad;     // min over threads of (key index << 8 | status), block path
     uint32_t           big_count;     // large groups this block has found among its own
@@ -327,7 +329,181 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
     }
 }
 
-__global__ void __launch_bounds__(kDecThreads)
+// Exclusive scans of NS values per thread at once (one barrier for all of them in a block).
+template <bool BLOCK, int NS>
+__device__ __forceinline__ void excl_scan_multi(const uint32_t (&v)[NS], uint32_t (&excl)[NS], uint32_t (&total)[NS],
+                                                DecShared& s, int lane, int warp, int which) {
+    uint32_t incl[NS];
+#pragma unroll
+    for (int w = 0; w < NS; ++w) incl[w] = warp_incl_scan(v[w], lane);
+    if (!BLOCK) {
+#pragma unroll
+        for (int w = 0; w < NS; ++w) { total[w] = __shfl_sync(kFullMask, incl[w], 31); excl[w] = incl[w] - v[w]; }
+        return;
+    }
+    if (lane == 31) {
+#pragma unroll
+        for (int w = 0; w < NS; ++w) s.scanm[which][w][warp] = incl[w];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        uint32_t before = 0, all = 0;
+#pragma unroll
+        for (int k = 0; k < kDecWarps; ++k) {
+            const uint32_t t = s.scanm[which][w][k];
+            if (k < warp) before += t;
+            all += t;
+        }
+        total[w] = all;
+        excl[w] = before + incl[w] - v[w];
+    }
+}
+
+// One group of NS streams, decoded together by a warp (BLOCK = false) or by the block: the streams
+// are parsed side by side (independent dependency chains, one scan barrier for all of them), each
+// is validated completely, and the sound ones are applied in stream order.  Every stream holds at
+// most KMAX * nthreads keys, so a thread's run of consecutive keys stays in registers.
+template <bool BLOCK, int NS, int KMAX>
+__device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, const uint32_t* const (&blob)[NS],
+                                             const uint32_t (&nwords)[NS], const uint32_t (&count)[NS], const uint32_t (&M)[NS],
+                                             const float* const (&val)[NS], uint32_t g, float* tile,
+                                             int t, int nthreads, int lane, int warp) {
+    const uint64_t lo64 = (uint64_t)g << a.group_log2;
+    const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+    const uint32_t lo = (uint32_t)lo64;
+    const uint32_t hi = (uint32_t)(hi64 < a.n ? hi64 : a.n);
+    const bool lead = (t == 0);
+    const uint32_t levels_m1 = (1u << a.l) - 1u;
+    uint32_t jb[NS], je[NS], wv[NS][KMAX], dv[NS][KMAX];
+    bool live[NS];                                    // uniform: the stream has keys here and has not failed a check
+
+    // phase 1: widths from the flags; their sum fixes the blob's length, which must be the directory's
+    uint32_t wsum[NS], pos0[NS], wtotal[NS];
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        live[w] = count[w] != 0u;
+        const uint32_t K = (count[w] + nthreads - 1) / nthreads;
+        jb[w] = min(count[w], (uint32_t)t * K); je[w] = min(count[w], jb[w] + K);
+        const uint32_t flag_pos0 = 8u * count[w];
+        wsum[w] = 0u;
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            wv[w][k] = 0u;
+            if (jb[w] + k < je[w]) {
+                const uint32_t f = get_bits(blob[w], nwords[w], flag_pos0 + a.l * (jb[w] + k), a.l);
+                wv[w][k] = ((f + 1u) * M[w] + levels_m1) >> a.l;
+            }
+            wsum[w] += wv[w][k];
+        }
+    }
+    excl_scan_multi<BLOCK, NS>(wsum, pos0, wtotal, s, lane, warp, 0);
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        const uint32_t delta_pos0 = (8u + a.l) * count[w];
+        pos0[w] += delta_pos0;
+        if (live[w] && (((uint64_t)delta_pos0 + wtotal[w] + 31ull) >> 5) != nwords[w]) {
+            if (lead) dec_fail(a, g, 0u, kStBadDirectory);
+            live[w] = false;
+        }
+    }
+
+    // phase 2: this thread's deltas and their sum, then the key before its first one
+    uint32_t dsum[NS], key0[NS], dtotal[NS];
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        uint32_t pos = pos0[w];
+        dsum[w] = 0u;
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            dv[w][k] = live[w] ? get_bits(blob[w], nwords[w], pos, wv[w][k]) : 0u;     // width 0 beyond the run: reads as 0
+            pos += wv[w][k];
+            dsum[w] = min(dsum[w] + dv[w][k], 1u << 21);                               // saturates only when already invalid
+        }
+    }
+    excl_scan_multi<BLOCK, NS>(dsum, key0, dtotal, s, lane, warp, 1);
+
+    // validation of each stream's whole group before anything of it is applied: first key index that
+    // repeats, leaves the group, or carries a code beyond tau
+    unsigned long long bad[NS];
+    bool any_bad = false;
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        key0[w] += lo;
+        bad[w] = ~0ull;
+        uint32_t key = key0[w];
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            const uint32_t j = jb[w] + k;
+            if (live[w] && j < je[w] && bad[w] == ~0ull) {
+                key += dv[w][k];
+                const uint32_t code = (blob[w][j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+                if ((j > 0 && dv[w][k] == 0u) || key >= hi) bad[w] = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
+                else if ((code & 0x7Fu) + 1u > a.tau) bad[w] = ((unsigned long long)j << 8) | (unsigned)kStBadCode;
+            }
+        }
+        any_bad = any_bad || bad[w] != ~0ull;
+    }
+    if (BLOCK) {
+        if (__syncthreads_or(any_bad ? 1 : 0)) {          // one barrier when every stream is sound
+            if (t < NS) s.first_bad_m[t] = ~0ull;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < NS; ++w) if (bad[w] != ~0ull) atomicMin(&s.first_bad_m[w], bad[w]);
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < NS; ++w) bad[w] = s.first_bad_m[w];
+            __syncthreads();
+        }
+    } else if (__any_sync(kFullMask, any_bad)) {
+#pragma unroll
+        for (int w = 0; w < NS; ++w) {
+            const uint32_t blo = __reduce_min_sync(kFullMask, (uint32_t)(bad[w] < 0xFFFFFFFFull ? bad[w] : 0xFFFFFFFFull));
+            bad[w] = blo == 0xFFFFFFFFu ? ~0ull : (unsigned long long)blo;
+        }
+    }
+#pragma unroll
+    for (int w = 0; w < NS; ++w)
+        if (live[w] && bad[w] != ~0ull) {
+            if (lead) dec_fail(a, g, (uint32_t)(bad[w] >> 8), (int)(bad[w] & 0xFFull));
+            live[w] = false;
+        }
+
+    // phases 3-4 and the aggregation, stream by stream
+    bool first = true;
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        if (!live[w]) continue;
+        if (!first) { if (BLOCK) __syncthreads(); else __syncwarp(); }    // the stream before may hold the same keys
+        first = false;
+        uint32_t key = key0[w];
+        uint32_t kk[KMAX]; float vv[KMAX];
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            const uint32_t j = jb[w] + k;
+            kk[k] = 0xFFFFFFFFu; vv[k] = 0.f;
+            if (j < je[w]) {
+                key += dv[w][k];
+                const uint32_t code = (blob[w][j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+                const float mag = val[w][(code & 0x7Fu) + 1u];
+                kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
+            }
+        }
+        if (BLOCK && tile != nullptr) {
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k)
+                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = __fadd_rn(tile[kk[k] - lo], vv[k]);
+        } else {
+            float dd[KMAX];                                    // distinct keys: all loads, then all stores
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = __fadd_rn(dd[k], vv[k]);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kDecThreads, 2)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char dec_smem_raw[];
     DecShared& s = *reinterpret_cast<DecShared*>(dec_smem_raw);
@@ -399,14 +575,30 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             for (uint32_t i = lane; i < nw; i += 32) stage[b + i] = __ldg(src + i);
         }
         __syncwarp();
-        for (uint32_t w = 0; w < W; ++w) {
-            const uint32_t c = __shfl_sync(kFullMask, count, w);
-            const uint32_t b = __shfl_sync(kFullMask, base, w), nw = __shfl_sync(kFullMask, nwords, w), m = __shfl_sync(kFullMask, M, w);
-            if (c == 0u) continue;
-            decode_group<false>(a, s, stage + b, nw, g, c, m, s.val[w], nullptr, lane, 32, lane, warp);
-            __syncwarp();          // this stream's stores before the next stream's loads of the same keys
+        // up to four streams at a time, parsed side by side and applied in stream order
+        for (uint32_t w0 = 0; w0 < W; w0 += 4u) {
+            const uint32_t ns = W - w0 < 4u ? W - w0 : 4u;
+            const uint32_t* bl[4]; uint32_t nwv[4], cv[4], mv[4]; const float* vl[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t src = (uint32_t)i < ns ? w0 + i : w0;
+                const uint32_t c = __shfl_sync(kFullMask, count, src), b = __shfl_sync(kFullMask, base, src);
+                nwv[i] = __shfl_sync(kFullMask, nwords, src); mv[i] = __shfl_sync(kFullMask, M, src);
+                cv[i] = (uint32_t)i < ns ? c : 0u;
+                bl[i] = stage + b; vl[i] = s.val[src];
+            }
+            if (ns == 1u) {
+                const uint32_t* b1[1] = {bl[0]}; const uint32_t n1[1] = {nwv[0]}, c1[1] = {cv[0]}, m1[1] = {mv[0]}; const float* v1[1] = {vl[0]};
+                decode_multi<false, 1, 4>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+            } else if (ns == 2u) {
+                const uint32_t* b2[2] = {bl[0], bl[1]}; const uint32_t n2[2] = {nwv[0], nwv[1]}, c2[2] = {cv[0], cv[1]}, m2[2] = {mv[0], mv[1]};
+                const float* v2[2] = {vl[0], vl[1]};
+                decode_multi<false, 2, 4>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+            } else {
+                decode_multi<false, 4, 4>(a, s, bl, nwv, cv, mv, vl, g, nullptr, lane, 32, lane, warp);
+            }
+            __syncwarp();          // these streams' stores before the next streams' loads of the same keys
         }
-        __syncwarp();
     }
     __syncthreads();
 
@@ -488,12 +680,29 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         }
         for (uint32_t w = 0; w < W; ++w) {
             const uint32_t c = s.g_count[w];
-            if (c == 0u) continue;
             const uint32_t* blob = s.g_valid[w] ? s.bstage + s.g_base[w]
                                                 : reinterpret_cast<const uint32_t*>(a.stream[w]) + s.g_off[w];
-            decode_group<true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
-                               tid, kDecThreads, lane, warp);
-            __syncthreads();       // this stream's updates before the next stream's
+            // short runs per thread: the leaner parser, two streams side by side where the next one qualifies too
+            if (c <= 4u * (uint32_t)kDecThreads && w + 1u < W && s.g_count[w + 1u] <= 4u * (uint32_t)kDecThreads) {
+                const uint32_t w2 = w + 1u;
+                const uint32_t* blob2 = s.g_valid[w2] ? s.bstage + s.g_base[w2]
+                                                      : reinterpret_cast<const uint32_t*>(a.stream[w2]) + s.g_off[w2];
+                const uint32_t* b2[2] = {blob, blob2}; const uint32_t n2[2] = {s.g_nwords[w], s.g_nwords[w2]};
+                const uint32_t c2[2] = {c, s.g_count[w2]}, m2[2] = {s.g_M[w], s.g_M[w2]};
+                const float* v2[2] = {s.val[w], s.val[w2]};
+                decode_multi<true, 2, 4>(a, s, b2, n2, c2, m2, v2, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+                ++w;
+            } else if (c == 0u) {
+                continue;
+            } else if (c <= 4u * (uint32_t)kDecThreads) {
+                const uint32_t* b1[1] = {blob}; const uint32_t n1[1] = {s.g_nwords[w]}, c1[1] = {c}, m1[1] = {s.g_M[w]};
+                const float* v1[1] = {s.val[w]};
+                decode_multi<true, 1, 4>(a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+            } else {
+                decode_group<true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                                   tid, kDecThreads, lane, warp);
+            }
+            __syncthreads();       // these streams' updates before the next stream's
         }
         if (use_tile && tid == 0) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // the updates above, before the copy reads them
