@@ -364,3 +364,60 @@ def test_batched_compress_with_two_teams_of_blocks(ngrads):
         k = np.abs(np.concatenate([g, np.zeros((-n) % 1024, np.float32)])) >= thr
         dense_tiles += int((k.reshape(-1, 1024).sum(1) > 192).sum())
     assert dense_tiles > 0
+
+
+@pytest.mark.parametrize("keep_div", [400, 30])
+def test_damaged_stream_among_sound_ones_in_one_launch(keep_div):
+    # three streams decoded by one launch, the middle one damaged inside a group's blob: the status is
+    # the oracle's for that stream, nothing outside dense_out is touched, and the groups the damage
+    # does not reach hold exactly what the oracle holds.  keep_div = 400 keeps the groups small
+    # (decoded by warps, streams parsed side by side), 30 makes them large enough for whole blocks.
+    import torch
+    import gpu_util as G
+    n = 6 * 16384 + 77
+    grads = [workloads.student_t_layers(n, seed=70 + w, blocks=1, lo=1e-2, hi=1e-2) for w in range(3)]
+    base = workloads.base_for_keep(grads[0], n // keep_div)
+    pg, po = _params(base)
+    streams = []
+    for v in grads:
+        orc, st = oracle.compress(v, po)
+        assert orc == 0
+        streams.append(st)
+    G_ = (n + 16383) // 16384
+    bad_group = 3
+    off = int.from_bytes(streams[1][64 + 8 * bad_group + 4:64 + 8 * bad_group + 8].tobytes(), "little")
+    cnt = int.from_bytes(streams[1][64 + 8 * bad_group:64 + 8 * bad_group + 4].tobytes(), "little") & 0xFFFFFF
+    assert cnt > 8
+    for kind in ("flags", "deltas"):
+        dmg = streams[1].copy()
+        if kind == "flags":
+            dmg[4 * off + cnt:4 * off + cnt + 2] ^= 0xFF           # first flag bytes: widths change, blob length no longer fits
+        else:
+            nxt = int.from_bytes(dmg[64 + 8 * (bad_group + 1) + 4:64 + 8 * (bad_group + 1) + 8].tobytes(), "little")
+            dmg[4 * nxt - 6:4 * nxt - 2] = 0                       # last deltas zero: a repeated key
+        expect = oracle.decompress_accumulate(dmg, n, po, np.zeros(n, np.float32))
+        assert expect != 0
+        odense = np.zeros(n, np.float32)
+        assert oracle.decompress_accumulate(streams[0], n, po, odense) == 0
+        good_only = odense.copy()
+        assert oracle.decompress_accumulate(streams[2], n, po, good_only) == 0
+        full = odense.copy()
+        assert oracle.decompress_accumulate(streams[1], n, po, full) == 0
+        assert oracle.decompress_accumulate(streams[2], n, po, full) == 0
+        binding.ensure_workspace(n, pg)
+        devs, sizes = [], []
+        for st in (streams[0], dmg, streams[2]):
+            pad = (-st.size) % 16
+            devs.append(G.to_dev(np.concatenate([st, np.zeros(pad + 16, np.uint8)])))
+            sizes.append(st.size)
+        buf = G.Guarded(4 * n)
+        dense = buf.view.view(torch.float32)
+        dense.zero_()
+        assert binding.decompress_accumulate_batch(devs, sizes, n, pg, dense) == 0
+        st = binding.decode_status()
+        assert st == expect and buf.intact(), (kind, st, expect)
+        got = dense.cpu().numpy()
+        lo, hi = bad_group * 16384, (bad_group + 1) * 16384
+        # the damaged group of the damaged stream is dropped as a whole; every other (group, stream) is applied
+        assert np.array_equal(got[:lo], full[:lo]) and np.array_equal(got[hi:], full[hi:]), kind
+        assert np.array_equal(got[lo:hi], good_only[lo:hi]), kind
