@@ -144,6 +144,93 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Config 5: n = 2^10 .. 2^30 in powers of 4, keep in {0.01, 0.1, 1, 10} %, one worker; compress-only,
+    decompress-only and combined, each as the median of single eager calls timed with CUDA events,
+    with a 256 MiB write between calls (every size up to 2^24 would otherwise sit in L2).  Writes a
+    markdown table to args.sweep and prints one JSON line about the largest point."""
+    import torch
+    from paper_2112_04291_b200 import binding, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    peak, peak_kind = measured_peak()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    iters = max(5, min(args.steps, 20))
+    rows, last = [], None
+    max_log2 = args.sweep_max_log2
+    for log2n in range(10, max_log2 + 1, 2):
+        n = 1 << log2n
+        v = workloads.normal_outliers(n, seed=0)
+        grad = torch.from_numpy(v).to(dev)
+        for keep in (1e-4, 1e-3, 1e-2, 1e-1):
+            base = workloads.base_for_keep(v, max(1, int(round(keep * n))))
+            pg = binding.params(base)
+            binding.ensure_workspace(n, pg, dev)
+            cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+            out = torch.zeros(cap, dtype=torch.uint8, device=dev)
+            dense = torch.zeros(n, dtype=torch.float32, device=dev)
+
+            def comp():
+                rc = binding.compress(grad, pg, out)
+                assert rc == 0, rc
+
+            def dec():
+                rc = binding.decompress_accumulate(out, cap, n, pg, dense)
+                assert rc == 0, rc
+
+            def both():
+                comp()
+                dec()
+
+            def med(fn):
+                ts = []
+                for it in range(iters + 3):
+                    flush.fill_(it & 0xFF)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                return statistics.median(ts)
+
+            both()
+            total, d, status = binding.stream_info(out)
+            assert status == 0 and binding.decode_status() == 0
+            ms_c, ms_d, ms_b = med(comp), med(dec), med(both)
+            alg_c, alg_d = 8.0 * n + total, total + 8.0 * d
+            row = {"log2n": log2n, "keep": keep, "kept": d, "stream_bytes": total,
+                   "compress_ms": ms_c, "decompress_ms": ms_d, "combined_ms": ms_b,
+                   "compress_in_gbs": 4.0 * n / ms_c / 1e6, "decompress_in_gbs": 4.0 * n / ms_d / 1e6,
+                   "combined_in_gbs": 4.0 * n / ms_b / 1e6,
+                   "compress_frac": alg_c / ms_c / 1e6 / peak, "decompress_frac": alg_d / ms_d / 1e6 / peak,
+                   "combined_frac": (alg_c + alg_d) / ms_b / 1e6 / peak}
+            rows.append(row)
+            last = row
+            del out, dense
+        del grad, v
+    with open(args.sweep, "w") as f:
+        f.write("| n | keep | kept | stream bytes | compress us | GB/s in | frac | decompress us | GB/s in | frac | combined us | GB/s in | frac |\n")
+        f.write("|---|---|---|---|---|---|---|---|---|---|---|---|---|\n")
+        for r in rows:
+            f.write("| 2^%d | %g | %d | %d | %.1f | %.0f | %.3f | %.1f | %.0f | %.3f | %.1f | %.0f | %.3f |\n" % (
+                r["log2n"], r["keep"], r["kept"], r["stream_bytes"], r["compress_ms"] * 1e3, r["compress_in_gbs"],
+                r["compress_frac"], r["decompress_ms"] * 1e3, r["decompress_in_gbs"], r["decompress_frac"],
+                r["combined_ms"] * 1e3, r["combined_in_gbs"], r["combined_frac"]))
+    line = {"metric": METRIC, "value": last["combined_in_gbs"], "unit": UNIT, "n_gpus": 1, "steps": iters, "warmup": 3,
+            "ms_per_step": last["combined_ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "c5 sweep, largest point: n=2^%d, keep %g" % (last["log2n"], last["keep"]),
+                       "points": len(rows), "table": args.sweep, "l2": "256 MiB written between timed calls",
+                       "launch": "eager, one call per timed region"},
+            "roofline": {"bound": "hbm", "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
+                         "achieved": last["combined_frac"] * peak, "frac": last["combined_frac"], "traffic": None}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -157,6 +244,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph of the step")
+    ap.add_argument("--sweep", default=None, metavar="FILE", help="config 5: size x keep-ratio sweep, markdown table written to FILE")
+    ap.add_argument("--sweep-max-log2", type=int, default=30)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -165,6 +254,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
         return
 
     import torch

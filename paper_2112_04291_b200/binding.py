@@ -139,8 +139,11 @@ def ensure_workspace(n: int, p: Params, device="cuda") -> torch.Tensor:
     """Allocates (torch) and registers a workspace large enough for n entries, if needed."""
     need = workspace_bytes(n, p)
     ws = _workspace_keepalive
-    if ws is None or ws.numel() < need or ws.device != torch.device(device, torch.cuda.current_device()):
-        ws = torch.empty(max(need, 4096), dtype=torch.uint8, device=device)
+    dev = torch.device(device)
+    if dev.index is None:
+        dev = torch.device(dev.type, torch.cuda.current_device())
+    if ws is None or ws.numel() < need or ws.device != dev:
+        ws = torch.empty(max(need, 4096), dtype=torch.uint8, device=dev)
         set_workspace(ws)
     return ws
 
