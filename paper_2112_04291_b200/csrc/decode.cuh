@@ -27,9 +27,10 @@ namespace fsg {
 constexpr int      kDecThreads     = 256;
 constexpr int      kDecWarps       = kDecThreads / 32;
 constexpr int      kDecMaxStreams  = 8;       // streams per launch
-constexpr uint32_t kDecWarpMax     = 128;     // groups with more keys (in any stream) go to the whole block
+constexpr uint32_t kDecWarpMax     = 256;     // groups with more keys (in any stream) go to the whole block (128 with more than two streams)
+constexpr uint32_t kDecWarpSide    = 128;     // up to this many keys per stream a warp parses the streams side by side
 constexpr int      kDecListMax     = 512;     // groups one block may own
-constexpr uint32_t kWarpStageWords = 1088;    // >= kDecMaxStreams * ceil(128 * (8 + 5 + 20) / 32)
+constexpr uint32_t kWarpStageWords = 2048;    // >= kDecMaxStreams * ceil(kDecWarpMax * (8 + 5 + 14) / 32); 8 warps x 8 KiB = the tile's 64 KiB
 constexpr uint32_t kBlockStageWords = 10240;  // blobs larger than this in total are parsed from global memory
 constexpr uint32_t kDecSpinLimit   = 1u << 20;
 
@@ -542,13 +543,15 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
 
     if (tid == 0) T1 = read_globaltimer_dec();
     // ---- this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
+    // (a warp applies the streams of a group one after the other: with many streams the whole block is the better choice sooner)
+    const uint32_t warp_max = W <= 2u ? kDecWarpMax : kDecWarpSide;
     for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += kDecWarps * gridDim.x) {
         // lane w reads and checks stream w's directory entry
         uint32_t count = 0, M = 0, off = 0, nwords = 0;
         if (lane < (int)W && s.ok[lane])
             read_dir(a, reinterpret_cast<const uint32_t*>(a.stream[lane]), g, s.total_words[lane], &count, &M, &off, &nwords);
         if (!__any_sync(kFullMask, count != 0u)) continue;
-        if (__any_sync(kFullMask, count > kDecWarpMax)) {
+        if (__any_sync(kFullMask, count > warp_max)) {
             // a large group: the first one the block finds is its own (directory entries kept in shared
             // memory), any further one goes to the grid-wide queue: reserve a slot, then fill it (g + 1: 0 = empty)
             uint32_t nth = 0;
@@ -575,6 +578,20 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             for (uint32_t i = lane; i < nw; i += 32) stage[b + i] = __ldg(src + i);
         }
         __syncwarp();
+        if (__any_sync(kFullMask, count > kDecWarpSide)) {
+            // longer runs per lane: two streams at a time
+            for (uint32_t w0 = 0; w0 < W; w0 += 2u) {
+                const uint32_t w1 = w0 + 1u < W ? w0 + 1u : w0;
+                const uint32_t* b2[2]; uint32_t n2[2], c2[2], m2[2]; const float* v2[2];
+                c2[0] = __shfl_sync(kFullMask, count, w0); c2[1] = w0 + 1u < W ? __shfl_sync(kFullMask, count, w1) : 0u;
+                b2[0] = stage + __shfl_sync(kFullMask, base, w0); b2[1] = stage + __shfl_sync(kFullMask, base, w1);
+                n2[0] = __shfl_sync(kFullMask, nwords, w0); n2[1] = __shfl_sync(kFullMask, nwords, w1);
+                m2[0] = __shfl_sync(kFullMask, M, w0); m2[1] = __shfl_sync(kFullMask, M, w1);
+                v2[0] = s.val[w0]; v2[1] = s.val[w1];
+                decode_multi<false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                __syncwarp();      // these streams' stores before the next streams' loads of the same keys
+            }
+        } else
         // up to four streams at a time, parsed side by side and applied in stream order
         for (uint32_t w0 = 0; w0 < W; w0 += 4u) {
             const uint32_t ns = W - w0 < 4u ? W - w0 : 4u;
