@@ -376,7 +376,7 @@ def main():
         run_step()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    step_exceeds_l2 = 4.0 * n * W > 2 * 126e6
+    step_exceeds_l2 = 4.0 * n * W > 1.5 * 126e6
     ms_total = timed(run_step, args.steps) if step_exceeds_l2 else timed_flushed(run_step, args.steps)
     launches = launches_per_step * args.steps
     sampler.sample_once()
@@ -441,7 +441,7 @@ def main():
                    "keep_fraction": wl.keep_fraction, "base": wl.base, "tau": wl.tau, "flag_bits": wl.flag_bits,
                    "group_log2": wl.group_log2, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": "cuda graph replay of the step's C-ABI calls" if g_step else "eager C-ABI calls",
-                   "l2": ("inputs of one step (W x 4n bytes) exceed twice the L2 size; no explicit flush" if step_exceeds_l2
+                   "l2": ("inputs of one step (W x 4n bytes) exceed 1.5 x the L2 size; no explicit flush" if step_exceeds_l2
                           else "256 MiB written before every timed step (its inputs would fit in L2)")
                          + "; decompress-only leg: 256 MiB written before every call"},
         "clocks": sampler.summary(),

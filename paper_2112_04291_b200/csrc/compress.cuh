@@ -267,6 +267,10 @@ __device__ __forceinline__ double reduce_partials(const double* partials, uint32
     return block_tree(y, s_tree, lane, warp);
 }
 
+// ceil(2^16 / M) for M = 1..20
+__device__ __constant__ uint32_t c_inv_m[21] = {0, 65536, 32768, 21846, 16384, 13108, 10923, 9363, 8192, 7282, 6554, 5958,
+                                                5462, 5042, 4682, 4370, 4096, 3856, 3641, 3450, 3277};
+
 // flag of a delta with bit length bl: least f with ceil((f+1) M / 2^l) >= bl, which is
 // floor((bl-1) 2^l / M) for bl >= 1; the division is a multiplication by ceil(2^16 / M)
 __device__ __forceinline__ uint32_t flag_of(uint32_t delta, uint32_t l, uint32_t inv_m) {
@@ -353,7 +357,7 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
     // ---- M; flags and deltas, 512 consecutive keys per round
     const uint32_t maxd = s.max_delta;
     const uint32_t M = maxd ? (32u - __clz(maxd)) : 1u;
-    const uint32_t inv_m = (65536u + M - 1u) / M;
+    const uint32_t inv_m = c_inv_m[M];
     const uint32_t round_up = (1u << a.l) - 1u;
     const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a.l * count;
     uint32_t dbase = delta_pos0;
@@ -913,35 +917,18 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
             }
-            // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c.
-            // A row (128 consecutive entries, one float4 per lane) is looked at entry by entry only
-            // if some lane holds an entry that reaches the threshold.
+            // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c
             const float* tile = s.stage[st];
             uint32_t m = 0;
             if (!skip) {
                 const float4* row = reinterpret_cast<const float4*>(tile + warp * 1024) + lane;
-                float rowmx[8];
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
                     const float4 q = row[r * 32];
-                    rowmx[r] = fmaxf(fmaxf(fabsf(q.x), fabsf(q.y)), fmaxf(fabsf(q.z), fabsf(q.w)));
-                }
-                const float mx = fmaxf(fmaxf(fmaxf(rowmx[0], rowmx[1]), fmaxf(rowmx[2], rowmx[3])),
-                                       fmaxf(fmaxf(rowmx[4], rowmx[5]), fmaxf(rowmx[6], rowmx[7])));
-                if (__any_sync(kFullMask, mx >= thr_e)) {
-#pragma unroll
-                    for (int r = 0; r < 8; ++r) {
-                        const bool has = rowmx[r] >= thr_e;
-                        if (__any_sync(kFullMask, has)) {
-                            if (has) {
-                                const float4 q = row[r * 32];
-                                m |= (fabsf(q.x) >= thr_e ? 1u : 0u) << (4 * r);
-                                m |= (fabsf(q.y) >= thr_e ? 1u : 0u) << (4 * r + 1);
-                                m |= (fabsf(q.z) >= thr_e ? 1u : 0u) << (4 * r + 2);
-                                m |= (fabsf(q.w) >= thr_e ? 1u : 0u) << (4 * r + 3);
-                            }
-                        }
-                    }
+                    if (fabsf(q.x) >= thr_e) m |= 1u << (4 * r);
+                    if (fabsf(q.y) >= thr_e) m |= 2u << (4 * r);
+                    if (fabsf(q.z) >= thr_e) m |= 4u << (4 * r);
+                    if (fabsf(q.w) >= thr_e) m |= 8u << (4 * r);
                 }
             }
             // ---- warp-local compaction in index order: per-row counts scanned over the lanes, four
@@ -962,7 +949,23 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 if (slab_count <= kSlabCap) {
                     uint16_t* wk = s.wkeys[warp];
                     uint32_t* wv = s.wvals[warp];
-                    if (m != 0u) {
+                    if (slab_count <= 64u) {
+                        // few entries: one round per kept entry of the lane that holds most
+                        // (position = entries of earlier rows + entries of earlier lanes in the row + earlier ones of the lane in the row)
+                        const uint32_t t0 = tot0 + (tot0 << 8) + (tot0 << 16) + (tot0 << 24);      // inclusive prefix of the rows' totals, a byte per row (<= 64)
+                        const uint32_t t1 = tot1 + (tot1 << 8) + (tot1 << 16) + (tot1 << 24) + (t0 >> 24) * 0x01010101u;
+                        const unsigned long long rowex = ((unsigned long long)(t1 - tot1 + ex1) << 32) | (t0 - tot0 + ex0);   // exclusive row prefix + lanes before
+                        uint32_t mm = m;
+                        while (mm) {
+                            const uint32_t b = (uint32_t)__ffs((int)mm) - 1u;
+                            mm &= mm - 1u;
+                            const uint32_t r = b >> 2;
+                            const uint32_t pos = ((uint32_t)(rowex >> (8u * r)) & 0xFFu) + (uint32_t)__popc(m & ((1u << b) - 1u) & (0xFu << (4u * r)));
+                            const uint32_t k = warp * 1024 + r * 128 + lane * 4 + (b & 3u);
+                            wk[pos] = (uint16_t)k;
+                            wv[pos] = __float_as_uint(tile[k]);
+                        }
+                    } else if (m != 0u) {
                         uint32_t row_base = 0;
 #pragma unroll
                         for (int r = 0; r < 8; ++r) {
@@ -1060,18 +1063,26 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 const uint32_t maxd_l = lane < kCmpWarps ? max(s.sum_maxd[par][lane], bd_l) : 0u;
                 const uint32_t maxd = __reduce_max_sync(kFullMask, maxd_l);
                 M = maxd ? (32u - __clz(maxd)) : 1u;
-                const uint32_t inv_m = (65536u + M - 1u) / M;
+                const uint32_t inv_m = c_inv_m[M];
                 const uint32_t my_bd = __shfl_sync(kFullMask, bd_l, warp);
                 const uint32_t my_cnt = __shfl_sync(kFullMask, cnt_l, warp);
                 const uint16_t* wk = s.wkeys[warp];
                 const uint32_t* wv = s.wvals[warp];
-                // payload bits of my slab
+                // payload bits of my slab; what the first 32 entries need again when packing stays in registers
+                uint32_t d0 = 0, f0 = 0, w0 = 0;
+                if ((uint32_t)lane < my_cnt) {
+                    d0 = lane ? (uint32_t)wk[lane] - (uint32_t)wk[lane - 1] : my_bd;
+                    f0 = flag_of(d0, a.l, inv_m);
+                    w0 = ((f0 + 1u) * M + round_up) >> a.l;
+                }
+                const uint32_t w0_incl = warp_incl_scan(w0, lane);
                 uint32_t bits = 0;
-                for (uint32_t j = lane; j < my_cnt; j += 32) {
-                    const uint32_t delta = j ? (uint32_t)wk[j] - (uint32_t)wk[j - 1] : my_bd;
+                for (uint32_t j = 32u + lane; j < my_cnt; j += 32) {
+                    const uint32_t delta = (uint32_t)wk[j] - (uint32_t)wk[j - 1];
                     bits += ((flag_of(delta, a.l, inv_m) + 1u) * M + round_up) >> a.l;
                 }
-                bits = __reduce_add_sync(kFullMask, bits);
+                if (my_cnt > 32u) bits = __reduce_add_sync(kFullMask, bits);
+                bits += __shfl_sync(kFullMask, w0_incl, 31);
                 if (lane == 0) s.sum_bits[par][warp] = bits;
                 {
                     const uint32_t bound_words = (count * (8u + a.l + M) + 31u) >> 5;
@@ -1086,17 +1097,24 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 words = (delta_pos0 + payload_bits + 31u) >> 5;
                 // pack my slab's entries: codes | flags | deltas (most significant bit first)
                 uint32_t dbase = delta_pos0 + bits_before;
-                for (uint32_t j0 = 0; j0 < my_cnt; j0 += 32) {
+                if ((uint32_t)lane < my_cnt) {
+                    const uint32_t q = warp_base + lane;                  // rank of the entry in the group
+                    put_bits_smem(blob, 8u * q, wv[lane] & 0xFFu, 8u);
+                    put_bits_smem(blob, flag_pos0 + a.l * q, f0, a.l);
+                    put_bits_smem(blob, dbase + (w0_incl - w0), d0, w0);
+                }
+                dbase += __shfl_sync(kFullMask, w0_incl, 31);
+                for (uint32_t j0 = 32u; j0 < my_cnt; j0 += 32) {
                     const uint32_t j = j0 + lane;
                     uint32_t delta = 0, f = 0, w = 0;
                     if (j < my_cnt) {
-                        delta = j ? (uint32_t)wk[j] - (uint32_t)wk[j - 1] : my_bd;
+                        delta = (uint32_t)wk[j] - (uint32_t)wk[j - 1];
                         f = flag_of(delta, a.l, inv_m);
                         w = ((f + 1u) * M + round_up) >> a.l;
                     }
                     const uint32_t w_incl = warp_incl_scan(w, lane);
                     if (j < my_cnt) {
-                        const uint32_t q = warp_base + j;                 // rank of the entry in the group
+                        const uint32_t q = warp_base + j;
                         put_bits_smem(blob, 8u * q, wv[j] & 0xFFu, 8u);
                         put_bits_smem(blob, flag_pos0 + a.l * q, f, a.l);
                         put_bits_smem(blob, dbase + (w_incl - w), delta, w);
