@@ -279,15 +279,17 @@ __device__ __forceinline__ uint32_t flag_of(uint32_t delta, uint32_t l, uint32_t
 }
 
 // L = least k in [0, tau] with |v| >= B_k (Eq. 2-3 as a table search; holds for k = tau), raised
-// to 1, and the sign: the code byte
+// to 1, and the sign: the code byte.  The search starts from an estimate of log_b(S / |v|)
+// (thr[130] = log2 S, thr[131] = 1 / log2 b, both approximate) and walks the non-increasing
+// table from there, so the result does not depend on how good the estimate is.
 __device__ __forceinline__ uint32_t code_byte_of(const float* thr, uint32_t tau, float val) {
     const float av = fabsf(val);
-    uint32_t lo = 0, hi = tau;
-    while (lo < hi) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (av >= thr[mid]) hi = mid; else lo = mid + 1;
-    }
-    const uint32_t L = lo < 1u ? 1u : lo;
+    int guess = (int)((thr[130] - __log2f(av)) * thr[131]) + 1;
+    guess = max(0, min((int)tau, guess));
+    uint32_t L = (uint32_t)guess;
+    while (L > 0u && av >= thr[L - 1u]) --L;
+    while (L < tau && av < thr[L]) ++L;
+    L = L < 1u ? 1u : L;
     return (val < 0.0f ? 0x80u : 0u) | (L - 1u);
 }
 
@@ -767,6 +769,8 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
         s.thr[tid] = finite ? fmaxf(__double2float_ru(Bk), __int_as_float(1)) : __int_as_float(0x7f800000);
     }
     if (tid == 0) {
+        s.thr[130] = (float)log2(S);                  // (only steer the table search)
+        s.thr[131] = (float)(1.0 / log2(a.base));
         s.job_sum[jp] = S; s.job_skip[jp] = skip;
         s.sc_pos = 0u; s.sc_count = 0u; s.sc_words = 0u;
         s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
