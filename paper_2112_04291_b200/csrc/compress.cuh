@@ -469,7 +469,7 @@ __device__ __forceinline__ void fetch_prefixes(CmpSmem& s, const CmpArgs& a, int
         uint32_t spin = 0;
         while ((v >> 62) == kDescInvalid) {
             if (++spin > kWaitLimit) { s.poison_seen = 2u; break; }
-            __nanosleep(64);
+            if (spin > 32u) __nanosleep(32);
             v = ld_relaxed_u64(p);
         }
         if ((v >> 62) == kDescPoison) s.poison_seen = 1u;
@@ -608,7 +608,7 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
                 uint32_t spin = 0;
                 while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
                     if (++spin > kWaitLimit) break;
-                    __nanosleep(64);
+                    if (spin > 32u) __nanosleep(32);
                     own[j] = ld_relaxed_u64(a.desc + idx);
                 }
             }
@@ -645,8 +645,9 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
 }
 
 // Phase 1 for one gradient: fp64 partial sum of every 2^14-entry tile.  Tiles grid..G-1 are handed
-// out by a ticket counter (so that the blocks finish together); the block's own tile c comes last
-// (and stays in the stage afterwards).  Thread 0 holds the ticket of the tile after the one at
+// out by a ticket counter (so that the blocks finish together; with one gradient from the last
+// tile down, so that the encode pass starts on what L2 still holds); the block's own tile c comes
+// last (and stays in the stage afterwards).  Thread 0 holds the ticket of the tile after the one at
 // hand, taken one iteration before it is used.  sum_begin starts the copy of the first tile and
 // returns; sum_rest does the rest (the caller has something else to do while that copy flies).
 // `limit` bounds the tiles the block takes (a block that only helps with a pass).
@@ -660,7 +661,7 @@ __device__ __forceinline__ SumCursor sum_begin(CmpSmem& s, const CmpArgs& a, uin
     SumCursor cur; cur.tk = 0u;
     if (tid == 0) {
         cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
-        s.p1_next[0] = full ? (cur.tk < a.G ? cur.tk : kNoTicket) : (grid + cur.tk < a.G ? grid + cur.tk : c);
+        s.p1_next[0] = full ? (cur.tk < a.G ? cur.tk : kNoTicket) : (grid + cur.tk < a.G ? a.G - 1u - cur.tk : c);
     }
     __syncthreads();
     cur.tile = s.p1_next[0];
@@ -692,7 +693,7 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         if (tid == 0)                                 // the tile after this one: a ticketed tile, then (one gradient) c, then none
             s.p1_next[(q + 1) & 1] = q + 1u >= limit ? kNoTicket
                                      : full ? (tk < a.G ? tk : kNoTicket)
-                                            : (tile == c ? kNoTicket : (grid + tk < a.G ? grid + tk : c));
+                                            : (tile == c ? kNoTicket : (grid + tk < a.G ? a.G - 1u - tk : c));
         __syncthreads();
         if (s.abort_flag) break;
         if (warp == 0) {
@@ -748,7 +749,7 @@ __device__ __forceinline__ void barrier_wait(CmpSmem& s, Control* ctl, uint32_t 
         uint32_t spin = 0;
         while (ld_acquire_u32(&ctl->bar_flag[job]) != gen_next) {
             if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
-            if (spin > 8u) __nanosleep(64);
+            if (spin > 64u) __nanosleep(32);
         }
         __threadfence();
     }
