@@ -10,7 +10,7 @@
 
 #include "common.cuh"
 #include "sum.cuh"
-#include "encode.cuh"
+#include "bits.cuh"
 #include "compress.cuh"
 #include "decode.cuh"
 
@@ -110,8 +110,6 @@ int ensure_device_setup() {
     if (g_state.attrs_set && g_state.device == dev) return FASTSGD_OK;
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
-    if (cudaFuncSetAttribute(k_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EncSmem)) != cudaSuccess)
-        return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_compress, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
     int b1 = 0, b2 = 0, b3 = 0;

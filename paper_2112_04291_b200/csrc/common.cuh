@@ -30,9 +30,9 @@ struct PowTable {
 // Control block at the start of the workspace.
 struct Control {
     unsigned int       done;           // blocks of the sum kernel that have finished (self-resetting)
-    unsigned int       ticket;         // next group for the encode kernel
+    unsigned int       ticket;         // (unused)
     unsigned int       error;          // encode: non-zero once a bounded wait ran out
-    unsigned int       skip;           // 0 encode normally, 1 sum == 0, 2 sum not finite
+    unsigned int       skip;           // (unused)
     unsigned long long decode_status;  // min over failures of (group << 32 | key index << 8 | status)
     double             sum;            // S
     unsigned int       bar_gen;        // launches of k_compress that have finished

@@ -25,7 +25,7 @@
 
 #include "common.cuh"
 #include "sum.cuh"
-#include "encode.cuh"
+#include "bits.cuh"
 
 namespace fsg {
 

@@ -19,7 +19,7 @@
 #include <cstddef>
 
 #include "common.cuh"
-#include "encode.cuh"
+#include "bits.cuh"
 #include "compress.cuh"     // mbarrier / bulk-copy primitives
 
 namespace fsg {
