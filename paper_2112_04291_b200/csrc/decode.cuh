@@ -588,7 +588,12 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 n2[0] = __shfl_sync(kFullMask, nwords, w0); n2[1] = __shfl_sync(kFullMask, nwords, w1);
                 m2[0] = __shfl_sync(kFullMask, M, w0); m2[1] = __shfl_sync(kFullMask, M, w1);
                 v2[0] = s.val[w0]; v2[1] = s.val[w1];
-                decode_multi<false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                if (w0 + 1u < W) {
+                    decode_multi<false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                } else {
+                    const uint32_t* b1[1] = {b2[0]}; const uint32_t n1[1] = {n2[0]}, c1[1] = {c2[0]}, m1[1] = {m2[0]}; const float* v1[1] = {v2[0]};
+                    decode_multi<false, 1, 8>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+                }
                 __syncwarp();      // these streams' stores before the next streams' loads of the same keys
             }
         } else
