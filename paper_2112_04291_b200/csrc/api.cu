@@ -116,9 +116,16 @@ int ensure_device_setup() {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
     g_state.cmp_blocks_per_sm = b3;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
-    if (cudaFuncSetAttribute(k_decode_accumulate, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+    if (cudaFuncSetAttribute(k_decode_accumulate<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
         return FASTSGD_E_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, k_decode_accumulate, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    {   // both instantiations must be resident with the grid the launch uses (the queue of large groups relies on it)
+        int b2a = 0, b2b = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2a, k_decode_accumulate<false>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2b, k_decode_accumulate<true>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        b2 = b2a < b2b ? b2a : b2b;
+    }
     g_state.device = dev;
     g_state.sm_count = sms;
     g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
@@ -362,7 +369,8 @@ int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uin
         da.group_log2 = params->group_log2;
         {
             LaunchTimer lt(2, st);
-            k_decode_accumulate<<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            if (da.W == 1u) k_decode_accumulate<true><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            else k_decode_accumulate<false><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
         }
         g_launches.fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;

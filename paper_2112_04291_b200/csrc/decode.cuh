@@ -365,15 +365,21 @@ __device__ __forceinline__ void excl_scan_multi(const uint32_t (&v)[NS], uint32_
 // are parsed side by side (independent dependency chains, one scan barrier for all of them), each
 // is validated completely, and the sound ones are applied in stream order.  Every stream holds at
 // most KMAX * nthreads keys, so a thread's run of consecutive keys stays in registers.
-template <bool BLOCK, int NS, int KMAX>
+template <bool BLOCK, int NS, int KMAX, bool TWO_GROUPS = false>
 __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, const uint32_t* const (&blob)[NS],
                                              const uint32_t (&nwords)[NS], const uint32_t (&count)[NS], const uint32_t (&M)[NS],
                                              const float* const (&val)[NS], uint32_t g, float* tile,
-                                             int t, int nthreads, int lane, int warp) {
-    const uint64_t lo64 = (uint64_t)g << a.group_log2;
-    const uint64_t hi64 = lo64 + (1ull << a.group_log2);
-    const uint32_t lo = (uint32_t)lo64;
-    const uint32_t hi = (uint32_t)(hi64 < a.n ? hi64 : a.n);
+                                             int t, int nthreads, int lane, int warp, uint32_t g_other = 0xFFFFFFFFu) {
+    // (g_other: slots 1.. hold another group of the same stream instead of other streams of group g)
+    uint32_t gs[NS], lo[NS], hi[NS];
+#pragma unroll
+    for (int w = 0; w < NS; ++w) {
+        gs[w] = (w == 0 || !TWO_GROUPS) ? g : g_other;
+        const uint64_t lo64 = (uint64_t)gs[w] << a.group_log2;
+        const uint64_t hi64 = lo64 + (1ull << a.group_log2);
+        lo[w] = (uint32_t)lo64;
+        hi[w] = (uint32_t)(hi64 < a.n ? hi64 : a.n);
+    }
     const bool lead = (t == 0);
     const uint32_t levels_m1 = (1u << a.l) - 1u;
     uint32_t jb[NS], je[NS], wv[NS][KMAX], dv[NS][KMAX];
@@ -404,7 +410,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
         const uint32_t delta_pos0 = (8u + a.l) * count[w];
         pos0[w] += delta_pos0;
         if (live[w] && (((uint64_t)delta_pos0 + wtotal[w] + 31ull) >> 5) != nwords[w]) {
-            if (lead) dec_fail(a, g, 0u, kStBadDirectory);
+            if (lead) dec_fail(a, gs[w], 0u, kStBadDirectory);
             live[w] = false;
         }
     }
@@ -430,7 +436,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
     bool any_bad = false;
 #pragma unroll
     for (int w = 0; w < NS; ++w) {
-        key0[w] += lo;
+        key0[w] += lo[w];
         bad[w] = ~0ull;
         uint32_t key = key0[w];
 #pragma unroll
@@ -439,7 +445,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
             if (live[w] && j < je[w] && bad[w] == ~0ull) {
                 key += dv[w][k];
                 const uint32_t code = (blob[w][j >> 2] >> (8u * (j & 3u))) & 0xFFu;
-                if ((j > 0 && dv[w][k] == 0u) || key >= hi) bad[w] = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
+                if ((j > 0 && dv[w][k] == 0u) || key >= hi[w]) bad[w] = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
                 else if ((code & 0x7Fu) + 1u > a.tau) bad[w] = ((unsigned long long)j << 8) | (unsigned)kStBadCode;
             }
         }
@@ -466,7 +472,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
 #pragma unroll
     for (int w = 0; w < NS; ++w)
         if (live[w] && bad[w] != ~0ull) {
-            if (lead) dec_fail(a, g, (uint32_t)(bad[w] >> 8), (int)(bad[w] & 0xFFull));
+            if (lead) dec_fail(a, gs[w], (uint32_t)(bad[w] >> 8), (int)(bad[w] & 0xFFull));
             live[w] = false;
         }
 
@@ -493,7 +499,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
         if (BLOCK && tile != nullptr) {
 #pragma unroll
             for (int k = 0; k < KMAX; ++k)
-                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = __fadd_rn(tile[kk[k] - lo], vv[k]);
+                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = __fadd_rn(tile[kk[k] - lo[w]], vv[k]);
         } else {
             float dd[KMAX];                                    // distinct keys: all loads, then all stores
 #pragma unroll
@@ -504,6 +510,26 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
     }
 }
 
+// Copies a blob of nw words into shared memory: all of a lane's loads (up to four) in flight before its stores.
+__device__ __forceinline__ void stage_blob(uint32_t* dst, const uint32_t* src, uint32_t nw, int lane) {
+    for (uint32_t i0 = 0; i0 < nw; i0 += 128u) {
+        uint32_t r[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t i = i0 + (uint32_t)u * 32u + (uint32_t)lane;
+            r[u] = i < nw ? __ldg(src + i) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t i = i0 + (uint32_t)u * 32u + (uint32_t)lane;
+            if (i < nw) dst[i] = r[u];
+        }
+    }
+}
+
+// ONE_STREAM: the launch holds a single stream (its own instantiation, so that the code of the
+// many-stream paths and of the two-groups-per-warp path do not weigh on each other)
+template <bool ONE_STREAM>
 __global__ void __launch_bounds__(kDecThreads, 2)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char dec_smem_raw[];
@@ -545,6 +571,71 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     // ---- this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
     // (a warp applies the streams of a group one after the other: with many streams the whole block is the better choice sooner)
     const uint32_t warp_max = W <= 2u ? kDecWarpMax : kDecWarpSide;
+    if (ONE_STREAM) {
+        // One stream: a warp takes its groups two at a time (lane 0: group g, lane 1: the warp's next
+        // group), so that their directory reads, blob copies, parses and updates overlap.
+        const uint32_t stride = kDecWarps * gridDim.x;
+        const uint32_t* sw0 = reinterpret_cast<const uint32_t*>(a.stream[0]);
+        for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += 2u * stride) {
+            const uint32_t gl = g + (uint32_t)lane * stride;
+            uint32_t count = 0, M = 0, off = 0, nwords = 0;
+            if (lane < 2 && gl < a.G && s.ok[0]) read_dir(a, sw0, gl, s.total_words[0], &count, &M, &off, &nwords);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const uint32_t cq = __shfl_sync(kFullMask, count, q);
+                if (cq <= warp_max) continue;
+                // a large group: the block's first one stays with it, further ones go to the grid-wide queue
+                const uint32_t mq = __shfl_sync(kFullMask, M, q), oq = __shfl_sync(kFullMask, off, q), nq = __shfl_sync(kFullMask, nwords, q);
+                if (lane == 0) {
+                    const uint32_t nth = atomicAdd(&s.big_count, 1u);
+                    if (nth == 0u) {
+                        s.g_count[0] = cq; s.g_M[0] = mq; s.g_off[0] = oq; s.g_nwords[0] = nq;
+                        s.local_g = g + (uint32_t)q * stride;
+                    } else {
+                        const uint32_t slot = atomicAdd(a.q_ctl + 4, 1u);
+                        __threadfence();
+                        *reinterpret_cast<volatile unsigned int*>(a.q_list + slot) = g + (uint32_t)q * stride + 1u;
+                    }
+                }
+                if (lane == q) { count = 0u; nwords = 0u; }
+            }
+            if (!__any_sync(kFullMask, count != 0u)) continue;
+            if (count == 0u) nwords = 0u;
+            const uint32_t nw_incl = warp_incl_scan(nwords, lane);
+            const uint32_t base = nw_incl - nwords;
+            uint32_t* stage = s.u.wstage[warp];
+            const uint32_t* b2[2]; uint32_t n2[2], c2[2], m2[2]; const float* v2[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                c2[q] = __shfl_sync(kFullMask, count, q); n2[q] = __shfl_sync(kFullMask, nwords, q);
+                m2[q] = __shfl_sync(kFullMask, M, q); b2[q] = stage + __shfl_sync(kFullMask, base, q); v2[q] = s.val[0];
+            }
+            // both copies' loads in flight together
+            {
+                const uint32_t o0 = __shfl_sync(kFullMask, off, 0), o1 = __shfl_sync(kFullMask, off, 1);
+                const uint32_t tot = n2[0] + n2[1];
+                for (uint32_t i0 = 0; i0 < tot; i0 += 128u) {
+                    uint32_t r[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t i = i0 + (uint32_t)u * 32u + (uint32_t)lane;
+                        r[u] = i < n2[0] ? __ldg(sw0 + o0 + i) : (i < tot ? __ldg(sw0 + o1 + (i - n2[0])) : 0u);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t i = i0 + (uint32_t)u * 32u + (uint32_t)lane;
+                        if (i < tot) stage[i] = r[u];          // (slot 1's blob follows slot 0's: base = n2[0])
+                    }
+                }
+            }
+            __syncwarp();
+            if (c2[0] <= kDecWarpSide && c2[1] <= kDecWarpSide)
+                decode_multi<false, 2, 4, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
+            else
+                decode_multi<false, 2, 8, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
+            __syncwarp();
+        }
+    } else
     for (uint32_t g = blockIdx.x + warp * gridDim.x; g < a.G; g += kDecWarps * gridDim.x) {
         // lane w reads and checks stream w's directory entry
         uint32_t count = 0, M = 0, off = 0, nwords = 0;
