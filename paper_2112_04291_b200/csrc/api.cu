@@ -110,10 +110,17 @@ int ensure_device_setup() {
     if (g_state.attrs_set && g_state.device == dev) return FASTSGD_OK;
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
-    if (cudaFuncSetAttribute(k_compress, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+    if (cudaFuncSetAttribute(k_compress<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_compress<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
     int b1 = 0, b2 = 0, b3 = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+    {
+        int b3b = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress<false>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (b3b < b3) b3 = b3b;
+    }
     g_state.cmp_blocks_per_sm = b3;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_decode_accumulate<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
@@ -303,7 +310,7 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
         cudaError_t err;
         {
             LaunchTimer lt(1, st);
-            err = cudaLaunchCooperativeKernel((const void*)k_compress, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
+            err = cudaLaunchCooperativeKernel(cb.jobs > 1u ? (const void*)k_compress<true> : (const void*)k_compress<false>, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
                                               sizeof(CmpSmem), st);
         }
         if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }

@@ -788,6 +788,9 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
 // latencies of the control steps hide behind tile copies in flight.  place(j) puts the tiles of
 // gradient j that were still pending at the end of its encode pass.  With a single gradient the
 // block's last tile of the sum pass stays in shared memory for the encode pass.
+// SEVERAL: the launch holds more than one gradient (its own instantiation: the single-gradient
+// launch carries none of the team and pipelining code, and the other way round)
+template <bool SEVERAL>
 __global__ void __launch_bounds__(kCmpThreads, 2)
 k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
@@ -796,7 +799,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     const uint32_t c = blockIdx.x;
     unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kJobTraceOffset) + 64u * c;
 
-    const bool full = b.jobs > 1u;            // several gradients: every tile of every pass is handed out by ticket
+    constexpr bool full = SEVERAL;            // several gradients: every tile of every pass is handed out by ticket
     unsigned int gen_next = 0u;
     if (tid == 0) {
         gen_next = ld_acquire_u32(&b.ctl->bar_gen) + 1u;      // before this block can arrive at a barrier
