@@ -301,11 +301,13 @@ __device__ __forceinline__ uint32_t code_byte_of(const float* thr, uint32_t tau,
 // `m` is the kept mask of this thread's 32 entries.
 static_assert((uint64_t)kTile * (8u + 5u + (uint32_t)kGroupLog2) <= (uint64_t)kTile * 32u, "the widest blob fits the stage");
 
-__device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, uint32_t count,
-                                             uint32_t warp_base, uint32_t m,
-                                             uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1,
-                                             uint32_t* words_out, uint32_t* M_out, int tid, int lane, int warp) {
-    unsigned char* slot = a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
+// (A real call, with plain values only: the sparse workloads' tile loop stays small.)  Returns words | M << 32.
+__device__ __noinline__ unsigned long long pack_tile_dense(CmpSmem* sp, unsigned char* dense_scratch, uint32_t a_l, uint32_t a_tau,
+                                                           uint32_t count, uint32_t warp_base, uint32_t m,
+                                                           uint32_t ex0, uint32_t ex1, uint32_t tot0, uint32_t tot1) {
+    CmpSmem& s = *sp;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned char* slot = dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes;
     uint32_t* vals = reinterpret_cast<uint32_t*>(slot);
     uint16_t* keys = reinterpret_cast<uint16_t*>(slot + (uint64_t)kTile * 4u);
     const float* tile = s.stage[0];
@@ -335,7 +337,7 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
 
     // ---- zero the words the blob can reach
     {
-        const uint32_t bound_words = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
+        const uint32_t bound_words = (count * (8u + a_l + (uint32_t)kGroupLog2) + 31u) >> 5;
         for (uint32_t i = tid; i < bound_words; i += kCmpThreads) blob[i] = 0u;
     }
     __syncthreads();
@@ -348,7 +350,7 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
         for (uint32_t j = tid; j < count; j += kCmpThreads) {
             const uint32_t key = keys[j];
             const uint32_t prev = j ? (uint32_t)keys[j - 1] : 0u;      // (the first delta of a group counts from 0)
-            blob_bytes[(j & ~3u) | (3u - (j & 3u))] = (uint8_t)code_byte_of(s.thr, a.tau, __uint_as_float(vals[j]));
+            blob_bytes[(j & ~3u) | (3u - (j & 3u))] = (uint8_t)code_byte_of(s.thr, a_tau, __uint_as_float(vals[j]));
             local_max = max(local_max, key - prev);
         }
         local_max = __reduce_max_sync(kFullMask, local_max);
@@ -360,16 +362,16 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
     const uint32_t maxd = s.max_delta;
     const uint32_t M = maxd ? (32u - __clz(maxd)) : 1u;
     const uint32_t inv_m = c_inv_m[M];
-    const uint32_t round_up = (1u << a.l) - 1u;
-    const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a.l * count;
+    const uint32_t round_up = (1u << a_l) - 1u;
+    const uint32_t flag_pos0 = 8u * count, delta_pos0 = flag_pos0 + a_l * count;
     uint32_t dbase = delta_pos0;
     for (uint32_t j0 = 0, round = 0; j0 < count; j0 += kCmpThreads, ++round) {
         const uint32_t j = j0 + (uint32_t)tid;
         uint32_t delta = 0, f = 0, w = 0;
         if (j < count) {
             delta = (uint32_t)keys[j] - (j ? (uint32_t)keys[j - 1] : 0u);
-            f = flag_of(delta, a.l, inv_m);
-            w = ((f + 1u) * M + round_up) >> a.l;
+            f = flag_of(delta, a_l, inv_m);
+            w = ((f + 1u) * M + round_up) >> a_l;
         }
         const uint32_t incl = warp_incl_scan(w, lane);
         if (lane == 31) s.scan_tot2[round & 1u][warp] = incl;
@@ -382,14 +384,13 @@ __device__ __forceinline__ void pack_tile_dense(CmpSmem& s, const CmpArgs& a, ui
             all += t;
         }
         if (j < count) {
-            put_bits_smem(blob, flag_pos0 + a.l * j, f, a.l);
+            put_bits_smem(blob, flag_pos0 + a_l * j, f, a_l);
             put_bits_smem(blob, dbase + before + (incl - w), delta, w);
         }
         dbase += all;
     }
     __syncthreads();      // blob complete
-    *words_out = (dbase + 31u) >> 5;
-    *M_out = M;
+    return (unsigned long long)((dbase + 31u) >> 5) | ((unsigned long long)M << 32);
 }
 
 // Running exclusive scan of the descriptors, kept by every block for itself.
@@ -1137,7 +1138,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     nprev = 0; npend = 0; arena_used = 0;
                 }
                 aoff = kDenseMark;
-                pack_tile_dense(s, a, count, warp_base, m, ex0, ex1, tot0, tot1, &words, &M, tid, lane, warp);
+                const unsigned long long wm = pack_tile_dense(&s, a.dense_scratch, a.l, a.tau, count, warp_base, m, ex0, ex1, tot0, tot1);
+                words = (uint32_t)wm; M = (uint32_t)(wm >> 32);
             }
             if (tid == 0) {
                 st_relaxed_u64(a.desc + g, desc_pack(kDescValid, count, words));
