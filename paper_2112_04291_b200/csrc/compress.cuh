@@ -448,15 +448,15 @@ __device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint
             outw[15] = a.G;
         }
     }
-    // a dense tile is always the last pending one when it is drained
-    if (npend > pbeg && s.pend_off[npend - 1] == kDenseMark) {
-        const int p = npend - 1;
+    // the blob of a tile that took the dense path (at most one is pending) waits in the block's slot of global scratch
+    for (int p = pbeg; p < npend; ++p) {
+        if (s.pend_off[p] != kDenseMark) continue;
         const uint32_t words = s.pend_words[p];
         const uint32_t off = fixed_words + (uint32_t)s.pend_prefix[p];
         const uint64_t end_bytes = ((uint64_t)off + words) << 2;
-        const uint32_t* blob = reinterpret_cast<const uint32_t*>(s.stage[0]);      // (still there: the caller refills the stage afterwards)
+        const uint32_t* blob = reinterpret_cast<const uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
         if (end_bytes <= a.out_bytes)
-            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(blob[i]);
+            for (uint32_t i = tid; i < words; i += kCmpThreads) outw[off + i] = bswap32(__ldcg(blob + i));
     }
 }
 
@@ -838,6 +838,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     // when their prefixes have long been published), tiles [nprev, npend) belong to this gradient.
     int nprev = 0, npend = 0;
     uint32_t arena_used = 0;
+    bool dense_pending = false;               // a blob of the dense path waits in the block's scratch slot
     CmpArgs a = job_view(b, 0u);
 
     if (step == 2u && team == 1u) {
@@ -1040,21 +1041,20 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     pending |= 1u << st;
                 }
                 if (tid == 0) {
-                    // (tiles too dense for the arena drain at once whatever is done)
-                    const bool stop_reserving = !overflow && worst_now <= kArenaWords / 4u &&
-                        (npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords);
+                    const bool stop_reserving = overflow || dense_pending ||
+                        npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords;
                     ticket_ahead = stop_reserving ? kNoTicket : atomicAdd(a.ticket, 1u);
                 }
             }
 
             uint32_t words = 0, M = 0, aoff = 0;
             if (count == 0u) {
-                if (npend == kPendMax) { if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; } nprev = 0; npend = 0; arena_used = 0; }
+                if (npend == kPendMax) { if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; } nprev = 0; npend = 0; arena_used = 0; dense_pending = false; }
             } else if (!overflow) {
                 const uint32_t worst = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
                 if (npend == kPendMax || arena_used + worst > kArenaWords) {
                     if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                    nprev = 0; npend = 0; arena_used = 0;
+                    nprev = 0; npend = 0; arena_used = 0; dense_pending = false;
                 }
                 aoff = arena_used;
                 uint32_t* blob = s.arena + aoff;
@@ -1132,14 +1132,29 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 }
                 arena_used += words;
             } else {
-                // a slab is too dense for its list: block-wide path, blob in the stage, placed at once
-                if (npend == kPendMax) {
+                // A slab is too dense for its list: block-wide path.  The blob is packed in the stage and
+                // moved to the block's slot of global scratch, where it waits like the blobs in the arena
+                // (one at a time; the block takes no new ticket while it holds one, so the drain that
+                // frees the slot never runs with a tile reserved).
+                if (dense_pending || npend == kPendMax) {
                     if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                    nprev = 0; npend = 0; arena_used = 0;
+                    nprev = 0; npend = 0; arena_used = 0; dense_pending = false;
                 }
                 aoff = kDenseMark;
                 const unsigned long long wm = pack_tile_dense(&s, a.dense_scratch, a.l, a.tau, count, warp_base, m, ex0, ex1, tot0, tot1);
                 words = (uint32_t)wm; M = (uint32_t)(wm >> 32);
+                {
+                    uint32_t* slot_blob = reinterpret_cast<uint32_t*>(a.dense_scratch + (uint64_t)blockIdx.x * kDenseScratchBytes);
+                    const uint32_t* stage_blob = reinterpret_cast<const uint32_t*>(s.stage[0]);
+                    for (uint32_t i2 = tid; i2 < words; i2 += kCmpThreads) slot_blob[i2] = stage_blob[i2];
+                }
+                dense_pending = true;
+                __syncthreads();                     // the stage is free
+                if (more) {                          // (generic-proxy writes before an async-proxy one)
+                    if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    issue_tile(s, a, st, g_next, tid);
+                    pending |= 1u << st;
+                }
             }
             if (tid == 0) {
                 st_relaxed_u64(a.desc + g, desc_pack(kDescValid, count, words));
@@ -1149,21 +1164,11 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 s.pend_off[npend] = aoff;
             }
             ++npend;
-            if (aoff == kDenseMark) {
-                __syncthreads();
-                if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                nprev = 0; npend = 0; arena_used = 0;
-                if (more) {                      // the stage is free now (generic-proxy writes before an async-proxy one)
-                    if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue_tile(s, a, st, g_next, tid);
-                    pending |= 1u << st;
-                }
-            }
             if (g_next == kNoTicket) {
                 // nothing reserved: drain now, then take the next ticket and start its copy
                 __syncthreads();
                 if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                nprev = 0; npend = 0; arena_used = 0;
+                nprev = 0; npend = 0; arena_used = 0; dense_pending = false;
                 if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
                 g = s.next_tile[par];
@@ -1207,6 +1212,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             if (tid < rest) { s.pend_g[tid] = e_g; s.pend_cm[tid] = e_cm; s.pend_words[tid] = e_w; s.pend_off[tid] = e_o; }
             __syncthreads();
             npend = rest;
+            dense_pending = false;
+            for (int p = 0; p < npend; ++p) dense_pending = dense_pending || s.pend_off[p] == kDenseMark;
         }
         nprev = npend;
         if (npend == 0) arena_used = 0;
