@@ -483,18 +483,16 @@ __device__ __forceinline__ void fetch_prefixes(CmpSmem& s, const CmpArgs& a, int
 // published scan.  Tiles [nprev, npend) belong to the gradient being encoded (view a, slot jp;
 // group numbers ascend): the block advances its own scan of the descriptors up to them.  Returns
 // false if a poisoned descriptor or a timeout was met (the caller aborts).
-__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, const CmpArgs& ap, uint32_t jp, int nprev, int npend,
-                                      int tid, int lane, int warp) {
-    if (npend == 0) return true;
+// First half (drain_wait): everything that may have to wait for other blocks; when it returns every
+// pending tile's prefix is known.  Second half (drain_place): the copies.
+__device__ __forceinline__ bool drain_wait(CmpSmem& s, const CmpArgs& a, const CmpArgs& ap, int nprev, int npend,
+                                           int tid, int lane, int warp) {
     if (tid == 0) s.poison_seen = 0u;
     __syncthreads();
     fetch_prefixes(s, ap, nprev, tid);
     if (npend == nprev) {
         __syncthreads();
-        if (s.poison_seen) return false;   // (rewritten only at the start of the next drain, behind a barrier)
-        place_pending(s, ap, jp ^ 1u, 0, nprev, tid, lane, warp);
-        __syncthreads();                   // the arena and the pending list are free again
-        return true;
+        return s.poison_seen == 0u;        // (rewritten only at the start of the next drain, behind a barrier)
     }
     ScanState sc; sc.pos = s.sc_pos; sc.count = s.sc_count; sc.words = s.sc_words;
     const uint32_t g_last = s.pend_g[npend - 1];
@@ -563,11 +561,22 @@ __device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, const CmpArg
     // the scan ran past g_last by whole steps: pull it back to g_last + 1
     // (descriptors beyond g_last were read as zero, so only the position needs correcting)
     sc.pos = g_last + 1u;
-    if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after the barrier below)
+    if (tid == 0) { s.sc_pos = sc.pos; s.sc_count = sc.count; s.sc_words = sc.words; }   // (read again after a later barrier)
+    return true;
+}
 
+__device__ __forceinline__ void drain_place(CmpSmem& s, const CmpArgs& a, const CmpArgs& ap, uint32_t jp, int nprev, int npend,
+                                            int tid, int lane, int warp) {
     place_pending(s, ap, jp ^ 1u, 0, nprev, tid, lane, warp);
     place_pending(s, a, jp, nprev, npend, tid, lane, warp);
     __syncthreads();                       // the arena and the pending list are free again
+}
+
+__device__ __forceinline__ bool drain(CmpSmem& s, const CmpArgs& a, const CmpArgs& ap, uint32_t jp, int nprev, int npend,
+                                      int tid, int lane, int warp) {
+    if (npend == 0) return true;
+    if (!drain_wait(s, a, ap, nprev, npend, tid, lane, warp)) return false;
+    drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
     return true;
 }
 
@@ -1165,10 +1174,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             }
             ++npend;
             if (g_next == kNoTicket) {
-                // nothing reserved: drain now, then take the next ticket and start its copy
+                // Nothing reserved: drain now.  Once the waiting half is over nobody can be held up by
+                // this block any more, so it takes its next ticket and starts that copy before it places its blobs.
                 __syncthreads();
-                if (!drain(s, a, ap, jp, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                nprev = 0; npend = 0; arena_used = 0; dense_pending = false;
+                if (npend > 0 && !drain_wait(s, a, ap, nprev, npend, tid, lane, warp)) { aborted = true; break; }
                 if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
                 __syncthreads();
                 g = s.next_tile[par];
@@ -1178,6 +1187,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     pending |= 1u << st;
                     if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
+                if (npend > 0) drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
+                nprev = 0; npend = 0; arena_used = 0; dense_pending = false;
                 __syncthreads();                   // next_tile[par] is rewritten two iterations from now at the earliest
             } else {
                 g = g_next;
