@@ -968,10 +968,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 if (slab_count <= kSlabCap) {
                     uint16_t* wk = s.wkeys[warp];
                     uint32_t* wv = s.wvals[warp];
-                    if (slab_count <= 64u) {
-                        // few entries: one round per kept entry of the lane that holds most
+                    if (slab_count <= 128u) {
+                        // up to 128 entries (measured): one round per kept entry of the lane that holds most
                         // (position = entries of earlier rows + entries of earlier lanes in the row + earlier ones of the lane in the row)
-                        const uint32_t t0 = tot0 + (tot0 << 8) + (tot0 << 16) + (tot0 << 24);      // inclusive prefix of the rows' totals, a byte per row (<= 64)
+                        const uint32_t t0 = tot0 + (tot0 << 8) + (tot0 << 16) + (tot0 << 24);      // inclusive prefix of the rows' totals, a byte per row (<= 128)
                         const uint32_t t1 = tot1 + (tot1 << 8) + (tot1 << 16) + (tot1 << 24) + (t0 >> 24) * 0x01010101u;
                         const unsigned long long rowex = ((unsigned long long)(t1 - tot1 + ex1) << 32) | (t0 - tot0 + ex0);   // exclusive row prefix + lanes before
                         uint32_t mm = m;
@@ -1117,7 +1117,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 uint32_t dbase = delta_pos0 + bits_before;
                 if ((uint32_t)lane < my_cnt) {
                     const uint32_t q = warp_base + lane;                  // rank of the entry in the group
-                    put_bits_smem(blob, 8u * q, wv[lane] & 0xFFu, 8u);
+                    put_byte_smem(blob, q, wv[lane] & 0xFFu);
                     put_bits_smem(blob, flag_pos0 + a.l * q, f0, a.l);
                     put_bits_smem(blob, dbase + (w0_incl - w0), d0, w0);
                 }
@@ -1133,7 +1133,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     const uint32_t w_incl = warp_incl_scan(w, lane);
                     if (j < my_cnt) {
                         const uint32_t q = warp_base + j;
-                        put_bits_smem(blob, 8u * q, wv[j] & 0xFFu, 8u);
+                        put_byte_smem(blob, q, wv[j] & 0xFFu);
                         put_bits_smem(blob, flag_pos0 + a.l * q, f, a.l);
                         put_bits_smem(blob, dbase + (w_incl - w), delta, w);
                     }
