@@ -73,7 +73,7 @@ typedef struct fastsgd_params {
 #define FASTSGD_ST_OK              0
 #define FASTSGD_ST_NONFINITE       1     /* compress: sum of |v| is Inf or NaN                               */
 #define FASTSGD_ST_CAPACITY        2     /* compress: stream does not fit in out_bytes                       */
-#define FASTSGD_ST_TIMEOUT         3     /* compress: a bounded wait between thread blocks ran out           */
+#define FASTSGD_ST_TIMEOUT         3     /* compress: a bounded wait between thread blocks ran out (see below) */
 #define FASTSGD_ST_BAD_MAGIC      16
 #define FASTSGD_ST_BAD_VERSION    17
 #define FASTSGD_ST_BAD_STATUS     18     /* decompress: the stream's own status is not OK                    */
@@ -102,6 +102,11 @@ typedef struct fastsgd_params {
  * If the stream does not fit, or the sum is not finite, only a 64-byte header
  * carrying the status is written.  Nothing outside out[0, out_bytes) is
  * written.
+ * The kernel is launched cooperatively (all its thread blocks resident at
+ * once, two per SM) and its blocks wait for one another with bounded waits; if
+ * one of them runs out (it should not on a GPU the kernel has to itself) every
+ * stream of that launch reports FASTSGD_ST_TIMEOUT, and the workspace must be
+ * registered again before the next call.
  */
 int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
                      void* out, uint64_t out_bytes, void* stream);
