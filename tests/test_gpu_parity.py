@@ -421,3 +421,70 @@ def test_damaged_stream_among_sound_ones_in_one_launch(keep_div):
         # the damaged group of the damaged stream is dropped as a whole; every other (group, stream) is applied
         assert np.array_equal(got[:lo], full[:lo]) and np.array_equal(got[hi:], full[hi:]), kind
         assert np.array_equal(got[lo:hi], good_only[lo:hi]), kind
+
+
+def _random_gradient(rng, n, kind):
+    if kind == 0:
+        return (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    if kind == 1:
+        return workloads.student_t_layers(n, seed=int(rng.integers(1 << 30)), blocks=int(rng.integers(1, 9)), lo=1e-4, hi=1e-1)
+    if kind == 2:          # mostly zeros with runs of non-zeros
+        v = np.zeros(n, np.float32)
+        for _ in range(int(rng.integers(1, 40))):
+            a = int(rng.integers(0, n))
+            b = min(n, a + int(rng.integers(1, 400)))
+            v[a:b] = rng.laplace(0.0, 1e-2, b - a).astype(np.float32)
+        return v
+    v = (rng.standard_normal(n) * 1e-3).astype(np.float32)          # a few huge entries, denormals and exact ties
+    idx = rng.integers(0, n, max(1, n // 50))
+    v[idx] *= np.float32(1e4)
+    v[rng.integers(0, n, max(1, n // 100))] = np.float32(1e-42)
+    v[rng.integers(0, n, max(1, n // 100))] = v[0]
+    return v
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_configurations_through_the_batched_calls(case):
+    # seeded random draws of size, parameters, value distribution, keep ratio and worker count; the
+    # batched calls must give the oracle's streams byte for byte and the oracle's accumulated vector
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(1000 + case)
+    tiles = int(rng.choice([1, 2, 3, 7, 20, 41, 310, 345]))
+    n = max(1, tiles * 16384 - int(rng.integers(0, 16384)))
+    workers = int(rng.integers(1, 6))
+    l = int(rng.integers(1, 6))
+    tau = int(rng.choice([1, 2, 5, 17, 64, 127, 128]))
+    kind = int(rng.integers(0, 4))
+    grads = [_random_gradient(rng, n, kind) for _ in range(workers)]
+    if workers > 2 and case % 3 == 0:
+        grads[1] = np.zeros(n, np.float32)
+    keep = float(rng.choice([0.0005, 0.005, 0.03, 0.2, 0.7]))
+    ref = grads[0] if np.count_nonzero(grads[0]) else grads[-1]
+    kth = max(1, min(int(np.count_nonzero(ref)), int(keep * n)))
+    base = workloads.base_for_keep(ref, kth, tau)
+    pg, po = binding.params(base, tau, l, 14), oracle.params(base, tau, l, 14)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    dg = [G.to_dev(v) for v in grads]
+    bufs = [G.Guarded(cap, fill=0x77) for _ in range(workers)]
+    assert binding.compress_batch(dg, pg, [b.view for b in bufs]) == 0
+    dense0 = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    odense = dense0.copy()
+    sizes = []
+    for w in range(workers):
+        total, d, status = binding.stream_info(bufs[w].view)
+        orc, ostream = oracle.compress(grads[w], po)
+        assert status == orc and bufs[w].intact(), (case, w, status, orc)
+        assert total == ostream.size and np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream), (case, w)
+        sizes.append(total)
+        if orc == 0:
+            assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+    if all(binding.stream_info(b.view)[2] == 0 for b in bufs):
+        buf = G.Guarded(4 * n)
+        dense = buf.view.view(torch.float32)
+        dense.copy_(torch.from_numpy(dense0))
+        assert binding.decompress_accumulate_batch([b.view for b in bufs], sizes, n, pg, dense) == 0
+        assert binding.decode_status() == 0 and buf.intact()
+        got = dense.cpu().numpy()
+        assert np.allclose(got, odense, rtol=RTOL, atol=ATOL) and np.array_equal(got, odense), case
