@@ -56,7 +56,7 @@ constexpr uint64_t kJobTraceOffset = kQueueOffset + kQueueBytes;  // u64 [320 bl
 constexpr uint64_t kJobTraceBytes  = 320ull * 8ull * 8ull * 8ull;
 constexpr uint64_t kSmSlotOffset   = kJobTraceOffset + kJobTraceBytes;  // u32 [256]: blocks of the running launch seen on each SM (zero between launches)
 constexpr uint64_t kSmSlotBytes    = 1024;
-constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]
+constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]; then float tmax[G]
 
 struct WorkspaceView {
     Control*            ctl;
@@ -64,6 +64,7 @@ struct WorkspaceView {
     double*             partials;
     unsigned long long* desc;
     unsigned long long* prefix;
+    float*              tmax;
 };
 
 __host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }

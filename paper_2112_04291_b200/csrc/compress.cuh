@@ -52,6 +52,7 @@ struct CmpSmem {
     float    stage[kStages][kTile];
     unsigned long long mbar[kStages];
     double   s_warp[2][kCmpWarps];
+    uint32_t s_wmax[2][kCmpWarps];           // sum pass: the slabs' largest |v| (bits of a non-negative float)
     double   s_tree[kCmpWarps];
     unsigned long long scan64[kDrainChunks][kCmpWarps];
     float    thr[132];
@@ -73,6 +74,7 @@ struct CmpSmem {
     uint32_t poison_seen;
     uint32_t pad;
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
+    uint32_t next_empty[2];                  // ... and whether its largest |v| is below the threshold (it is not read then)
     uint32_t held[2];                        // tiles this block has taken and not yet published (for the give-up path)
     uint32_t sc_pos, sc_count, sc_words;     // running exclusive scan of the descriptors: [0, pos) included
     uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
@@ -102,6 +104,7 @@ struct CmpArgs {
     double*             partials;
     unsigned long long* desc;
     unsigned long long* prefix;          // exclusive scan of desc, written by the last block to finish the encode pass
+    float*              tmax;            // largest |v| of each tile, from the sum pass: the encode pass does not read tiles below the threshold
     unsigned int*       enc_done;        // blocks that have finished this gradient's encode pass
     unsigned char*      dense_scratch;
     double              base;
@@ -122,6 +125,7 @@ struct CmpBatch {
     double*             partials;        // [jobs][G]
     unsigned long long* desc;            // [jobs][G]
     unsigned long long* prefix;          // [jobs][G]
+    float*              tmax;            // [jobs][G]
     unsigned int*       sm_slots;        // [256] blocks of this launch per SM
     unsigned char*      dense_scratch;
     double              base;
@@ -140,6 +144,7 @@ __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
     a.partials = b.partials + (uint64_t)w * b.G;
     a.desc = b.desc + (uint64_t)w * b.G;
     a.prefix = b.prefix + (uint64_t)w * b.G;
+    a.tmax = b.tmax + (uint64_t)w * b.G;
     a.enc_done = b.ctl->enc_done + w;
     a.dense_scratch = b.dense_scratch; a.base = b.base; a.G = b.G; a.tau = b.tau; a.l = b.l;
     return a;
@@ -695,11 +700,17 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         parity ^= 1u;
         pending &= ~1u;
         double x[8];
+        float mx = 0.0f;
         const float4* row = reinterpret_cast<const float4*>(&s.stage[0][warp * 1024]) + lane;
 #pragma unroll
-        for (int r = 0; r < 8; ++r) x[r] = abs_sum4(row[r * 32]);
+        for (int r = 0; r < 8; ++r) {
+            const float4 v4 = row[r * 32];
+            x[r] = abs_sum4(v4);
+            mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v4.x), fabsf(v4.y)), fmaxf(fabsf(v4.z), fabsf(v4.w))));
+        }
         const double u = warp_slab_tree(x, lane);
-        if (lane == 0) s.s_warp[q & 1][warp] = u;
+        const uint32_t wmx = __reduce_max_sync(kFullMask, __float_as_uint(mx));     // (non-negative floats order like their bits; a NaN shows in the sum)
+        if (lane == 0) { s.s_warp[q & 1][warp] = u; s.s_wmax[q & 1][warp] = wmx; }
         if (tid == 0)                                 // the tile after this one: a ticketed tile, then (one gradient) c, then none
             s.p1_next[(q + 1) & 1] = q + 1u >= limit ? kNoTicket
                                      : full ? (tk < a.G ? tk : kNoTicket)
@@ -709,7 +720,8 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         if (warp == 0) {
             double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
             t = warp_tree(t, kCmpWarps);
-            if (lane == 0) a.partials[tile] = t;
+            const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? s.s_wmax[q & 1][lane] : 0u);
+            if (lane == 0) { a.partials[tile] = t; a.tmax[tile] = __uint_as_float(tm); }
         }
         const uint32_t nxt = s.p1_next[(q + 1) & 1];
         if (nxt == kNoTicket) break;
@@ -897,23 +909,30 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     if (!aborted) {
         // the block's first tile of the encode pass: with one gradient its own tile c, still there from
         // the sum pass; otherwise the first ticket it gets
+        const uint32_t skip = s.job_skip[jp];
+        const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
+        // A tile whose largest |v| (recorded by the sum pass) is below the threshold holds nothing to
+        // keep: it goes through the loop as an empty tile without being read again.
         const bool preloaded = full;
         uint32_t g = c;
-        bool have = true;
+        bool have = true, cur_empty = false;
         if (full) {
-            if (tid == 0) s.next_tile[1] = atomicAdd(a.ticket, 1u);
+            if (tid == 0) {
+                const uint32_t t0 = atomicAdd(a.ticket, 1u);
+                s.next_tile[1] = t0;
+                s.next_empty[1] = (t0 < a.G && (skip != 0u || __ldcg(a.tmax + t0) < thr_e)) ? 1u : 0u;
+            }
             __syncthreads();
             g = s.next_tile[1];
+            cur_empty = s.next_empty[1] != 0u;
             have = g < a.G;
-            if (have) {
+            if (have && !cur_empty) {
                 issue_tile(s, a, 0, g, tid);
                 pending |= 1u;
             }
         }
         const CmpArgs ap = job_view(b, prev_job);
         if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
-        const uint32_t skip = s.job_skip[jp];
-        const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
 
         // =============================== phase 2: encode ===============================
         // Tile i of this block sits in stage (k-1-(i%kStages))%kStages; the last ones of phase 1 are
@@ -931,7 +950,11 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         for (uint32_t i = 0; have && !aborted; ++i) {
             const int st = 0;
             const uint32_t par = i & 1u;
-            if (i > 0u || preloaded) {
+            // thread 0: is the tile after the next one worth reading?  (its ticket came back an iteration ago;
+            // the answer is needed before this iteration's first barrier)
+            uint32_t ahead_empty = 0u;
+            if (tid == 0 && ticket_ahead < a.G) ahead_empty = (skip != 0u || __ldcg(a.tmax + ticket_ahead) < thr_e) ? 1u : 0u;
+            if ((i > 0u || preloaded) && !cur_empty) {
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
@@ -939,7 +962,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c
             const float* tile = s.stage[st];
             uint32_t m = 0;
-            if (!skip) {
+            if (!skip && !cur_empty) {
                 const float4* row = reinterpret_cast<const float4*>(tile + warp * 1024) + lane;
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
@@ -1013,7 +1036,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     slab_last = wk[slab_count - 1];
                 }
             }
-            if (tid == 0) { s.next_tile[par] = ticket_ahead; s.held[0] = g; s.held[1] = ticket_ahead; }
+            if (tid == 0) { s.next_tile[par] = ticket_ahead; s.next_empty[par] = ahead_empty; s.held[0] = g; s.held[1] = ticket_ahead; }
             if (lane == 0) {
                 s.sum_count[par][warp] = slab_count | (slab_count > kSlabCap ? 0x80000000u : 0u);
                 s.sum_first[par][warp] = slab_first;
@@ -1043,9 +1066,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // then takes its next ticket.
             const uint32_t worst_now = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
             const uint32_t g_next = s.next_tile[par];
+            const bool next_empty = s.next_empty[par] != 0u;
             const bool more = g_next < a.G;                  // (false for kNoTicket too)
             if (more) {
-                if (!overflow) {                 // (a tile too dense for the lists packs its blob in the stage first)
+                if (!overflow && !next_empty) {  // (a tile too dense for the lists packs its blob in the stage first)
                     issue_tile(s, a, st, g_next, tid);
                     pending |= 1u << st;
                 }
@@ -1159,7 +1183,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 }
                 dense_pending = true;
                 __syncthreads();                     // the stage is free
-                if (more) {                          // (generic-proxy writes before an async-proxy one)
+                if (more && !next_empty) {           // (generic-proxy writes before an async-proxy one)
                     if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     issue_tile(s, a, st, g_next, tid);
                     pending |= 1u << st;
@@ -1178,13 +1202,20 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 // this block any more, so it takes its next ticket and starts that copy before it places its blobs.
                 __syncthreads();
                 if (npend > 0 && !drain_wait(s, a, ap, nprev, npend, tid, lane, warp)) { aborted = true; break; }
-                if (tid == 0) s.next_tile[par] = atomicAdd(a.ticket, 1u);
+                if (tid == 0) {
+                    const uint32_t t1 = atomicAdd(a.ticket, 1u);
+                    s.next_tile[par] = t1;
+                    s.next_empty[par] = (t1 < a.G && (skip != 0u || __ldcg(a.tmax + t1) < thr_e)) ? 1u : 0u;
+                }
                 __syncthreads();
                 g = s.next_tile[par];
+                cur_empty = s.next_empty[par] != 0u;
                 have = g < a.G;
                 if (have) {
-                    issue_tile(s, a, st, g, tid);
-                    pending |= 1u << st;
+                    if (!cur_empty) {
+                        issue_tile(s, a, st, g, tid);
+                        pending |= 1u << st;
+                    }
                     if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
                 if (npend > 0) drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
@@ -1193,6 +1224,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             } else {
                 g = g_next;
                 have = more;
+                cur_empty = next_empty;
             }
         }
         if (tid == 0) btrace[8u * job + 5] = read_globaltimer();
