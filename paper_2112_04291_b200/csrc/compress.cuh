@@ -50,9 +50,9 @@ constexpr unsigned long long kDescValid = 1ull;               // status of a pub
 
 struct CmpSmem {
     float    stage[kStages][kTile];
-    unsigned long long mbar[kStages];
-    double   s_warp[2][kCmpWarps];
-    uint32_t s_wmax[2][kCmpWarps];           // sum pass: the slabs' largest |v| (bits of a non-negative float)
+    unsigned long long mbar[2];              // [0]: the whole tile (encode pass) or its first half (sum pass); [1]: its second half (sum pass)
+    double   s_warp[2][2][kCmpWarps];        // sum pass, by tile parity and half: the warps' tree nodes (512 entries each)
+    uint32_t s_wmax[2][2][kCmpWarps];        // ... and largest |v| (bits of a non-negative float)
     double   s_tree[kCmpWarps];
     unsigned long long scan64[kDrainChunks][kCmpWarps];
     float    thr[132];
@@ -220,6 +220,31 @@ __device__ __forceinline__ void issue_tile(CmpSmem& s, const CmpArgs& a, int sta
     if (valid < kTile) {                                             // block-uniform
         for (uint32_t i = (bulk_bytes >> 2) + tid; i < kTile; i += kCmpThreads)
             s.stage[stage][i] = i < valid ? __ldg(a.grad + e0 + i) : 0.0f;
+        __syncthreads();
+        // these were generic-proxy writes to a buffer that a later bulk copy (async proxy) overwrites
+        if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+}
+
+// Starts the copy of one half (8192 entries) of a tile into its half of the stage, signalling mbar[part].
+// Entries beyond n are zero (written by the threads themselves; block-wide call).
+__device__ __forceinline__ void issue_half(CmpSmem& s, const CmpArgs& a, uint32_t tile, int part, int tid) {
+    constexpr uint32_t kHalf = kTile / 2u;
+    const uint64_t e0 = ((uint64_t)tile << kGroupLog2) + (uint64_t)part * kHalf;
+    const uint64_t valid = e0 < a.n ? min((uint64_t)kHalf, a.n - e0) : 0ull;
+    const uint32_t bulk_bytes = (uint32_t)(valid * 4u) & ~15u;
+    float* dst = &s.stage[0][part * kHalf];
+    if (tid == 0) {
+        if (bulk_bytes) {
+            mbar_expect_tx(&s.mbar[part], bulk_bytes);
+            bulk_load(dst, a.grad + e0, bulk_bytes, &s.mbar[part]);
+        } else {
+            mbar_arrive(&s.mbar[part]);
+        }
+    }
+    if (valid < kHalf) {                                             // block-uniform
+        for (uint32_t i = (bulk_bytes >> 2) + tid; i < kHalf; i += kCmpThreads)
+            dst[i] = i < valid ? __ldg(a.grad + e0 + i) : 0.0f;
         __syncthreads();
         // these were generic-proxy writes to a buffer that a later bulk copy (async proxy) overwrites
         if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -681,54 +706,83 @@ __device__ __forceinline__ SumCursor sum_begin(CmpSmem& s, const CmpArgs& a, uin
     __syncthreads();
     cur.tile = s.p1_next[0];
     if (cur.tile != kNoTicket) {
-        issue_tile(s, a, 0, cur.tile, tid);
-        pending |= 1u;
+        issue_half(s, a, cur.tile, 0, tid);
+        issue_half(s, a, cur.tile, 1, tid);
+        pending |= 3u;
         if (tid == 0 && limit > 1u && (full || cur.tile != c)) cur.tk = atomicAdd(a.ctl->tickets1 + job, 1u);
     }
     return cur;
 }
 
+// The tile goes through the stage in two halves with a barrier each: as soon as the block has read
+// a half it starts the copy of the same half of its next tile, so that one copy is in flight while
+// the other half is being summed.  Warp w sums entries [512 w, 512 w + 512) of the half; the tile's
+// node is that of the first half plus that of the second (the same fixed tree as everywhere).
 __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t c, uint32_t grid,
                                          uint32_t limit, SumCursor cur, uint32_t& parity, uint32_t& pending,
                                          int tid, int lane, int warp) {
     unsigned int tk = cur.tk;
     uint32_t tile = cur.tile;
     if (tile == kNoTicket) return;                    // (several gradients, fewer tiles than blocks)
-    for (uint32_t q = 0;; ++q) {
-        if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }   // phase 2's descriptors and prefixes (ordered by the grid barrier)
-        if (!mbar_wait(&s.mbar[0], parity & 1u)) s.abort_flag = 1u;
-        parity ^= 1u;
-        pending &= ~1u;
-        double x[8];
-        float mx = 0.0f;
-        const float4* row = reinterpret_cast<const float4*>(&s.stage[0][warp * 1024]) + lane;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-            const float4 v4 = row[r * 32];
-            x[r] = abs_sum4(v4);
-            mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v4.x), fabsf(v4.y)), fmaxf(fabsf(v4.z), fabsf(v4.w))));
-        }
-        const double u = warp_slab_tree(x, lane);
-        const uint32_t wmx = __reduce_max_sync(kFullMask, __float_as_uint(mx));     // (non-negative floats order like their bits; a NaN shows in the sum)
-        if (lane == 0) { s.s_warp[q & 1][warp] = u; s.s_wmax[q & 1][warp] = wmx; }
-        if (tid == 0)                                 // the tile after this one: a ticketed tile, then (one gradient) c, then none
+    uint32_t prev_tile = kNoTicket;                   // its halves' nodes wait in s_warp[(q - 1) & 1]
+    uint32_t q = 0;
+    for (;; ++q) {
+        const uint32_t qp = q & 1u;
+        if (tid == 0) {
+            a.desc[tile] = 0ull; a.prefix[tile] = 0ull;   // phase 2's descriptors and prefixes (ordered by the grid barrier)
+            // the tile after this one: a ticketed tile, then (one gradient) c, then none
             s.p1_next[(q + 1) & 1] = q + 1u >= limit ? kNoTicket
                                      : full ? (tk < a.G ? tk : kNoTicket)
                                             : (tile == c ? kNoTicket : (grid + tk < a.G ? a.G - 1u - tk : c));
-        __syncthreads();
-        if (s.abort_flag) break;
-        if (warp == 0) {
-            double t = lane < kCmpWarps ? s.s_warp[q & 1][lane] : 0.0;
-            t = warp_tree(t, kCmpWarps);
-            const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? s.s_wmax[q & 1][lane] : 0u);
-            if (lane == 0) { a.partials[tile] = t; a.tmax[tile] = __uint_as_float(tm); }
         }
-        const uint32_t nxt = s.p1_next[(q + 1) & 1];
+        uint32_t nxt = kNoTicket;
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            if (!mbar_wait(&s.mbar[part], (parity >> part) & 1u)) s.abort_flag = 1u;
+            parity ^= 1u << part;
+            pending &= ~(1u << part);
+            double x[4];
+            float mx = 0.0f;
+            const float4* row = reinterpret_cast<const float4*>(&s.stage[0][part * (int)(kTile / 2) + warp * 512]) + lane;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float4 v4 = row[r * 32];
+                x[r] = abs_sum4(v4);
+                mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v4.x), fabsf(v4.y)), fmaxf(fabsf(v4.z), fabsf(v4.w))));
+            }
+            __syncthreads();                          // the half has been read (and p1_next is visible)
+            if (s.abort_flag) return;
+            if (part == 0) nxt = s.p1_next[(q + 1) & 1];
+            if (nxt != kNoTicket) {                   // (with one gradient the last tile, c, stays in the stage)
+                issue_half(s, a, nxt, part, tid);
+                pending |= 1u << part;
+            }
+            const double u = warp_halfslab_tree(x, lane);
+            const uint32_t wmx = __reduce_max_sync(kFullMask, __float_as_uint(mx));     // (non-negative floats order like their bits; a NaN shows in the sum)
+            if (lane == 0) { s.s_warp[qp][part][warp] = u; s.s_wmax[qp][part][warp] = wmx; }
+            if (part == 0 && warp == 0 && prev_tile != kNoTicket) {
+                // the tile before this one: both of its halves' nodes are complete since the barrier above
+                double t0 = lane < kCmpWarps ? s.s_warp[qp ^ 1u][0][lane] : 0.0, t1 = lane < kCmpWarps ? s.s_warp[qp ^ 1u][1][lane] : 0.0;
+                t0 = warp_tree(t0, kCmpWarps);
+                t1 = warp_tree(t1, kCmpWarps);
+                const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? max(s.s_wmax[qp ^ 1u][0][lane], s.s_wmax[qp ^ 1u][1][lane]) : 0u);
+                if (lane == 0) { a.partials[prev_tile] = __dadd_rn(t0, t1); a.tmax[prev_tile] = __uint_as_float(tm); }
+            }
+        }
+        prev_tile = tile;
         if (nxt == kNoTicket) break;
-        issue_tile(s, a, 0, nxt, tid);
-        pending |= 1u;
         if (tid == 0 && q + 2u < limit && (full || nxt != c)) tk = atomicAdd(a.ctl->tickets1 + job, 1u);
         tile = nxt;
+    }
+    // the last tile's nodes
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t qp = q & 1u;
+        double t0 = lane < kCmpWarps ? s.s_warp[qp][0][lane] : 0.0, t1 = lane < kCmpWarps ? s.s_warp[qp][1][lane] : 0.0;
+        t0 = warp_tree(t0, kCmpWarps);
+        t1 = warp_tree(t1, kCmpWarps);
+        const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? max(s.s_wmax[qp][0][lane], s.s_wmax[qp][1][lane]) : 0u);
+        if (lane == 0) { a.partials[prev_tile] = __dadd_rn(t0, t1); a.tmax[prev_tile] = __uint_as_float(tm); }
     }
 }
 
@@ -825,7 +879,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     unsigned int gen_next = 0u;
     if (tid == 0) {
         gen_next = ld_acquire_u32(&b.ctl->bar_gen) + 1u;      // before this block can arrive at a barrier
-        for (int st = 0; st < kStages; ++st) mbar_init(&s.mbar[st], 1u);
+        for (int st = 0; st < 2; ++st) mbar_init(&s.mbar[st], 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s.abort_flag = 0u;
         s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
@@ -1279,7 +1333,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // (in the sum pass nobody waits for descriptors yet)
             if (s.held[0] < a.G) st_relaxed_u64(a.desc + s.held[0], desc_pack(kDescPoison, 0, 0));
             if (s.held[1] < a.G) st_relaxed_u64(a.desc + s.held[1], desc_pack(kDescPoison, 0, 0));
-            for (int st = 0; st < kStages; ++st)
+            for (int st = 0; st < 2; ++st)
                 if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
             // every stream of the launch reports the timeout (identical words from every block that gives up)
             for (uint32_t w = 0; w < b.jobs; ++w) {

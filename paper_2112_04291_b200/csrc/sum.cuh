@@ -57,6 +57,28 @@ __device__ __forceinline__ double warp_slab_tree(const double (&x)[8], int lane)
     return u;
 }
 
+// The same for half a slab: x[r] = tree node of this lane's 4 entries in row r of 4 consecutive rows.
+// Returns, in every lane, the tree node of the 512 entries.
+__device__ __forceinline__ double warp_halfslab_tree(const double (&x)[4], int lane) {
+    const bool b0 = lane & 1, b1 = lane & 2;
+    double y[2], z, u;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {   // lanes 2k,2k+1: 8 entries of row i (even lane) / i+2 (odd lane)
+        double keep = b0 ? x[i + 2] : x[i], send = b0 ? x[i] : x[i + 2];
+        y[i] = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 1));
+    }
+    {                               // 16 entries of row b1 + 2*b0
+        double keep = b1 ? y[1] : y[0], send = b1 ? y[0] : y[1];
+        z = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 2));
+    }
+    u = __dadd_rn(z, __shfl_xor_sync(kFullMask, z, 4));    // 32 entries
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 8));    // 64 entries
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 16));   // the row (128)
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 2));    // rows 2k, 2k+1
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 1));    // 4 rows = 512 entries
+    return u;
+}
+
 // tree over the 32 lanes' values (lane = position)
 __device__ __forceinline__ double warp_tree(double u, int width = 32) {
     for (int o = 1; o < width; o <<= 1) u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, o));
