@@ -631,18 +631,20 @@ __device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32
 // for them.  A descriptor that is not valid (or never comes) poisons its own and every later prefix.
 template <bool POLL>
 __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, int tid, int lane, int warp) {
+    // (following the others, small steps: what is complete is published at once)
+    constexpr int kChunks = POLL ? 1 : kDrainChunks;
     unsigned long long running = 0ull;
     bool bad = false;
-    for (uint32_t pos = 0; pos < a.G; pos += (uint32_t)kDrainChunks * kCmpThreads) {
-        unsigned long long own[kDrainChunks], excl[kDrainChunks];
+    for (uint32_t pos = 0; pos < a.G; pos += (uint32_t)kChunks * kCmpThreads) {
+        unsigned long long own[kChunks], excl[kChunks];
         bool bad_here = false;
 #pragma unroll
-        for (int j = 0; j < kDrainChunks; ++j) {
+        for (int j = 0; j < kChunks; ++j) {
             const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
             own[j] = idx < a.G ? ld_relaxed_u64(a.desc + idx) : desc_pack(kDescValid, 0, 0);
         }
 #pragma unroll
-        for (int j = 0; j < kDrainChunks; ++j) {
+        for (int j = 0; j < kChunks; ++j) {
             if (POLL && !bad) {
                 const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
                 uint32_t spin = 0;
@@ -665,7 +667,7 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
         }
         if (__syncthreads_or(bad_here ? 1 : 0)) bad = true;
 #pragma unroll
-        for (int j = 0; j < kDrainChunks; ++j) {
+        for (int j = 0; j < kChunks; ++j) {
             unsigned long long before = running, all = 0ull;
 #pragma unroll
             for (int w = 0; w < kCmpWarps; ++w) {
