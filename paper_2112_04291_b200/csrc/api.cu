@@ -83,8 +83,9 @@ uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
 }
 
 uint64_t ws_dense_offset(uint64_t n, uint32_t group_log2) {
-    // partials, descriptors, prefixes and tile maxima for every gradient one launch can take
-    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 20ull * groups_of(n, group_log2));
+    // partials, descriptors, prefixes, tile maxima, the list of tiles to encode and its bitmap for every gradient one launch can take
+    const uint64_t G = groups_of(n, group_log2);
+    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 24ull * G + 4ull * ((G + 31ull) >> 5));
     return (b + 255ull) & ~255ull;
 }
 
@@ -101,6 +102,8 @@ WorkspaceView view(void* ws, uint64_t n) {
     v.desc = reinterpret_cast<unsigned long long*>(base + kPartialsOffset + (uint64_t)kCmpMaxJobs * 8ull * chunks_of(n));
     v.prefix = v.desc + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2);
     v.tmax = reinterpret_cast<float*>(v.prefix + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
+    v.nelist = reinterpret_cast<uint32_t*>(v.tmax + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
+    v.nebits = v.nelist + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2);
     return v;
 }
 
@@ -290,7 +293,7 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
             cb.grad[i] = grads[first + i];
             cb.out[i] = static_cast<uint8_t*>(outs[first + i]);
         }
-        cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc; cb.prefix = w.prefix; cb.tmax = w.tmax;
+        cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc; cb.prefix = w.prefix; cb.tmax = w.tmax; cb.nelist = w.nelist; cb.nebits = w.nebits;
         cb.sm_slots = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kSmSlotOffset);
         cb.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
         cb.base = params->base; cb.G = (uint32_t)G; cb.tau = params->tau; cb.l = params->flag_bits;

@@ -43,7 +43,7 @@ struct Control {
     unsigned int       enc_done[8];    // encode pass: blocks that have published all their tiles of each gradient (self-resetting)
     unsigned int       bar_count[8];   // blocks that have finished each gradient's sum pass (self-resetting)
     unsigned int       bar_flag[8];    // set to bar_gen + 1 by the last of them: that gradient's partial sums are complete
-    unsigned int       pad[8];
+    unsigned int       ne_count[8];    // tiles of each gradient the encode pass has to read (written before bar_flag)
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -56,7 +56,7 @@ constexpr uint64_t kJobTraceOffset = kQueueOffset + kQueueBytes;  // u64 [320 bl
 constexpr uint64_t kJobTraceBytes  = 320ull * 8ull * 8ull * 8ull;
 constexpr uint64_t kSmSlotOffset   = kJobTraceOffset + kJobTraceBytes;  // u32 [256]: blocks of the running launch seen on each SM (zero between launches)
 constexpr uint64_t kSmSlotBytes    = 1024;
-constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]; then float tmax[G]
+constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]; then float tmax[G]; then u32 nelist[G]; then u32 nebits[ceil(G / 32)]
 
 struct WorkspaceView {
     Control*            ctl;
@@ -65,6 +65,8 @@ struct WorkspaceView {
     unsigned long long* desc;
     unsigned long long* prefix;
     float*              tmax;
+    uint32_t*           nelist;
+    uint32_t*           nebits;
 };
 
 __host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }

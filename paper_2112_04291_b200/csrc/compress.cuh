@@ -41,6 +41,7 @@ constexpr uint32_t kMaxCtas      = 320;                       // scratch slots f
 constexpr uint32_t kWaitLimit    = 1u << 22;                  // polls before a wait gives up
 constexpr int      kDrainChunks  = 4;                         // descriptors read at once when draining: 4 x 512
 constexpr uint32_t kNoTicket     = 0xFFFFFFFEu;               // "no tile reserved": the block drains before it takes one
+constexpr uint32_t kNoMore       = 0xFFFFFFFDu;               // "no tile left": the gradient's list is exhausted
 constexpr uint32_t kDenseMark    = 0xFFFFFFFFu;               // arena offset of a blob that sits in global scratch
 // dense path scratch per block: values / blob u32[T] | keys u16[T] | codes u8[T]
 constexpr uint64_t kDenseScratchBytes = (uint64_t)kTile * 4u + (uint64_t)kTile * 2u + kTile;
@@ -74,7 +75,8 @@ struct CmpSmem {
     uint32_t poison_seen;
     uint32_t pad;
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
-    uint32_t next_empty[2];                  // ... and whether its largest |v| is below the threshold (it is not read then)
+    uint32_t ne_count;                       // tiles the gradient's encode pass hands out by ticket
+    uint32_t pad6;
     uint32_t held[2];                        // tiles this block has taken and not yet published (for the give-up path)
     uint32_t sc_pos, sc_count, sc_words;     // running exclusive scan of the descriptors: [0, pos) included
     uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
@@ -104,7 +106,9 @@ struct CmpArgs {
     double*             partials;
     unsigned long long* desc;
     unsigned long long* prefix;          // exclusive scan of desc, written by the last block to finish the encode pass
-    float*              tmax;            // largest |v| of each tile, from the sum pass: the encode pass does not read tiles below the threshold
+    float*              tmax;            // largest |v| of each tile, from the sum pass
+    uint32_t*           nelist;          // the tiles the encode pass reads, ascending: those whose largest |v| reaches the threshold
+    uint32_t*           nebits;          // the same as a bitmap (scratch of the block that builds the list)
     unsigned int*       enc_done;        // blocks that have finished this gradient's encode pass
     unsigned char*      dense_scratch;
     double              base;
@@ -126,6 +130,8 @@ struct CmpBatch {
     unsigned long long* desc;            // [jobs][G]
     unsigned long long* prefix;          // [jobs][G]
     float*              tmax;            // [jobs][G]
+    uint32_t*           nelist;          // [jobs][G]
+    uint32_t*           nebits;          // [jobs][ceil(G / 32)]
     unsigned int*       sm_slots;        // [256] blocks of this launch per SM
     unsigned char*      dense_scratch;
     double              base;
@@ -145,6 +151,8 @@ __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
     a.desc = b.desc + (uint64_t)w * b.G;
     a.prefix = b.prefix + (uint64_t)w * b.G;
     a.tmax = b.tmax + (uint64_t)w * b.G;
+    a.nelist = b.nelist + (uint64_t)w * b.G;
+    a.nebits = b.nebits + (uint64_t)w * ((b.G + 31u) >> 5);
     a.enc_done = b.ctl->enc_done + w;
     a.dense_scratch = b.dense_scratch; a.base = b.base; a.G = b.G; a.tau = b.tau; a.l = b.l;
     return a;
@@ -633,6 +641,8 @@ template <bool POLL>
 __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, int tid, int lane, int warp) {
     // (following the others, small steps: what is complete is published at once)
     constexpr int kChunks = POLL ? 1 : kDrainChunks;
+    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
+    uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
     unsigned long long running = 0ull;
     bool bad = false;
     for (uint32_t pos = 0; pos < a.G; pos += (uint32_t)kChunks * kCmpThreads) {
@@ -678,9 +688,15 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
             excl[j] += before;
             running += all;
             const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
-            if (idx < a.G)
+            if (idx < a.G) {
                 st_relaxed_u64(a.prefix + idx, bad ? desc_pack(kDescPoison, 0, 0)
                                                    : desc_pack(kDescValid, (uint32_t)(excl[j] >> 32), (uint32_t)excl[j]));
+                // a group without kept entries: its directory entry (most of these tiles were never read by the encode pass)
+                if (!bad && (own[j] >> 32) == 0ull) {
+                    outw[(kHeaderBytes >> 2) + 2u * idx]      = 0u;
+                    outw[(kHeaderBytes >> 2) + 2u * idx + 1u] = fixed_words + (uint32_t)excl[j];
+                }
+            }
         }
         __syncthreads();
     }
@@ -788,14 +804,73 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
     }
 }
 
+// Run by one block when a gradient's sum S is known: which tiles does the encode pass have to read?
+// A tile whose largest |v| (recorded by the sum pass) is below the early-stop threshold B_tau holds
+// nothing to keep.  Such a tile gets its descriptor (0 entries, 0 words) here; its directory entry
+// is written by the block that publishes the prefixes.  The others go into a.nelist in ascending
+// order, and the encode pass hands out positions of that list.  Tiles below first_ticketed are not
+// listed (with one gradient each block encodes its own tile, which it still holds); the last tile
+// is always listed, since whoever encodes it writes the header.  Returns the length of the list
+// (valid in thread 0).
+__device__ __forceinline__ uint32_t build_tile_list(CmpSmem& s, const CmpArgs& a, const PowTable& pw, double S, uint32_t first_ticketed,
+                                                    int tid, int lane, int warp) {
+    // the threshold exactly as the encode pass forms it
+    const float thr_e = isfinite(S) ? fmaxf(__double2float_ru(__ddiv_rn(S, pw.P[a.tau])), __int_as_float(1)) : __int_as_float(0x7f800000);
+    for (uint32_t base = 0; base < a.G; base += 4u * kCmpThreads) {
+        float tm[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t tile = base + (uint32_t)j * kCmpThreads + tid;
+            tm[j] = tile < a.G ? __ldcg(a.tmax + tile) : 0.0f;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t tile = base + (uint32_t)j * kCmpThreads + tid;
+            const bool ticketed = tile < a.G && tile >= first_ticketed;
+            const bool listed = ticketed && (!(tm[j] < thr_e) || tile == a.G - 1u);
+            if (ticketed && !listed) st_relaxed_u64(a.desc + tile, desc_pack(kDescValid, 0, 0));
+            const uint32_t word = __ballot_sync(kFullMask, listed);
+            if (lane == 0 && (tile - lane) < a.G) a.nebits[tile >> 5] = word;
+        }
+    }
+    __syncthreads();                                   // the bitmap is complete (same block: visible after the barrier)
+    const uint32_t nwords = (a.G + 31u) >> 5;
+    uint32_t running = 0;
+    for (uint32_t base = 0; base < nwords; base += kCmpThreads) {
+        const uint32_t wi = base + tid;
+        uint32_t word = wi < nwords ? __ldcg(a.nebits + wi) : 0u;
+        const uint32_t cnt = (uint32_t)__popc(word);
+        const uint32_t incl = warp_incl_scan(cnt, lane);
+        if (lane == 31) s.scan_tot[warp] = incl;
+        __syncthreads();
+        uint32_t before = running, all = 0;
+#pragma unroll
+        for (int w = 0; w < kCmpWarps; ++w) {
+            const uint32_t v = s.scan_tot[w];
+            if (w < warp) before += v;
+            all += v;
+        }
+        uint32_t pos = before + incl - cnt;
+        while (word) {
+            const uint32_t bit = (uint32_t)__ffs((int)word) - 1u;
+            word &= word - 1u;
+            a.nelist[pos++] = (wi << 5) + bit;
+        }
+        running += all;
+        __syncthreads();
+    }
+    return running;
+}
+
 // Grid barrier of gradient `job` among the `expect` blocks that sum it, first half: this
 // block's partial sums are written.  The last block to arrive reduces all partials on the fixed
 // tree (alone: hundreds of blocks reading the same few lines at once queue up in L2), stores S,
-// clears the count, readies the gradient's ticket counters (encode pass: with one gradient the
-// tiles below `tgrid` are taken; sum pass: zero for the next launch) and sets the gradient's flag
-// to the launch's generation (read by every block when it started, bumped by the last block to
-// leave the kernel: no state outside the workspace, so a launch can be replayed).
-__device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, uint32_t job, bool full, uint32_t tgrid,
+// lists the tiles the encode pass has to read (build_tile_list), clears the count, readies the
+// gradient's ticket counters and sets the gradient's flag to the launch's generation (read by
+// every block when it started, bumped by the last block to leave the kernel: no state outside
+// the workspace, so a launch can be replayed).  With one gradient the tiles below `tgrid` are
+// encoded by the blocks that summed them last and take no ticket.
+__device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, const PowTable& pw, uint32_t job, bool full, uint32_t tgrid,
                                                uint32_t expect, unsigned int gen_next, int tid, int lane, int warp) {
     Control* ctl = a.ctl;
     __syncthreads();
@@ -810,11 +885,13 @@ __device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, uin
     __syncthreads();
     if (s.last_arrival) {
         const double S = reduce_partials(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
+        const uint32_t listed = build_tile_list(s, a, pw, S, full ? 0u : tgrid, tid, lane, warp);      // (every thread holds S)
         if (tid == 0) {
             reinterpret_cast<double*>(reinterpret_cast<unsigned char*>(ctl) + kJobSumOffset)[job] = S;
             ctl->bar_count[job] = 0u;
-            ctl->tickets[job] = full ? 0u : tgrid;
+            ctl->tickets[job] = 0u;
             ctl->tickets1[job] = 0u;
+            ctl->ne_count[job] = listed;
             __threadfence();
             st_release_u32(&ctl->bar_flag[job], gen_next);
         }
@@ -851,6 +928,7 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
         s.thr[130] = (float)log2(S);                  // (only steer the table search)
         s.thr[131] = (float)(1.0 / log2(a.base));
         s.job_sum[jp] = S; s.job_skip[jp] = skip;
+        s.ne_count = __ldcg(&a.ctl->ne_count[job]);
         s.sc_pos = 0u; s.sc_count = 0u; s.sc_words = 0u;
         s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
     }
@@ -922,7 +1000,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[8u * 7u + 0] = read_globaltimer();
         const SumCursor cur = sum_begin(s, a, 0u, full, c, grid, 2u, pending, tid);
         sum_rest(s, a, 0u, full, c, grid, 2u, cur, parity, pending, tid, lane, warp);
-        barrier_arrive(s, a, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
+        barrier_arrive(s, a, pw, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
         __syncthreads();
     }
     if (nown) {
@@ -931,7 +1009,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
         sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
-        barrier_arrive(s, a, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
+        barrier_arrive(s, a, pw, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
     }
 
     for (uint32_t it = 0; it < niter && !aborted; ++it) {
@@ -952,7 +1030,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
         sum_rest(s, an, nj, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
-        barrier_arrive(s, an, nj, full, grid, grid, gen_next, tid, lane, warp);
+        barrier_arrive(s, an, pw, nj, full, grid, grid, gen_next, tid, lane, warp);
     } else {
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
@@ -967,22 +1045,21 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // the sum pass; otherwise the first ticket it gets
         const uint32_t skip = s.job_skip[jp];
         const float thr_e = s.thr[a.tau];          // early-stop threshold tau_e
-        // A tile whose largest |v| (recorded by the sum pass) is below the threshold holds nothing to
-        // keep: it goes through the loop as an empty tile without being read again.
+        // Tickets of the encode pass are positions in the gradient's list of tiles worth reading
+        // (build_tile_list); kNoMore stands for "the list is exhausted".
+        const uint32_t listed = s.ne_count;
         const bool preloaded = full;
         uint32_t g = c;
-        bool have = true, cur_empty = false;
+        bool have = true;
         if (full) {
             if (tid == 0) {
                 const uint32_t t0 = atomicAdd(a.ticket, 1u);
-                s.next_tile[1] = t0;
-                s.next_empty[1] = (t0 < a.G && (skip != 0u || __ldcg(a.tmax + t0) < thr_e)) ? 1u : 0u;
+                s.next_tile[1] = t0 < listed ? __ldcg(a.nelist + t0) : kNoMore;
             }
             __syncthreads();
             g = s.next_tile[1];
-            cur_empty = s.next_empty[1] != 0u;
             have = g < a.G;
-            if (have && !cur_empty) {
+            if (have) {
                 issue_tile(s, a, 0, g, tid);
                 pending |= 1u;
             }
@@ -1006,11 +1083,11 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         for (uint32_t i = 0; have && !aborted; ++i) {
             const int st = 0;
             const uint32_t par = i & 1u;
-            // thread 0: is the tile after the next one worth reading?  (its ticket came back an iteration ago;
-            // the answer is needed before this iteration's first barrier)
-            uint32_t ahead_empty = 0u;
-            if (tid == 0 && ticket_ahead < a.G) ahead_empty = (skip != 0u || __ldcg(a.tmax + ticket_ahead) < thr_e) ? 1u : 0u;
-            if ((i > 0u || preloaded) && !cur_empty) {
+            // thread 0: which tile does the ticket taken an iteration ago stand for?  (needed before this
+            // iteration's first barrier)
+            uint32_t tile_ahead = kNoMore;
+            if (tid == 0) tile_ahead = ticket_ahead == kNoTicket ? kNoTicket : (ticket_ahead < listed ? __ldcg(a.nelist + ticket_ahead) : kNoMore);
+            if (i > 0u || preloaded) {
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
@@ -1018,7 +1095,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // ---- threshold filter on the warp's slab: kept mask, bit 4r+c <-> entry warp*1024 + r*128 + lane*4 + c
             const float* tile = s.stage[st];
             uint32_t m = 0;
-            if (!skip && !cur_empty) {
+            if (!skip) {
                 const float4* row = reinterpret_cast<const float4*>(tile + warp * 1024) + lane;
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
@@ -1092,7 +1169,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                     slab_last = wk[slab_count - 1];
                 }
             }
-            if (tid == 0) { s.next_tile[par] = ticket_ahead; s.next_empty[par] = ahead_empty; s.held[0] = g; s.held[1] = ticket_ahead; }
+            if (tid == 0) { s.next_tile[par] = tile_ahead; s.held[0] = g; s.held[1] = tile_ahead; }
             if (lane == 0) {
                 s.sum_count[par][warp] = slab_count | (slab_count > kSlabCap ? 0x80000000u : 0u);
                 s.sum_first[par][warp] = slab_first;
@@ -1122,10 +1199,9 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // then takes its next ticket.
             const uint32_t worst_now = (count * (8u + a.l + (uint32_t)kGroupLog2) + 31u) >> 5;
             const uint32_t g_next = s.next_tile[par];
-            const bool next_empty = s.next_empty[par] != 0u;
             const bool more = g_next < a.G;                  // (false for kNoTicket too)
             if (more) {
-                if (!overflow && !next_empty) {  // (a tile too dense for the lists packs its blob in the stage first)
+                if (!overflow) {                 // (a tile too dense for the lists packs its blob in the stage first)
                     issue_tile(s, a, st, g_next, tid);
                     pending |= 1u << st;
                 }
@@ -1239,7 +1315,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 }
                 dense_pending = true;
                 __syncthreads();                     // the stage is free
-                if (more && !next_empty) {           // (generic-proxy writes before an async-proxy one)
+                if (more) {                          // (generic-proxy writes before an async-proxy one)
                     if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     issue_tile(s, a, st, g_next, tid);
                     pending |= 1u << st;
@@ -1260,18 +1336,14 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 if (npend > 0 && !drain_wait(s, a, ap, nprev, npend, tid, lane, warp)) { aborted = true; break; }
                 if (tid == 0) {
                     const uint32_t t1 = atomicAdd(a.ticket, 1u);
-                    s.next_tile[par] = t1;
-                    s.next_empty[par] = (t1 < a.G && (skip != 0u || __ldcg(a.tmax + t1) < thr_e)) ? 1u : 0u;
+                    s.next_tile[par] = t1 < listed ? __ldcg(a.nelist + t1) : kNoMore;
                 }
                 __syncthreads();
                 g = s.next_tile[par];
-                cur_empty = s.next_empty[par] != 0u;
                 have = g < a.G;
                 if (have) {
-                    if (!cur_empty) {
-                        issue_tile(s, a, st, g, tid);
-                        pending |= 1u << st;
-                    }
+                    issue_tile(s, a, st, g, tid);
+                    pending |= 1u << st;
                     if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
                 if (npend > 0) drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
@@ -1280,7 +1352,6 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             } else {
                 g = g_next;
                 have = more;
-                cur_empty = next_empty;
             }
         }
         if (tid == 0) btrace[8u * job + 5] = read_globaltimer();

@@ -488,3 +488,40 @@ def test_random_configurations_through_the_batched_calls(case):
         assert binding.decode_status() == 0 and buf.intact()
         got = dense.cpu().numpy()
         assert np.allclose(got, odense, rtol=RTOL, atol=ATOL) and np.array_equal(got, odense), case
+
+
+@pytest.mark.parametrize("workers", [1, 3])
+@pytest.mark.parametrize("tiles", [5, 345])
+def test_tiles_below_the_threshold_are_never_read_again(tiles, workers):
+    # the kept entries sit in a few tiles; every other tile is non-zero but stays below the early-stop
+    # threshold, so the encode pass lists only the hot tiles (and the last one, which carries the
+    # header); the first and the last tile are cold, one gradient has no hot tile at all
+    import gpu_util as G
+    n = tiles * 16384 - 5000
+    grads = []
+    for w in range(workers):
+        rng = np.random.default_rng(77 + 10 * tiles + w)
+        v = (rng.standard_normal(n) * 1e-6).astype(np.float32)
+        if w != 1:
+            hot = rng.choice(np.arange(1, tiles - 1), size=max(1, tiles // 9), replace=False)
+            for t in hot:
+                k = int(rng.integers(1, 3000))
+                idx = t * 16384 + rng.choice(16384, size=k, replace=False)
+                v[idx] = (rng.standard_normal(k) * 1e-1).astype(np.float32)
+        grads.append(v)
+    S = float(np.abs(grads[0].astype(np.float64)).sum())
+    base = float((S / 1e-3) ** (1.0 / 128.0))             # B_tau = 1e-3: far above the cold entries, below most hot ones
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    dg = [G.to_dev(v) for v in grads]
+    bufs = [G.Guarded(cap, fill=0xA7) for _ in range(workers)]
+    for rep in range(2):
+        assert binding.compress_batch(dg, pg, [b.view for b in bufs]) == 0
+        for w in range(workers):
+            total, d, status = binding.stream_info(bufs[w].view)
+            orc, ostream = oracle.compress(grads[w], po)
+            assert status == orc == 0 and total == ostream.size and bufs[w].intact()
+            assert np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream), (w, rep)
+            if w != 1:
+                assert 0 < d < n // 10
