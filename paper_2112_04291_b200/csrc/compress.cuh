@@ -205,6 +205,12 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// counter increment that publishes this thread's earlier writes and, for whoever comes last, makes the others' visible
+__device__ __forceinline__ unsigned int atom_add_acq_rel_u32(unsigned int* p, unsigned int v) {
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 __device__ __forceinline__ unsigned long long read_globaltimer() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -877,9 +883,8 @@ __device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, con
     if (tid == 0) {                                   // (thread 0 wrote the partials and cleared the descriptors itself)
         s.last_arrival = 0u;
         if (!s.abort_flag) {
-            __threadfence();
-            const unsigned int old = atomicAdd(&ctl->bar_count[job], 1u);
-            if (old == expect - 1u) { s.last_arrival = 1u; __threadfence(); }
+            const unsigned int old = atom_add_acq_rel_u32(&ctl->bar_count[job], 1u);
+            if (old == expect - 1u) s.last_arrival = 1u;
         }
     }
     __syncthreads();
@@ -892,8 +897,7 @@ __device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, con
             ctl->tickets[job] = 0u;
             ctl->tickets1[job] = 0u;
             ctl->ne_count[job] = listed;
-            __threadfence();
-            st_release_u32(&ctl->bar_flag[job], gen_next);
+            st_release_u32(&ctl->bar_flag[job], gen_next);       // (the other threads' list entries were written before a block barrier)
         }
     }
 }
@@ -906,7 +910,6 @@ __device__ __forceinline__ void barrier_wait(CmpSmem& s, Control* ctl, uint32_t 
             if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
             if (spin > 64u) __nanosleep(32);
         }
-        __threadfence();
     }
     __syncthreads();
 }
@@ -1360,9 +1363,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) {
             s.publisher = 0u;
             if (!aborted) {
-                __threadfence();                            // this block's descriptors before its count
-                const unsigned int old = atomicAdd(a.enc_done, 1u);
-                if (old == enc_expect - 1u) { *a.enc_done = 0u; __threadfence(); }
+                const unsigned int old = atom_add_acq_rel_u32(a.enc_done, 1u);      // this block's descriptors before its count
+                if (old == enc_expect - 1u) *a.enc_done = 0u;
                 // the launch's last gradient: the first block through follows the others; else the last one scans
                 s.publisher = (job == H ? old == 0u : old == enc_expect - 1u) ? 1u : 0u;
             }
@@ -1426,12 +1428,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
 
     // the last block to leave readies the workspace for the next launch
     if (tid == 0) {
-        __threadfence();
-        const unsigned int old = atomicAdd(&b.ctl->exit_count, 1u);
+        const unsigned int old = atom_add_acq_rel_u32(&b.ctl->exit_count, 1u);
         if (old == gridDim.x - 1u) {
             b.ctl->exit_count = 0u;
             if (b.teams == 2u) for (int i = 0; i < 256; ++i) b.sm_slots[i] = 0u;
-            __threadfence();
             st_release_u32(&b.ctl->bar_gen, gen_next);
         }
     }
