@@ -429,7 +429,7 @@ def main():
     dom = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else None
     # dram__bytes_read.sum + dram__bytes_write.sum of one k_compress launch, from the ncu capture of
     # this very workload summarised in profiles/k_compress_c2_4workers.md; other workloads: not captured
-    traffic = 826.3e6 if (dom == "k_compress" and args.workload == "c2" and args.n is None and args.workers is None
+    traffic = 583.7e6 if (dom == "k_compress" and args.workload == "c2" and args.n is None and args.workers is None
                           and args.keep is None) else None
     roofline = None
     if dom:
