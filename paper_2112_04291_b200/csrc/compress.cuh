@@ -1,26 +1,28 @@
-// The encoder as ONE persistent kernel (one thread block per SM, cooperative launch).
+// The encoder as ONE persistent kernel (two thread blocks per SM, cooperative launch) that takes up
+// to eight gradients of the same length.
 //
-// Phase 1 (Algorithm 1, first step): every block streams its tiles of 2^14 entries through a
-// three-stage ring of shared-memory buffers filled by bulk asynchronous copies (TMA, no
-// multicast) and reduces each tile on the fixed fp64 pairwise tree; one partial per tile.
-// Grid barrier (bounded wait).  Every block then reduces all partials in the same tree order,
-// so that each holds sum and the boundary table B_k = sum / b^k without a second hop.
-// Phase 2 (rest of Algorithm 1, Algorithm 2 per group): the block walks its tiles again in the
-// opposite order, so that the last three tiles of phase 1 are still in shared memory and are
-// not read from HBM a second time; the others arrive through the same ring while the block
-// filters, compacts, quantises, delta-encodes and bit-packs the tile at hand, every warp on its
-// own slab of 1024 entries, with two block barriers per non-empty tile.
+// Sum pass (Algorithm 1, first step): tiles of 2^14 entries, handed out by a ticket counter, go
+// through a 64 KiB shared-memory stage in two halves filled by bulk asynchronous copies (TMA, no
+// multicast): one half is summed while the other is in flight.  Each tile is reduced on the fixed
+// fp64 pairwise tree; one partial and the tile's largest |v| are left in the workspace.  Grid
+// barrier (bounded wait).  The last block to arrive reduces all partials in the same tree order,
+// stores the sum and lists the tiles whose largest |v| reaches the early-stop threshold.
+// Encode pass (rest of Algorithm 1, Algorithm 2 per group): blocks take the listed tiles by ticket
+// (the others hold nothing to keep and are not read again); the next tile's copy runs while the
+// block filters, compacts, quantises, delta-encodes and bit-packs the tile at hand, every warp on
+// its own slab of 1024 entries, with two block barriers per tile.
 //
 // Device-wide offsets.  A packed blob stays in a shared-memory arena and the tile's
 // (count, words) is published as a descriptor; no block waits for another while it packs.
-// When the arena fills up, and at the end, the block drains it: it brings its running
-// exclusive scan of all descriptors up to its pending tiles (block-wide shuffle scans over
-// 512 descriptors at a time, bounded polls for the ones not published yet), copies the blobs
-// to their places in the stream and writes their directory entries.  The block that owns the
-// lowest unpublished tile never waits for anything, so the scheme cannot deadlock provided all
-// blocks are resident (cooperative launch).  Every wait is bounded; when one runs out the block
-// records FASTSGD_ST_TIMEOUT, poisons its descriptors, waits (bounded) for its own copies in
-// flight and returns.
+// When the arena fills up the block drains it: it brings its running exclusive scan of all
+// descriptors up to its pending tiles (block-wide shuffle scans over 4 x 512 descriptors at a
+// time, bounded polls for the ones not published yet), copies the blobs to their places in the
+// stream and writes their directory entries.  A block never waits while it holds a reserved tile,
+// and the block that owns the lowest unpublished tile never waits for anything, so the scheme
+// cannot deadlock provided all blocks are resident (cooperative launch).  What is pending at the
+// end of a gradient's encode pass is placed from prefixes that one block computes for everybody.
+// Every wait is bounded; when one runs out the block records FASTSGD_ST_TIMEOUT, poisons its
+// descriptors, waits (bounded) for its own copies in flight and returns.
 #pragma once
 
 #include "common.cuh"
@@ -1070,16 +1072,16 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         const CmpArgs ap = job_view(b, prev_job);
         if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
 
-        // =============================== phase 2: encode ===============================
-        // Tile i of this block sits in stage (k-1-(i%kStages))%kStages; the last ones of phase 1 are
-        // already there.  Every warp owns one slab of 1024 consecutive entries of the tile: it
-        // filters it, compacts its kept entries into its own list, quantises them and forms their
-        // deltas without talking to the other warps; two block barriers per non-empty tile exchange
-        // the slab summaries (counts, boundary keys, largest delta -> M) and the payload bits.
+        // =============================== encode pass ===============================
+        // Every warp owns one slab of 1024 consecutive entries of the tile in the stage: it filters
+        // it, compacts its kept entries into its own list, quantises them and forms their deltas
+        // without talking to the other warps; two block barriers per tile exchange the slab
+        // summaries (counts, boundary keys, largest delta -> M) and the payload bits.
         const uint32_t round_up = (1u << a.l) - 1u;
-        // The block's first tile is the one it summed last (still in shared memory); every further tile
-        // is handed out by a ticket counter, so that blocks that met dense tiles take fewer.  Thread 0
-        // holds the ticket of the tile after the one at hand, taken a whole iteration before it is used.
+        // With one gradient the block's first tile is the one it summed last (still in shared memory);
+        // every further tile is handed out by a ticket counter, so that blocks that met dense tiles
+        // take fewer.  Thread 0 holds the ticket of the tile after the one at hand, taken a whole
+        // iteration before it is used.
         static_assert(kStages == 1, "the encode pass keeps one tile in flight per block");
         unsigned int ticket_ahead = 0u;
         if (tid == 0 && have) ticket_ahead = atomicAdd(a.ticket, 1u);
