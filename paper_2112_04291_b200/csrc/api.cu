@@ -118,11 +118,15 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_compress<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_compress<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
     int b1 = 0, b2 = 0, b3 = 0;
     {
         int b3b = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3, k_compress<false>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (b3b < b3) b3 = b3b;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<false, true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (b3b < b3) b3 = b3b;
     }
     g_state.cmp_blocks_per_sm = b3;
@@ -314,7 +318,7 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
         cudaError_t err;
         {
             LaunchTimer lt(1, st);
-            err = cudaLaunchCooperativeKernel(cb.jobs > 1u ? (const void*)k_compress<true> : (const void*)k_compress<false>, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
+            err = cudaLaunchCooperativeKernel(cb.jobs > 1u ? (const void*)k_compress<true> : (cb.G > kCmpBigTiles ? (const void*)k_compress<false, true> : (const void*)k_compress<false>), dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
                                               sizeof(CmpSmem), st);
         }
         if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }

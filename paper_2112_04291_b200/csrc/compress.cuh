@@ -96,6 +96,7 @@ struct CmpSmem {
 static_assert(sizeof(CmpSmem) <= 232448, "shared memory of one block on sm_100");
 
 constexpr int kCmpMaxJobs = 8;             // gradients (simulated workers) one launch can take
+constexpr uint32_t kCmpBigTiles = 8192;   // a single gradient with more tiles than this is compressed by the kernel variant for very many tiles
 
 // One gradient's view of the launch arguments.
 struct CmpArgs {
@@ -281,6 +282,11 @@ __device__ __forceinline__ double block_tree(double x, double* s_tree, int lane,
     return __shfl_sync(kFullMask, t, 0);
 }
 
+// BIG: with more than 8 passes a warp forms the node of a whole pass by itself (16 partials per lane,
+// all in flight at once; the same tree by the transposing shuffle pattern) and the warps take the
+// passes in turn.  (Only in the kernel variant for very many tiles: the tile loops of the others
+// have proved sensitive to every bit of extra code around them.)
+template <bool BIG>
 __device__ __forceinline__ double reduce_partials(const double* partials, uint32_t chunks, double* s_tree,
                                                   double* s_nodes, int tid, int lane, int warp) {
     const uint32_t passes = (chunks + kCmpThreads - 1) / kCmpThreads;       // <= 256 for n < 2^31
@@ -299,6 +305,18 @@ __device__ __forceinline__ double reduce_partials(const double* partials, uint32
                                    __dadd_rn(__dadd_rn(v[4], v[5]), __dadd_rn(v[6], v[7])));
         return block_tree(x, s_tree, lane, warp);
     }
+    if constexpr (BIG) {
+        for (uint32_t p = (uint32_t)warp; p < passes; p += kCmpWarps) {
+            double x[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const uint64_t idx = (uint64_t)p * kCmpThreads + 32u * (uint32_t)j + (uint32_t)lane;
+                x[j] = idx < chunks ? __ldcg(partials + idx) : 0.0;
+            }
+            const double node = warp_rows16_tree(x, lane);
+            if (lane == 0) s_nodes[p] = node;
+        }
+    } else {
     double next = (uint32_t)tid < chunks ? __ldcg(partials + tid) : 0.0;
     for (uint32_t p = 0; p < passes; ++p) {
         const double x = next;
@@ -306,6 +324,7 @@ __device__ __forceinline__ double reduce_partials(const double* partials, uint32
         next = (p + 1 < passes && idx < chunks) ? __ldcg(partials + idx) : 0.0;    // in flight during this pass
         const double node = block_tree(x, s_tree, lane, warp);
         if (tid == 0) s_nodes[p] = node;
+    }
     }
     __syncthreads();
     // the nodes of the passes, zero-padded to 512 positions, reduced on the same tree
@@ -645,10 +664,8 @@ __device__ __forceinline__ bool drain_final(CmpSmem& s, const CmpArgs& a, uint32
 // others' descriptors as they appear (bounded polls), so that the prefixes are complete right
 // after the last tile is published -- used for the launch's last gradient, where everybody waits
 // for them.  A descriptor that is not valid (or never comes) poisons its own and every later prefix.
-template <bool POLL>
+template <bool POLL, int kChunks>
 __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, int tid, int lane, int warp) {
-    // (following the others, small steps: what is complete is published at once)
-    constexpr int kChunks = POLL ? 1 : kDrainChunks;
     const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
     uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
     unsigned long long running = 0ull;
@@ -820,19 +837,21 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
 // listed (with one gradient each block encodes its own tile, which it still holds); the last tile
 // is always listed, since whoever encodes it writes the header.  Returns the length of the list
 // (valid in thread 0).
+template <bool BIG>
 __device__ __forceinline__ uint32_t build_tile_list(CmpSmem& s, const CmpArgs& a, const PowTable& pw, double S, uint32_t first_ticketed,
                                                     int tid, int lane, int warp) {
     // the threshold exactly as the encode pass forms it
     const float thr_e = isfinite(S) ? fmaxf(__double2float_ru(__ddiv_rn(S, pw.P[a.tau])), __int_as_float(1)) : __int_as_float(0x7f800000);
-    for (uint32_t base = 0; base < a.G; base += 4u * kCmpThreads) {
-        float tm[4];
+    constexpr int kInFlight = BIG ? 16 : 4;
+    for (uint32_t base = 0; base < a.G; base += (uint32_t)kInFlight * kCmpThreads) {
+        float tm[kInFlight];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kInFlight; ++j) {
             const uint32_t tile = base + (uint32_t)j * kCmpThreads + tid;
             tm[j] = tile < a.G ? __ldcg(a.tmax + tile) : 0.0f;
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kInFlight; ++j) {
             const uint32_t tile = base + (uint32_t)j * kCmpThreads + tid;
             const bool ticketed = tile < a.G && tile >= first_ticketed;
             const bool listed = ticketed && (!(tm[j] < thr_e) || tile == a.G - 1u);
@@ -859,10 +878,19 @@ __device__ __forceinline__ uint32_t build_tile_list(CmpSmem& s, const CmpArgs& a
             all += v;
         }
         uint32_t pos = before + incl - cnt;
-        while (word) {
-            const uint32_t bit = (uint32_t)__ffs((int)word) - 1u;
-            word &= word - 1u;
-            a.nelist[pos++] = (wi << 5) + bit;
+        if constexpr (BIG) {
+            // the warp writes the tiles of its 32 words one word at a time: consecutive list entries from consecutive lanes
+            for (int j = 0; j < 32; ++j) {
+                const uint32_t wj = __shfl_sync(kFullMask, word, j), pj = __shfl_sync(kFullMask, pos, j);
+                if ((wj >> lane) & 1u)
+                    a.nelist[pj + (uint32_t)__popc(wj & ((1u << lane) - 1u))] = ((base + 32u * (uint32_t)warp + (uint32_t)j) << 5) + (uint32_t)lane;
+            }
+        } else {
+            while (word) {
+                const uint32_t bit = (uint32_t)__ffs((int)word) - 1u;
+                word &= word - 1u;
+                a.nelist[pos++] = (wi << 5) + bit;
+            }
         }
         running += all;
         __syncthreads();
@@ -878,6 +906,7 @@ __device__ __forceinline__ uint32_t build_tile_list(CmpSmem& s, const CmpArgs& a
 // every block when it started, bumped by the last block to leave the kernel: no state outside
 // the workspace, so a launch can be replayed).  With one gradient the tiles below `tgrid` are
 // encoded by the blocks that summed them last and take no ticket.
+template <bool BIG>
 __device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, const PowTable& pw, uint32_t job, bool full, uint32_t tgrid,
                                                uint32_t expect, unsigned int gen_next, int tid, int lane, int warp) {
     Control* ctl = a.ctl;
@@ -891,8 +920,8 @@ __device__ __forceinline__ void barrier_arrive(CmpSmem& s, const CmpArgs& a, con
     }
     __syncthreads();
     if (s.last_arrival) {
-        const double S = reduce_partials(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
-        const uint32_t listed = build_tile_list(s, a, pw, S, full ? 0u : tgrid, tid, lane, warp);      // (every thread holds S)
+        const double S = reduce_partials<BIG>(a.partials, a.G, s.s_tree, s.s_nodes, tid, lane, warp);
+        const uint32_t listed = build_tile_list<BIG>(s, a, pw, S, full ? 0u : tgrid, tid, lane, warp);      // (every thread holds S)
         if (tid == 0) {
             reinterpret_cast<double*>(reinterpret_cast<unsigned char*>(ctl) + kJobSumOffset)[job] = S;
             ctl->bar_count[job] = 0u;
@@ -951,7 +980,10 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
 // block's last tile of the sum pass stays in shared memory for the encode pass.
 // SEVERAL: the launch holds more than one gradient (its own instantiation: the single-gradient
 // launch carries none of the team and pipelining code, and the other way round)
-template <bool SEVERAL>
+// BIG (one gradient only): the variant for gradients with very many tiles, where the steps that one
+// block does for everybody (reducing the partials, listing the tiles, scanning the descriptors) take
+// forms that cost less per tile and more to start with.
+template <bool SEVERAL, bool BIG = false>
 __global__ void __launch_bounds__(kCmpThreads, 2)
 k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
@@ -1005,7 +1037,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[8u * 7u + 0] = read_globaltimer();
         const SumCursor cur = sum_begin(s, a, 0u, full, c, grid, 2u, pending, tid);
         sum_rest(s, a, 0u, full, c, grid, 2u, cur, parity, pending, tid, lane, warp);
-        barrier_arrive(s, a, pw, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
+        barrier_arrive<BIG>(s, a, pw, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
         __syncthreads();
     }
     if (nown) {
@@ -1014,7 +1046,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
         sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
-        barrier_arrive(s, a, pw, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
+        barrier_arrive<BIG>(s, a, pw, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
     }
 
     for (uint32_t it = 0; it < niter && !aborted; ++it) {
@@ -1035,7 +1067,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
         sum_rest(s, an, nj, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
-        barrier_arrive(s, an, pw, nj, full, grid, grid, gen_next, tid, lane, warp);
+        barrier_arrive<BIG>(s, an, pw, nj, full, grid, grid, gen_next, tid, lane, warp);
     } else {
         barrier_wait(s, b.ctl, job, gen_next, tid);
         if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
@@ -1373,8 +1405,9 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         }
         __syncthreads();
         if (s.publisher) {
-            if (job == H) publish_prefixes<true>(s, a, tid, lane, warp);
-            else publish_prefixes<false>(s, a, tid, lane, warp);
+            // (following the others: small steps, so that what is complete is published at once; with very many tiles large steps)
+            if (job == H) publish_prefixes<true, BIG ? kDrainChunks : 1>(s, a, tid, lane, warp);
+            else publish_prefixes<false, kDrainChunks>(s, a, tid, lane, warp);
         }
         // place what the previous gradient left behind; what this one leaves waits for the next turn
         if (!aborted && nprev > 0) {

@@ -79,6 +79,38 @@ __device__ __forceinline__ double warp_halfslab_tree(const double (&x)[4], int l
     return u;
 }
 
+// x[j] = the value at position 32 j + lane of 512 consecutive positions (16 rows of 32).  Returns,
+// in every lane, the tree node of the 512 positions (rows first, then the rows pairwise).
+__device__ __forceinline__ double warp_rows16_tree(const double (&x)[16], int lane) {
+    const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4, b3 = lane & 8;
+    double y[8], z[4], w[2], u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {   // lanes 2k,2k+1: positions 2k,2k+1 of row i (even lane) / i+8 (odd lane)
+        double keep = b0 ? x[i + 8] : x[i], send = b0 ? x[i] : x[i + 8];
+        y[i] = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 1));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {   // 4 positions of row i + 4*b1 + 8*b0
+        double keep = b1 ? y[i + 4] : y[i], send = b1 ? y[i] : y[i + 4];
+        z[i] = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 2));
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {   // 8 positions of row i + 2*b2 + 4*b1 + 8*b0
+        double keep = b2 ? z[i + 2] : z[i], send = b2 ? z[i] : z[i + 2];
+        w[i] = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 4));
+    }
+    {                               // 16 positions of row b3 + 2*b2 + 4*b1 + 8*b0
+        double keep = b3 ? w[1] : w[0], send = b3 ? w[0] : w[1];
+        u = __dadd_rn(keep, __shfl_xor_sync(kFullMask, send, 8));
+    }
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 16));   // the row
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 8));    // rows 2k, 2k+1
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 4));    // 4 rows
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 2));    // 8 rows
+    u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, 1));    // 16 rows = 512 positions
+    return u;
+}
+
 // tree over the 32 lanes' values (lane = position)
 __device__ __forceinline__ double warp_tree(double u, int width = 32) {
     for (int o = 1; o < width; o <<= 1) u = __dadd_rn(u, __shfl_xor_sync(kFullMask, u, o));
