@@ -156,6 +156,46 @@ int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uin
                                         uint32_t num_streams, uint64_t n, const fastsgd_params* params,
                                         float* dense_out, void* stream);
 
+/*
+ * Model update on the decoded coordinates only (Sec. 5.1, "Implementation":
+ * the models are trained with Adam; Table of the running-time breakdown, part
+ * "model updating").  Hyper-parameters of the two Adam equations of Sec. 5.1.
+ */
+typedef struct fastsgd_adam {
+    float lr;      /* eta */
+    float beta1;
+    float beta2;
+    float eps;
+} fastsgd_adam;
+
+/*
+ * Decodes the workers' streams and applies one Adam step to the coordinates
+ * that received a non-zero aggregated gradient; all other coordinates keep
+ * theta, m and v (the update costs time in proportion to the kept entries, not
+ * to n).
+ *   streams_in, bytes, num_streams, n, params   as for
+ *                fastsgd_decompress_accumulate_batch
+ *   hyper        host pointer
+ *   grad_scratch device, n floats, ALL ZERO on entry and all zero again when
+ *                the call has run: the aggregated gradient g lives here between
+ *                the two passes (the caller clears it once, when it allocates it)
+ *   theta, m, v  device, n floats each, updated in place where g != 0:
+ *                  m = beta1 * m + (1 - beta1) * g
+ *                  v = beta2 * v + (1 - beta2) * g * g
+ *                  theta = theta - lr / sqrt(v + eps) * m
+ *                every operation one IEEE fp32 operation (round to nearest, no
+ *                fused multiply-add), in the order written
+ * g is the sum of the decoded streams in the given order, exactly as
+ * fastsgd_decompress_accumulate_batch forms it.  Two launches per 8 streams:
+ * aggregation, then the update.  Errors and damaged streams as for
+ * fastsgd_decompress_accumulate_batch (theta, m, v and grad_scratch are then
+ * unspecified, never accessed out of bounds).
+ */
+int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64_t* bytes,
+                                     uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                     const fastsgd_adam* hyper, float* grad_scratch,
+                                     float* theta, float* m, float* v, void* stream);
+
 /* ---- helpers, not on the timed path (no counterpart in the paper) ---------- */
 
 /* worst-case stream size in bytes (every entry kept, every delta at the widest

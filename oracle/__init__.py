@@ -40,6 +40,10 @@ class Params(C.Structure):
                 ("group_log2", C.c_uint32), ("reserved", C.c_uint32)]
 
 
+class Adam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
 def params(base: float, tau: int = 128, flag_bits: int = 2, group_log2: int = 14) -> Params:
     return Params(float(base), int(tau), int(flag_bits), int(group_log2), 0)
 
@@ -84,6 +88,8 @@ def lib():
         L.fsgo_parse.argtypes = [u8p, C.c_uint64, C.c_uint64, PP, u64p, i32p, u64p, f64p]
         L.fsgo_decompress_accumulate.restype = C.c_int
         L.fsgo_decompress_accumulate.argtypes = [u8p, C.c_uint64, C.c_uint64, PP, f32p]
+        L.fsgo_sparse_adam_update.restype = C.c_int
+        L.fsgo_sparse_adam_update.argtypes = [C.POINTER(u8p), u64p, C.c_uint32, C.c_uint64, PP, C.POINTER(Adam), f32p, f32p, f32p]
         _lib = L
     return _lib
 
@@ -210,3 +216,18 @@ def decompress_accumulate(stream, n: int, p: Params, dense: np.ndarray, nbytes: 
     nbytes = s.size if nbytes is None else nbytes
     assert dense.dtype == np.float32 and dense.flags.c_contiguous and dense.size == n
     return lib().fsgo_decompress_accumulate(_ptr(s, C.c_uint8), nbytes, n, C.byref(p), _ptr(dense, C.c_float))
+
+
+def sparse_adam_update(streams, n: int, p: Params, lr: float, beta1: float, beta2: float, eps: float,
+                       theta: np.ndarray, m: np.ndarray, v: np.ndarray) -> int:
+    """Adam (the experimental set-up's equations, no bias correction) on the coordinates where the sum of
+    the decoded streams is non-zero; in place on theta, m, v (float32, n entries each)."""
+    ss = [np.ascontiguousarray(s, np.uint8) for s in streams]
+    for a in (theta, m, v):
+        assert a.dtype == np.float32 and a.flags.c_contiguous and a.size == n
+    u8p = C.POINTER(C.c_uint8)
+    ptrs = (u8p * len(ss))(*[_ptr(s, C.c_uint8) for s in ss])
+    sizes = (C.c_uint64 * len(ss))(*[s.size for s in ss])
+    h = Adam(lr, beta1, beta2, eps)
+    return lib().fsgo_sparse_adam_update(ptrs, sizes, len(ss), n, C.byref(p), C.byref(h),
+                                         _ptr(theta, C.c_float), _ptr(m, C.c_float), _ptr(v, C.c_float))

@@ -488,3 +488,37 @@ int fsgo_decompress_accumulate(const uint8_t *stream, uint64_t bytes, uint64_t n
     }
     return walk_stream(stream, bytes, n, p, NULL, NULL, acc_sink, &c);
 }
+
+/* ---------------------------------------------------------- model update */
+
+int fsgo_sparse_adam_update(const uint8_t *const *streams, const uint64_t *bytes,
+                            uint32_t num_streams, uint64_t n, const fsgo_params *p,
+                            const fsgo_adam *h, float *theta, float *m, float *v)
+{
+    if (!params_ok(p) || n == 0) return FSGO_BAD_PARAM;
+    float *g = (float *)calloc(n, sizeof(float));
+    if (!g) return FSGO_BAD_PARAM;
+    /* the aggregated gradient: the workers' decoded streams added up in order */
+    for (uint32_t w = 0; w < num_streams; ++w) {
+        int rc = fsgo_decompress_accumulate(streams[w], bytes[w], n, p, g);
+        if (rc) { free(g); return rc; }
+    }
+    const float one_m_b1 = 1.0f - h->beta1, one_m_b2 = 1.0f - h->beta2;
+    for (uint64_t k = 0; k < n; ++k) {
+        const float gk = g[k];
+        if (gk == 0.0f) continue;
+        const float a1 = h->beta1 * m[k], a2 = one_m_b1 * gk;
+        const float mk = a1 + a2;
+        const float g2 = gk * gk;
+        const float c1 = h->beta2 * v[k], c2 = one_m_b2 * g2;
+        const float vk = c1 + c2;
+        const float den = sqrtf(vk + h->eps);
+        const float step = h->lr / den;
+        const float upd = step * mk;
+        m[k] = mk;
+        v[k] = vk;
+        theta[k] = theta[k] - upd;
+    }
+    free(g);
+    return FSGO_OK;
+}

@@ -127,6 +127,18 @@ int fsgo_parse(const uint8_t *stream, uint64_t bytes, uint64_t n,
 int fsgo_decompress_accumulate(const uint8_t *stream, uint64_t bytes,
                                uint64_t n, const fsgo_params *p, float *dense);
 
+/* Model update on the decoded coordinates only (Adam as printed in the
+ * experimental set-up: m = beta1 m + (1 - beta1) g, v = beta2 v + (1 - beta2) g^2,
+ * theta = theta - lr / sqrt(v + eps) * m, no bias correction).  g is the sum, in
+ * the order given, of the decoded streams; a coordinate whose g is zero (in no
+ * stream, or cancelled) keeps theta, m and v.  Every operation is one IEEE
+ * single-precision operation, in the order written in the source.  Returns the
+ * first stream's error, if any, with nothing updated. */
+typedef struct { float lr, beta1, beta2, eps; } fsgo_adam;
+int fsgo_sparse_adam_update(const uint8_t *const *streams, const uint64_t *bytes,
+                            uint32_t num_streams, uint64_t n, const fsgo_params *p,
+                            const fsgo_adam *h, float *theta, float *m, float *v);
+
 #ifdef __cplusplus
 }
 #endif

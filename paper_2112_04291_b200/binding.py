@@ -28,12 +28,17 @@ EXPORTS = [
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
+    "fastsgd_sparse_adam_update_batch",
 ]
 
 
 class Params(C.Structure):
     _fields_ = [("base", C.c_double), ("tau", C.c_uint32), ("flag_bits", C.c_uint32),
                 ("group_log2", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class Adam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
 
 
 def params(base: float, tau: int = 128, flag_bits: int = 2, group_log2: int = 14) -> Params:
@@ -68,6 +73,8 @@ def lib():
         L.fastsgd_compress_batch.argtypes = [C.POINTER(vp), u64, PP, C.POINTER(vp), u64, C.c_uint32, vp]
         L.fastsgd_decompress_accumulate_batch.restype = C.c_int
         L.fastsgd_decompress_accumulate_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, vp]
+        L.fastsgd_sparse_adam_update_batch.restype = C.c_int
+        L.fastsgd_sparse_adam_update_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, C.POINTER(Adam), vp, vp, vp, vp, vp]
         L.fastsgd_compress_bound.restype = u64
         L.fastsgd_compress_bound.argtypes = [u64, PP]
         L.fastsgd_workspace_bytes.restype = u64
@@ -186,6 +193,19 @@ def decompress_accumulate_batch(streams_in, nbytes, n: int, p: Params, dense: to
     sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
     return lib().fastsgd_decompress_accumulate_batch(ptrs, sizes, k, int(n), C.byref(p), dense.data_ptr(),
                                                      _stream_handle(stream))
+
+
+def sparse_adam_update_batch(streams_in, nbytes, n: int, p: Params, hyper: Adam, grad_scratch: torch.Tensor,
+                             theta: torch.Tensor, m: torch.Tensor, v: torch.Tensor, stream=None) -> int:
+    """fastsgd_sparse_adam_update_batch: decode the workers' streams, one Adam step where the aggregated gradient is non-zero."""
+    for a in (grad_scratch, theta, m, v):
+        assert a.is_cuda and a.dtype == torch.float32 and a.is_contiguous() and a.numel() == n
+    k = len(streams_in)
+    assert all(s.is_cuda and s.dtype == torch.uint8 for s in streams_in) and len(nbytes) == k
+    ptrs = (C.c_void_p * k)(*[int(s.data_ptr()) for s in streams_in])
+    sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
+    return lib().fastsgd_sparse_adam_update_batch(ptrs, sizes, k, int(n), C.byref(p), C.byref(hyper), grad_scratch.data_ptr(),
+                                                  theta.data_ptr(), m.data_ptr(), v.data_ptr(), _stream_handle(stream))
 
 
 def stream_info(stream_in: torch.Tensor, stream=None):

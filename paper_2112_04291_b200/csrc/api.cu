@@ -135,11 +135,18 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_decode_accumulate<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
         return FASTSGD_E_CUDA;
-    {   // both instantiations must be resident with the grid the launch uses (the queue of large groups relies on it)
-        int b2a = 0, b2b = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2a, k_decode_accumulate<false>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2b, k_decode_accumulate<true>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
-        b2 = b2a < b2b ? b2a : b2b;
+    if (cudaFuncSetAttribute(k_decode_accumulate<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    {   // every instantiation must be resident with the grid the launch uses (the queue of large groups relies on it)
+        int b2x[4] = {0, 0, 0, 0};
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[0], k_decode_accumulate<false>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[1], k_decode_accumulate<true>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[2], k_decode_accumulate<false, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[3], k_decode_accumulate<true, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        b2 = b2x[0];
+        for (int i = 1; i < 4; ++i) if (b2x[i] < b2) b2 = b2x[i];
     }
     g_state.device = dev;
     g_state.sm_count = sms;
@@ -335,9 +342,12 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
     return fastsgd_compress_batch(g1, n, params, o1, out_bytes, 1u, stream);
 }
 
-int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uint64_t* bytes,
-                                        uint32_t num_streams, uint64_t n, const fastsgd_params* params,
-                                        float* dense_out, void* stream) {
+namespace {
+// The decoder's launches over a list of streams, 8 per launch.  adam == nullptr: aggregation into
+// dense_out; else the model-update pass (dense_out holds the aggregated gradient).
+int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32_t num_streams, uint64_t n,
+                    const fastsgd_params* params, float* dense_out, const fastsgd_adam* adam,
+                    float* theta, float* m, float* v, void* stream) {
     if (!streams_in || !bytes || !dense_out || !params) return FASTSGD_E_NULL;
     if (!aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
     PowTable pw;
@@ -382,15 +392,43 @@ int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uin
         da.q_list = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kQueueOffset);
         da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
         da.group_log2 = params->group_log2;
+        if (adam) {
+            da.theta = theta; da.m = m; da.v = v;
+            da.lr = adam->lr; da.beta1 = adam->beta1; da.beta2 = adam->beta2; da.eps = adam->eps;
+        }
         {
             LaunchTimer lt(2, st);
-            if (da.W == 1u) k_decode_accumulate<true><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
-            else k_decode_accumulate<false><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            if (adam) {
+                if (da.W == 1u) k_decode_accumulate<true, 1><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+                else k_decode_accumulate<false, 1><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            } else {
+                if (da.W == 1u) k_decode_accumulate<true><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+                else k_decode_accumulate<false><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            }
         }
         g_launches.fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;
     }
     return FASTSGD_OK;
+}
+}  // namespace
+
+int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uint64_t* bytes,
+                                        uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                        float* dense_out, void* stream) {
+    return decode_launches(streams_in, bytes, num_streams, n, params, dense_out, nullptr, nullptr, nullptr, nullptr, stream);
+}
+
+int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64_t* bytes,
+                                     uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                     const fastsgd_adam* hyper, float* grad_scratch,
+                                     float* theta, float* m, float* v, void* stream) {
+    if (!hyper || !grad_scratch || !theta || !m || !v) return FASTSGD_E_NULL;
+    if (!aligned(theta, 4) || !aligned(m, 4) || !aligned(v, 4)) return FASTSGD_E_ALIGN;
+    // pass 1: the aggregated gradient; pass 2: the same streams again, every key's coordinate updated once
+    int rc = decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, nullptr, nullptr, nullptr, nullptr, stream);
+    if (rc) return rc;
+    return decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, hyper, theta, m, v, stream);
 }
 
 int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,

@@ -49,7 +49,31 @@ struct DecArgs {
     uint32_t            tau;
     uint32_t            l;
     uint32_t            group_log2;
+    // model update on the decoded coordinates (second pass; `dense` then holds the aggregated gradient)
+    float*              theta;
+    float*              m;
+    float*              v;
+    float               lr, beta1, beta2, eps;
 };
+
+// What a decoded (key, value) does to the entry `cur` of dense_out at that key; the result is stored there.
+// MODE 0: aggregation, cur + value.  MODE 1: model update: `cur` is the aggregated gradient g at that
+// key, left there by an aggregation pass over the same streams; where it is non-zero the coordinate takes one
+// Adam step (the experimental set-up's equations, no bias correction; one IEEE fp32 operation at a
+// time) and g returns to zero, so that a key that several streams hold is updated once.
+template <int MODE>
+__device__ __forceinline__ float apply_value(const DecArgs& a, uint32_t key, float cur, float value) {
+    if (MODE == 0) return __fadd_rn(cur, value);
+    if (cur != 0.0f) {
+        const float mk = __fadd_rn(__fmul_rn(a.beta1, a.m[key]), __fmul_rn(__fsub_rn(1.0f, a.beta1), cur));
+        const float vk = __fadd_rn(__fmul_rn(a.beta2, a.v[key]), __fmul_rn(__fsub_rn(1.0f, a.beta2), __fmul_rn(cur, cur)));
+        const float step = __fdiv_rn(a.lr, __fsqrt_rn(__fadd_rn(vk, a.eps)));
+        a.m[key] = mk;
+        a.v[key] = vk;
+        a.theta[key] = __fsub_rn(a.theta[key], __fmul_rn(step, mk));
+    }
+    return 0.0f;
+}
 
 __device__ __forceinline__ unsigned long long read_globaltimer_dec() {
     unsigned long long t;
@@ -174,7 +198,7 @@ __device__ __forceinline__ bool read_dir(const DecArgs& a, const uint32_t* sw, u
 // run of K consecutive keys; for K <= 8 (up to 2048 keys per block) everything it parses stays in
 // registers between the passes.  With `tile` the values go into the group's slice of dense_out held
 // in shared memory (block path), else straight into dense_out.
-template <bool BLOCK>
+template <int MODE, bool BLOCK>
 __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* blob, uint32_t nwords,
                                              uint32_t g, uint32_t count, uint32_t M, const float* val, float* tile,
                                              int t, int nthreads, int lane, int warp) {
@@ -304,13 +328,13 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
         if (BLOCK && tile != nullptr) {
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = __fadd_rn(tile[kk[k] - lo], vv[k]);
+                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = apply_value<MODE>(a, kk[k], tile[kk[k] - lo], vv[k]);
         } else {
             float dd[8];                                       // distinct keys: all loads, then all stores
 #pragma unroll
             for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = __fadd_rn(dd[k], vv[k]);
+            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = apply_value<MODE>(a, kk[k], dd[k], vv[k]);
         }
         return;
     }
@@ -324,8 +348,8 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
             const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
             const float mag = val[(code & 0x7Fu) + 1u];
             const float add = (code & 0x80u) ? -mag : mag;
-            if (BLOCK && tile != nullptr) tile[key - lo] = __fadd_rn(tile[key - lo], add);
-            else a.dense[key] = __fadd_rn(a.dense[key], add);
+            if (BLOCK && tile != nullptr) tile[key - lo] = apply_value<MODE>(a, key, tile[key - lo], add);
+            else a.dense[key] = apply_value<MODE>(a, key, a.dense[key], add);
         }
     }
 }
@@ -365,7 +389,7 @@ __device__ __forceinline__ void excl_scan_multi(const uint32_t (&v)[NS], uint32_
 // are parsed side by side (independent dependency chains, one scan barrier for all of them), each
 // is validated completely, and the sound ones are applied in stream order.  Every stream holds at
 // most KMAX * nthreads keys, so a thread's run of consecutive keys stays in registers.
-template <bool BLOCK, int NS, int KMAX, bool TWO_GROUPS = false>
+template <int MODE, bool BLOCK, int NS, int KMAX, bool TWO_GROUPS = false>
 __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, const uint32_t* const (&blob)[NS],
                                              const uint32_t (&nwords)[NS], const uint32_t (&count)[NS], const uint32_t (&M)[NS],
                                              const float* const (&val)[NS], uint32_t g, float* tile,
@@ -499,13 +523,13 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
         if (BLOCK && tile != nullptr) {
 #pragma unroll
             for (int k = 0; k < KMAX; ++k)
-                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = __fadd_rn(tile[kk[k] - lo[w]], vv[k]);
+                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = apply_value<MODE>(a, kk[k], tile[kk[k] - lo[w]], vv[k]);
         } else {
             float dd[KMAX];                                    // distinct keys: all loads, then all stores
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = __fadd_rn(dd[k], vv[k]);
+            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = apply_value<MODE>(a, kk[k], dd[k], vv[k]);
         }
     }
 }
@@ -529,7 +553,8 @@ __device__ __forceinline__ void stage_blob(uint32_t* dst, const uint32_t* src, u
 
 // ONE_STREAM: the launch holds a single stream (its own instantiation, so that the code of the
 // many-stream paths and of the two-groups-per-warp path do not weigh on each other)
-template <bool ONE_STREAM>
+// MODE: what a decoded value does to dense_out (apply_value): 0 aggregation, 1 model update.
+template <bool ONE_STREAM, int MODE = 0>
 __global__ void __launch_bounds__(kDecThreads, 2)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char dec_smem_raw[];
@@ -630,9 +655,9 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             }
             __syncwarp();
             if (c2[0] <= kDecWarpSide && c2[1] <= kDecWarpSide)
-                decode_multi<false, 2, 4, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
+                decode_multi<MODE, false, 2, 4, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
             else
-                decode_multi<false, 2, 8, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
+                decode_multi<MODE, false, 2, 8, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
             __syncwarp();
         }
     } else
@@ -680,10 +705,10 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 m2[0] = __shfl_sync(kFullMask, M, w0); m2[1] = __shfl_sync(kFullMask, M, w1);
                 v2[0] = s.val[w0]; v2[1] = s.val[w1];
                 if (w0 + 1u < W) {
-                    decode_multi<false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                    decode_multi<MODE, false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
                 } else {
                     const uint32_t* b1[1] = {b2[0]}; const uint32_t n1[1] = {n2[0]}, c1[1] = {c2[0]}, m1[1] = {m2[0]}; const float* v1[1] = {v2[0]};
-                    decode_multi<false, 1, 8>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+                    decode_multi<MODE, false, 1, 8>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
                 }
                 __syncwarp();      // these streams' stores before the next streams' loads of the same keys
             }
@@ -702,13 +727,13 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             }
             if (ns == 1u) {
                 const uint32_t* b1[1] = {bl[0]}; const uint32_t n1[1] = {nwv[0]}, c1[1] = {cv[0]}, m1[1] = {mv[0]}; const float* v1[1] = {vl[0]};
-                decode_multi<false, 1, 4>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+                decode_multi<MODE, false, 1, 4>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
             } else if (ns == 2u) {
                 const uint32_t* b2[2] = {bl[0], bl[1]}; const uint32_t n2[2] = {nwv[0], nwv[1]}, c2[2] = {cv[0], cv[1]}, m2[2] = {mv[0], mv[1]};
                 const float* v2[2] = {vl[0], vl[1]};
-                decode_multi<false, 2, 4>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                decode_multi<MODE, false, 2, 4>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
             } else {
-                decode_multi<false, 4, 4>(a, s, bl, nwv, cv, mv, vl, g, nullptr, lane, 32, lane, warp);
+                decode_multi<MODE, false, 4, 4>(a, s, bl, nwv, cv, mv, vl, g, nullptr, lane, 32, lane, warp);
             }
             __syncwarp();          // these streams' stores before the next streams' loads of the same keys
         }
@@ -803,16 +828,16 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 const uint32_t* b2[2] = {blob, blob2}; const uint32_t n2[2] = {s.g_nwords[w], s.g_nwords[w2]};
                 const uint32_t c2[2] = {c, s.g_count[w2]}, m2[2] = {s.g_M[w], s.g_M[w2]};
                 const float* v2[2] = {s.val[w], s.val[w2]};
-                decode_multi<true, 2, 4>(a, s, b2, n2, c2, m2, v2, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+                decode_multi<MODE, true, 2, 4>(a, s, b2, n2, c2, m2, v2, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
                 ++w;
             } else if (c == 0u) {
                 continue;
             } else if (c <= 4u * (uint32_t)kDecThreads) {
                 const uint32_t* b1[1] = {blob}; const uint32_t n1[1] = {s.g_nwords[w]}, c1[1] = {c}, m1[1] = {s.g_M[w]};
                 const float* v1[1] = {s.val[w]};
-                decode_multi<true, 1, 4>(a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+                decode_multi<MODE, true, 1, 4>(a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
             } else {
-                decode_group<true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                decode_group<MODE, true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
                                    tid, kDecThreads, lane, warp);
             }
             __syncthreads();       // these streams' updates before the next stream's

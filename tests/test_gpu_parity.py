@@ -525,3 +525,86 @@ def test_tiles_below_the_threshold_are_never_read_again(tiles, workers):
             assert np.array_equal(bufs[w].view[:total].cpu().numpy(), ostream), (w, rep)
             if w != 1:
                 assert 0 < d < n // 10
+
+
+@pytest.mark.parametrize("workers", [1, 3, 8, 10])
+def test_sparse_adam_update_equals_the_oracles(workers):
+    # the workers' streams decoded and one Adam step applied where the aggregated gradient is non-zero:
+    # theta, m, v bit-equal to the oracle's, untouched coordinates untouched, the scratch vector back to zero;
+    # two workers hold opposite values at shared keys (cancelled coordinates stay), tiles of every density
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(300 + workers)
+    n = 41 * 16384 - 1234
+    grads = [workloads.student_t_layers(n, seed=50 + w, blocks=7, lo=1e-4, hi=1e-1) for w in range(workers)]
+    if workers >= 3:
+        grads[2] = -grads[0]
+    base = workloads.base_for_keep(grads[0], n // 25)
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    bufs = [G.Guarded(cap) for _ in range(workers)]
+    assert binding.compress_batch([G.to_dev(v) for v in grads], pg, [b.view for b in bufs]) == 0
+    streams, sizes = [], []
+    for b in bufs:
+        total, d, status = binding.stream_info(b.view)
+        assert status == 0
+        streams.append(b.view[:total].cpu().numpy()); sizes.append(total)
+    theta0 = rng.standard_normal(n).astype(np.float32)
+    m0 = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    v0 = (rng.standard_normal(n) ** 2 * 1e-6).astype(np.float32)
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    ot, om, ov = theta0.copy(), m0.copy(), v0.copy()
+    assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+    gt, gm, gv, gs = (G.Guarded(4 * n) for _ in range(4))
+    theta, m, v, scratch = (x.view.view(torch.float32) for x in (gt, gm, gv, gs))
+    theta.copy_(torch.from_numpy(theta0)); m.copy_(torch.from_numpy(m0)); v.copy_(torch.from_numpy(v0))
+    for rep in range(2):                  # a second step right after: the scratch vector came back clean
+        rc = binding.sparse_adam_update_batch([b.view for b in bufs], sizes, n, pg, binding.Adam(lr, b1, b2, eps),
+                                              scratch, theta, m, v)
+        assert rc == 0 and binding.decode_status() == 0
+        assert all(x.intact() for x in (gt, gm, gv, gs))
+        assert not bool(scratch.any().item())
+        if rep == 1:
+            assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+        assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
+    changed = int((ot != theta0).sum())
+    assert 0 < changed < n // 4
+    if workers == 3:
+        # coordinates kept by workers 0 and 2 alone cancel and must not move
+        dense = np.zeros(n, np.float32)
+        for s in streams:
+            assert oracle.decompress_accumulate(s, n, po, dense) == 0
+        assert np.array_equal(m0[dense == 0], om[dense == 0])
+
+
+def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(77)
+    n = 5 * 16384 + 100
+    v_in = rng.standard_normal(n).astype(np.float32)
+    v_in[3 * 16384:4 * 16384] = 0.0
+    base = workloads.base_for_keep(v_in, n // 3)            # a third kept: whole blocks decode the groups
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    buf = G.Guarded(binding.compress_bound(n, pg))
+    assert binding.compress(G.to_dev(v_in), pg, buf.view) == 0
+    total, d, status = binding.stream_info(buf.view)
+    assert status == 0 and d > n // 4
+    s = buf.view[:total].cpu().numpy()
+    ot, om, ov = np.ones(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    assert oracle.sparse_adam_update([s], n, po, 0.01, 0.9, 0.999, 1e-8, ot, om, ov) == 0
+    theta = torch.ones(n, dtype=torch.float32, device=G.dev())
+    m = torch.zeros(n, dtype=torch.float32, device=G.dev()); v = torch.zeros_like(m); scratch = torch.zeros_like(m)
+    h = binding.Adam(0.01, 0.9, 0.999, 1e-8)
+    assert binding.sparse_adam_update_batch([buf.view], [total], n, pg, h, scratch, theta, m, v) == 0
+    assert binding.decode_status() == 0 and not bool(scratch.any().item())
+    assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
+    import ctypes as C
+    lib = binding.lib()
+    ptrs = (C.c_void_p * 1)(int(buf.view.data_ptr())); sizes = (C.c_uint64 * 1)(total)
+    assert lib.fastsgd_sparse_adam_update_batch(ptrs, sizes, 1, n, C.byref(pg), None, scratch.data_ptr(), theta.data_ptr(),
+                                                m.data_ptr(), v.data_ptr(), None) == binding.E_NULL
+    assert lib.fastsgd_sparse_adam_update_batch(ptrs, sizes, 1, n, C.byref(pg), C.byref(h), scratch.data_ptr(), None,
+                                                m.data_ptr(), v.data_ptr(), None) == binding.E_NULL
