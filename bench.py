@@ -387,6 +387,21 @@ def main():
     sub = max(3, min(args.steps, 50))
     ms_comp = (timed(run_comp, sub) if step_exceeds_l2 else timed_flushed(run_comp, sub)) / sub
     ms_dec = timed_flushed(run_dec, sub) / sub      # (streams and touched lines of dense_out would otherwise stay in L2)
+
+    # the step that follows the path: decode + Adam on the decoded coordinates only (same streams; eager, flushed)
+    theta = torch.zeros(n, dtype=torch.float32, device=dev)
+    adam_m, adam_v, adam_g = torch.zeros_like(theta), torch.zeros_like(theta), torch.zeros_like(theta)
+    hyper = binding.Adam(1e-3, 0.9, 0.999, 1e-8)
+
+    def adam_all():
+        rc = binding.sparse_adam_update_batch(outs, [cap] * W, n, pg, hyper, adam_g, theta, adam_m, adam_v)
+        if rc:
+            raise binding.FastSGDError(rc, "fastsgd_sparse_adam_update_batch")
+
+    adam_all()
+    ms_adam = timed_flushed(adam_all, sub) / sub
+    assert binding.decode_status() == 0
+    del theta, adam_m, adam_v, adam_g
     assert all(binding.stream_info(o)[2] == 0 for o in outs) and binding.decode_status() == 0
 
     # per-kernel durations from CUDA events recorded on the launching stream
@@ -459,6 +474,9 @@ def main():
         "decompress": {"ms": ms_dec, "input_gbs": in_bytes / (ms_dec * 1e-3) / 1e9,
                        "algorithmic_gbs": alg_dec / (ms_dec * 1e-3) / 1e9,
                        "frac_of_hbm_peak": alg_dec / (ms_dec * 1e-3) / 1e9 / peak},
+        "sparse_adam_update": {"ms": ms_adam, "touched_bytes": float(sum(stream_bytes)) * 2.0 + 40.0 * float(sum(kept)),
+                               "note": "decode + Adam step on decoded coordinates only; two launches per 8 streams; "
+                                       "256 MiB written before every call; not part of value / ms_per_step"},
         "stream": {"bytes_per_worker": float(sum(stream_bytes)) / W, "kept_per_worker": float(sum(kept)) / W,
                    "bits_per_kept_entry": 8.0 * sum(stream_bytes) / max(1, sum(kept)),
                    "ratio_vs_dense_fp32": in_bytes / max(1.0, float(sum(stream_bytes)))},

@@ -56,23 +56,41 @@ struct DecArgs {
     float               lr, beta1, beta2, eps;
 };
 
-// What a decoded (key, value) does to the entry `cur` of dense_out at that key; the result is stored there.
+// What a thread's run of K decoded (key, value) pairs does to the entries `cur` of dense_out at those keys
+// (distinct; 0xFFFFFFFF: no key); the results are stored there by the caller.
 // MODE 0: aggregation, cur + value.  MODE 1: model update: `cur` is the aggregated gradient g at that
 // key, left there by an aggregation pass over the same streams; where it is non-zero the coordinate takes one
 // Adam step (the experimental set-up's equations, no bias correction; one IEEE fp32 operation at a
-// time) and g returns to zero, so that a key that several streams hold is updated once.
-template <int MODE>
-__device__ __forceinline__ float apply_value(const DecArgs& a, uint32_t key, float cur, float value) {
-    if (MODE == 0) return __fadd_rn(cur, value);
-    if (cur != 0.0f) {
-        const float mk = __fadd_rn(__fmul_rn(a.beta1, a.m[key]), __fmul_rn(__fsub_rn(1.0f, a.beta1), cur));
-        const float vk = __fadd_rn(__fmul_rn(a.beta2, a.v[key]), __fmul_rn(__fsub_rn(1.0f, a.beta2), __fmul_rn(cur, cur)));
-        const float step = __fdiv_rn(a.lr, __fsqrt_rn(__fadd_rn(vk, a.eps)));
-        a.m[key] = mk;
-        a.v[key] = vk;
-        a.theta[key] = __fsub_rn(a.theta[key], __fmul_rn(step, mk));
+// time) and g returns to zero, so that a key that several streams hold is updated once.  All loads of
+// the moments and the parameters are issued before the first of them is needed.
+template <int MODE, int K>
+__device__ __forceinline__ void apply_run(const DecArgs& a, const uint32_t (&kk)[K], const float (&cur)[K],
+                                          const float (&value)[K], float (&res)[K]) {
+    if (MODE == 0) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) res[k] = __fadd_rn(cur[k], value[k]);
+        return;
     }
-    return 0.0f;
+    float pm[K], pv[K], pt[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const bool on = kk[k] != 0xFFFFFFFFu && cur[k] != 0.0f;
+        pm[k] = on ? a.m[kk[k]] : 0.0f;
+        pv[k] = on ? a.v[kk[k]] : 0.0f;
+        pt[k] = on ? a.theta[kk[k]] : 0.0f;
+    }
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (kk[k] != 0xFFFFFFFFu && cur[k] != 0.0f) {
+            const float mk = __fadd_rn(__fmul_rn(a.beta1, pm[k]), __fmul_rn(__fsub_rn(1.0f, a.beta1), cur[k]));
+            const float vk = __fadd_rn(__fmul_rn(a.beta2, pv[k]), __fmul_rn(__fsub_rn(1.0f, a.beta2), __fmul_rn(cur[k], cur[k])));
+            const float step = __fdiv_rn(a.lr, __fsqrt_rn(__fadd_rn(vk, a.eps)));
+            a.m[kk[k]] = mk;
+            a.v[kk[k]] = vk;
+            a.theta[kk[k]] = __fsub_rn(pt[k], __fmul_rn(step, mk));
+        }
+        res[k] = 0.0f;
+    }
 }
 
 __device__ __forceinline__ unsigned long long read_globaltimer_dec() {
@@ -325,31 +343,54 @@ __device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, con
                 kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
             }
         }
+        float dd[8], res[8];                                   // distinct keys: all loads, then all stores
         if (BLOCK && tile != nullptr) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = apply_value<MODE>(a, kk[k], tile[kk[k] - lo], vv[k]);
+            for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo] : 0.f;
+            apply_run<MODE, 8>(a, kk, dd, vv, res);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = res[k];
         } else {
-            float dd[8];                                       // distinct keys: all loads, then all stores
 #pragma unroll
             for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
+            apply_run<MODE, 8>(a, kk, dd, vv, res);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = apply_value<MODE>(a, kk[k], dd[k], vv[k]);
+            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
         }
         return;
     }
     {
+        // longer runs: four keys at a time (their loads in flight together)
         uint32_t pos = pos0, key = key0;
-        for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            key += get_bits(blob, nwords, pos, w);
-            pos += w;
-            const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
-            const float mag = val[(code & 0x7Fu) + 1u];
-            const float add = (code & 0x80u) ? -mag : mag;
-            if (BLOCK && tile != nullptr) tile[key - lo] = apply_value<MODE>(a, key, tile[key - lo], add);
-            else a.dense[key] = apply_value<MODE>(a, key, a.dense[key], add);
+        for (uint32_t j0 = jb; j0 < je; j0 += 4u) {
+            uint32_t kk[4]; float vv[4], dd[4], res[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t j = j0 + (uint32_t)u;
+                kk[u] = 0xFFFFFFFFu; vv[u] = 0.f;
+                if (j < je) {
+                    const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
+                    const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
+                    key += get_bits(blob, nwords, pos, w);
+                    pos += w;
+                    const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+                    const float mag = val[(code & 0x7Fu) + 1u];
+                    kk[u] = key; vv[u] = (code & 0x80u) ? -mag : mag;
+                }
+            }
+            if (BLOCK && tile != nullptr) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) dd[u] = kk[u] != 0xFFFFFFFFu ? tile[kk[u] - lo] : 0.f;
+                apply_run<MODE, 4>(a, kk, dd, vv, res);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (kk[u] != 0xFFFFFFFFu) tile[kk[u] - lo] = res[u];
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) dd[u] = kk[u] != 0xFFFFFFFFu ? a.dense[kk[u]] : 0.f;
+                apply_run<MODE, 4>(a, kk, dd, vv, res);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (kk[u] != 0xFFFFFFFFu) a.dense[kk[u]] = res[u];
+            }
         }
     }
 }
@@ -520,16 +561,19 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
                 kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
             }
         }
+        float dd[KMAX], res[KMAX];                             // distinct keys: all loads, then all stores
         if (BLOCK && tile != nullptr) {
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k)
-                if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = apply_value<MODE>(a, kk[k], tile[kk[k] - lo[w]], vv[k]);
+            for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo[w]] : 0.f;
+            apply_run<MODE, KMAX>(a, kk, dd, vv, res);
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = res[k];
         } else {
-            float dd[KMAX];                                    // distinct keys: all loads, then all stores
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
+            apply_run<MODE, KMAX>(a, kk, dd, vv, res);
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = apply_value<MODE>(a, kk[k], dd[k], vv[k]);
+            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
         }
     }
 }

@@ -124,3 +124,31 @@ def test_config5_sweep(log2n, keep):
 def test_config5_sweep_largest():
     wl = workloads.make("c5", n=1 << 30, keep=1e-3)
     _run(wl)
+
+
+def test_config2_sparse_adam_update_as_benchmarked():
+    # config 2's four streams, the model update bench.py times: theta, m, v bit-equal to the oracle's
+    wl = workloads.make("c2")
+    n, W = wl.n, wl.workers
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg)
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    outs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(W)]
+    assert binding.compress_batch([torch.from_numpy(g).cuda() for g in wl.grads], pg, outs) == 0
+    streams = []
+    for o in outs:
+        total, d, status = binding.stream_info(o)
+        assert status == 0
+        streams.append(o[:total].cpu().numpy())
+    rng = np.random.default_rng(9)
+    theta0 = rng.standard_normal(n).astype(np.float32)
+    ot, om, ov = theta0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+    theta = torch.from_numpy(theta0).cuda()
+    m = torch.zeros(n, dtype=torch.float32, device="cuda"); v = torch.zeros_like(m); scratch = torch.zeros_like(m)
+    assert binding.sparse_adam_update_batch(outs, [cap] * W, n, pg, binding.Adam(lr, b1, b2, eps), scratch, theta, m, v) == 0
+    assert binding.decode_status() == 0 and not bool(scratch.any().item())
+    assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
+    assert 0 < int((ot != theta0).sum()) <= 4 * n // 100
