@@ -231,6 +231,82 @@ def run_sweep(args):
     print(json.dumps(line), flush=True)
 
 
+def run_keys_table(args):
+    """Size per gradient key (the paper's two tables on the space cost of the gradient key, restated on
+    synthetic keys): Algorithm 2 as printed (one chain, one M; written by fastsgd_key_encode_paper) for
+    l = 1..5, the product stream's key part (groups of 2^14, flags and deltas as planes) for the same l,
+    and a byte-granular delta baseline (every delta in whole bytes plus a 2-bit byte count).  The key sets
+    are the kept keys of the benchmark gradients, obtained through the product path (compress, decode
+    into a zero vector, positions of the non-zeros).  Writes a markdown table to args.keys_table."""
+    import torch
+    from paper_2112_04291_b200 import binding, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    rows = []
+    sets = [("c2 worker 0 (25.6 M, 0.5 %, layered)", "c2", {}), ("c3 (50 M, clustered runs)", "c3", {}),
+            ("c5 2^24, 1 % (uniform)", "c5", {"n": 1 << 24, "keep": 1e-2}), ("c5 2^26, 0.1 % (uniform)", "c5", {"n": 1 << 26, "keep": 1e-3})]
+    for label, name, kw in sets:
+        wl = workloads.make(name, workers=1, **kw)
+        n = wl.n
+        grad = torch.from_numpy(wl.grads[0]).to(dev)
+        row = {"set": label, "n": n}
+        keys = None
+        for l in (1, 2, 3, 4, 5):
+            pg = binding.params(wl.base, wl.tau, l, wl.group_log2)
+            binding.ensure_workspace(n, pg, dev)
+            cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+            out = torch.zeros(cap, dtype=torch.uint8, device=dev)
+            assert binding.compress(grad, pg, out) == 0
+            total, d, status = binding.stream_info(out)
+            assert status == 0 and d > 0
+            G = (n + (1 << wl.group_log2) - 1) >> wl.group_log2
+            row["grouped_l%d" % l] = (8.0 * (total - 64 - 8 * G) - 8.0 * d) / d      # blobs minus the code bytes (incl. padding)
+            row["grouped_dir_l%d" % l] = (8.0 * (total - 64) - 8.0 * d) / d          # ... plus the directory
+            if keys is None:
+                dense = torch.zeros(n, dtype=torch.float32, device=dev)
+                assert binding.decompress_accumulate(out, cap, n, pg, dense) == 0 and binding.decode_status() == 0
+                keys = torch.nonzero(dense).flatten().to(torch.int32).contiguous()
+                assert keys.numel() == d
+                del dense
+            buf = torch.empty(binding.key_encode_paper_bound(keys.numel(), l), dtype=torch.uint8, device=dev)
+            ts = []
+            for it in range(8):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                assert binding.key_encode_paper(keys, l, buf) == 0
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            hdr = buf[:16].cpu().numpy()
+            nbits = int(hdr[8:16].view(np.uint64)[0])
+            row["paper_l%d" % l] = nbits / keys.numel()
+            row["paper_M"] = int(hdr[0:4].view(np.uint32)[0])
+            row["paper_us_l%d" % l] = statistics.median(ts[2:]) * 1e3
+            del out, buf
+        k = keys.cpu().numpy().astype(np.int64)
+        delta = np.diff(np.concatenate([[0], k]))
+        nbytes = np.maximum(1, (np.floor(np.log2(np.maximum(delta, 1))).astype(np.int64) + 8) // 8)
+        row["byte_granular"] = float((8 * nbytes + 2).sum()) / k.size
+        row["d"] = int(k.size)
+        rows.append(row)
+        del grad, keys
+    with open(args.keys_table, "w") as f:
+        f.write("| key set | kept keys | format | l=1 | l=2 | l=3 | l=4 | l=5 |\n|---|---|---|---|---|---|---|---|\n")
+        for r in rows:
+            f.write("| %s | %d | Algorithm 2 as printed (one chain, M = %d), bits per key | %s |\n" % (
+                r["set"], r["d"], r["paper_M"], " | ".join("%.2f" % r["paper_l%d" % l] for l in range(1, 6))))
+            f.write("| | | product stream, key part of the blobs | %s |\n" % " | ".join("%.2f" % r["grouped_l%d" % l] for l in range(1, 6)))
+            f.write("| | | product stream, key part + directory | %s |\n" % " | ".join("%.2f" % r["grouped_dir_l%d" % l] for l in range(1, 6)))
+            f.write("| | | byte-granular deltas + 2-bit byte count: %.2f; plain 32-bit keys: 32.00 | | | | | |\n" % r["byte_granular"])
+            f.write("| | | fastsgd_key_encode_paper, us per call | %s |\n" % " | ".join("%.1f" % r["paper_us_l%d" % l] for l in range(1, 6)))
+    best = rows[0]
+    print(json.dumps({"metric": "bits per gradient key", "value": best["paper_l2"], "unit": "bits", "n_gpus": 1,
+                      "higher_is_better": False, "data": "synthetic", "config": {"workload": "key sets of c2, c3, c5", "table": args.keys_table},
+                      "rows": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -246,6 +322,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph of the step")
     ap.add_argument("--sweep", default=None, metavar="FILE", help="config 5: size x keep-ratio sweep, markdown table written to FILE")
     ap.add_argument("--sweep-max-log2", type=int, default=30)
+    ap.add_argument("--keys-table", default=None, metavar="FILE", help="size per gradient key for l = 1..5 on the benchmark key sets, markdown table written to FILE")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -258,6 +335,10 @@ def main():
     if args.sweep:
         if rank == 0:
             run_sweep(args)
+        return
+    if args.keys_table:
+        if rank == 0:
+            run_keys_table(args)
         return
 
     import torch

@@ -196,6 +196,29 @@ int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64
                                      const fastsgd_adam* hyper, float* grad_scratch,
                                      float* theta, float* m, float* v, void* stream);
 
+/*
+ * Algorithm 2 exactly as printed (Sec. 3.3): one delta chain over all kept keys
+ * starting from preKey = 0, one M = max(1, bitlen(maxDelta)), and the binary
+ * sequence BK = flag || delta for each key in turn, most significant bit first
+ * (level f of the 2^l levels holds ceil((f+1) M / 2^l) bits; a delta takes the
+ * lowest level that holds it).  The product stream of fastsgd_compress uses the
+ * same code per group of 2^14 indices; this call states the paper's own format
+ * and its size per key (Tables "space cost of gradient key").
+ *   keys       device, d ascending 32-bit keys (a first key of 0 gives a delta
+ *              of 0; later deltas are >= 1)
+ *   flag_bits  l, 1..5
+ *   out        device, 16-byte aligned, fastsgd_key_encode_paper_bound(d, l)
+ *              bytes at least (else FASTSGD_E_CAPACITY):
+ *                u32 M | u32 l | u64 number of bits in BK
+ *                u64 index[ceil(d / 2048)]: bit offset in BK of key 2048 i
+ *                BK, zero bits up to a multiple of 32
+ * Four small launches on `stream`; no workspace.  Keys that do not ascend give
+ * an unspecified BK, never an access outside the buffers.
+ */
+uint64_t fastsgd_key_encode_paper_bound(uint64_t d, uint32_t flag_bits);
+int fastsgd_key_encode_paper(const uint32_t* keys, uint64_t d, uint32_t flag_bits,
+                             void* out, uint64_t out_bytes, void* stream);
+
 /* ---- helpers, not on the timed path (no counterpart in the paper) ---------- */
 
 /* worst-case stream size in bytes (every entry kept, every delta at the widest

@@ -28,7 +28,7 @@ EXPORTS = [
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
-    "fastsgd_sparse_adam_update_batch",
+    "fastsgd_sparse_adam_update_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
 ]
 
 
@@ -73,6 +73,10 @@ def lib():
         L.fastsgd_compress_batch.argtypes = [C.POINTER(vp), u64, PP, C.POINTER(vp), u64, C.c_uint32, vp]
         L.fastsgd_decompress_accumulate_batch.restype = C.c_int
         L.fastsgd_decompress_accumulate_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, vp]
+        L.fastsgd_key_encode_paper_bound.restype = C.c_uint64
+        L.fastsgd_key_encode_paper_bound.argtypes = [u64, C.c_uint32]
+        L.fastsgd_key_encode_paper.restype = C.c_int
+        L.fastsgd_key_encode_paper.argtypes = [vp, u64, C.c_uint32, vp, u64, vp]
         L.fastsgd_sparse_adam_update_batch.restype = C.c_int
         L.fastsgd_sparse_adam_update_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, C.POINTER(Adam), vp, vp, vp, vp, vp]
         L.fastsgd_compress_bound.restype = u64
@@ -206,6 +210,18 @@ def sparse_adam_update_batch(streams_in, nbytes, n: int, p: Params, hyper: Adam,
     sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
     return lib().fastsgd_sparse_adam_update_batch(ptrs, sizes, k, int(n), C.byref(p), C.byref(hyper), grad_scratch.data_ptr(),
                                                   theta.data_ptr(), m.data_ptr(), v.data_ptr(), _stream_handle(stream))
+
+
+def key_encode_paper_bound(d: int, flag_bits: int) -> int:
+    return int(lib().fastsgd_key_encode_paper_bound(int(d), int(flag_bits)))
+
+
+def key_encode_paper(keys: torch.Tensor, flag_bits: int, out: torch.Tensor, stream=None) -> int:
+    """fastsgd_key_encode_paper: Algorithm 2 as printed over `keys` (int32 tensor holding ascending 32-bit keys)."""
+    assert keys.is_cuda and keys.dtype == torch.int32 and keys.is_contiguous()
+    assert out.is_cuda and out.dtype == torch.uint8 and out.is_contiguous()
+    return lib().fastsgd_key_encode_paper(keys.data_ptr() if keys.numel() else None, keys.numel(), int(flag_bits),
+                                          out.data_ptr(), out.numel(), _stream_handle(stream))
 
 
 def stream_info(stream_in: torch.Tensor, stream=None):

@@ -12,6 +12,7 @@
 #include "sum.cuh"
 #include "bits.cuh"
 #include "compress.cuh"
+#include "keys_paper.cuh"
 #include "decode.cuh"
 
 namespace {
@@ -429,6 +430,46 @@ int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64
     int rc = decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, nullptr, nullptr, nullptr, nullptr, stream);
     if (rc) return rc;
     return decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, hyper, theta, m, v, stream);
+}
+
+uint64_t fastsgd_key_encode_paper_bound(uint64_t d, uint32_t flag_bits) {
+    if (flag_bits < 1 || flag_bits > 5 || d >= (1ull << 31)) return 0;
+    const uint64_t blocks = (d + kBkBlockKeys - 1) / kBkBlockKeys;
+    const uint64_t words = (d * (flag_bits + 32ull) + 31ull) / 32ull + 1ull;      // widest levels everywhere, and the padding word
+    return 16ull + 8ull * blocks + 4ull * words;
+}
+
+int fastsgd_key_encode_paper(const uint32_t* keys, uint64_t d, uint32_t flag_bits,
+                             void* out, uint64_t out_bytes, void* stream) {
+    if (!out || (!keys && d)) return FASTSGD_E_NULL;
+    if (!aligned(out, 16) || !aligned(keys, 4)) return FASTSGD_E_ALIGN;
+    const uint64_t need = fastsgd_key_encode_paper_bound(d, flag_bits);
+    if (!need) return FASTSGD_E_BAD_PARAM;
+    if (out_bytes < need) return FASTSGD_E_CAPACITY;
+    {
+        std::lock_guard<std::mutex> lock(g_state.mu);
+        const int rc = ensure_device_setup();
+        if (rc) return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    BkArgs a;
+    a.keys = keys; a.d = d; a.l = flag_bits;
+    a.blocks = (uint32_t)((d + kBkBlockKeys - 1) / kBkBlockKeys);
+    a.header = static_cast<uint32_t*>(out);
+    a.index = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(out) + 16);
+    a.bk = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(out) + 16 + 8ull * a.blocks);
+    if (cudaMemsetAsync(out, 0, 16, st) != cudaSuccess) return FASTSGD_E_CUDA;
+    if (a.blocks) {
+        const unsigned cap = 8u * (unsigned)g_state.sm_count;
+        const unsigned want = (unsigned)((d + kBkThreads - 1) / kBkThreads);
+        k_bk_maxdelta<<<want < cap ? want : cap, kBkThreads, 0, st>>>(a);
+        k_bk_sizes<<<a.blocks, kBkThreads, 0, st>>>(a);
+    }
+    k_bk_scan<<<1, kBkThreads, 0, st>>>(a);
+    if (a.blocks) k_bk_pack<<<a.blocks, kBkThreads, 0, st>>>(a);
+    g_launches.fetch_add(a.blocks ? 4 : 1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;
+    return FASTSGD_OK;
 }
 
 int fastsgd_decompress_accumulate(const void* stream_in, uint64_t bytes, uint64_t n,

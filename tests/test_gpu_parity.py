@@ -608,3 +608,73 @@ def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
                                                 m.data_ptr(), v.data_ptr(), None) == binding.E_NULL
     assert lib.fastsgd_sparse_adam_update_batch(ptrs, sizes, 1, n, C.byref(pg), C.byref(h), scratch.data_ptr(), None,
                                                 m.data_ptr(), v.data_ptr(), None) == binding.E_NULL
+
+
+def _gpu_bk(keys, l):
+    """Algorithm 2 as printed, on the GPU -> (BK as a '0'/'1' string, M, index of bit offsets)."""
+    import torch
+    import gpu_util as G
+    k = np.ascontiguousarray(keys, np.uint32)
+    need = binding.key_encode_paper_bound(k.size, l)
+    buf = G.Guarded(need, fill=0xC3)
+    dk = torch.from_numpy(k.view(np.int32)).to(G.dev())
+    assert binding.key_encode_paper(dk, l, buf.view) == 0
+    raw = buf.view.cpu().numpy()
+    assert buf.intact()
+    M, l_got = int(raw[0:4].view(np.uint32)[0]), int(raw[4:8].view(np.uint32)[0])
+    nbits = int(raw[8:16].view(np.uint64)[0])
+    blocks = (k.size + 2047) // 2048
+    index = raw[16:16 + 8 * blocks].view(np.uint64).copy()
+    bits = np.unpackbits(raw[16 + 8 * blocks:16 + 8 * blocks + 4 * ((nbits + 31) // 32)])
+    assert l_got == l and not bits[nbits:].any(), "padding bits must be zero"
+    return "".join("01"[b] for b in bits[:nbits]), M, index
+
+
+def test_paper_key_stream_worked_example_on_the_gpu():
+    # the key list of the worked example under Fig. 3 (largest delta 232 -> M = 8, last key 578 -> '0011')
+    keys = [10, 242, 300, 400, 575, 578]
+    bk, M, index = _gpu_bk(keys, 2)
+    obk, oM = oracle.key_encode_paper(keys, 2)
+    assert M == oM == 8 and bk == obk and bk.endswith("0011") and list(index) == [0]
+
+
+@pytest.mark.parametrize("l", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("d", [0, 1, 2, 2047, 2048, 2049, 70_001])
+def test_paper_key_stream_equals_the_oracles(d, l):
+    rng = np.random.default_rng(1000 * l + d)
+    if d % 2:
+        gaps = rng.geometric(0.01, size=d).astype(np.int64)                     # smooth gaps
+    else:
+        gaps = np.where(rng.random(d) < 0.97, rng.integers(1, 9, d), rng.integers(1, 200_000, d)).astype(np.int64)   # mostly tiny, some huge
+    if d:
+        gaps[0] = 0 if d % 3 == 0 else gaps[0]                                  # a first key of 0
+    keys = np.cumsum(gaps)
+    assert d == 0 or keys[-1] < 2 ** 31
+    bk, M, index = _gpu_bk(keys, l)
+    obk, oM = oracle.key_encode_paper(keys, l)
+    assert M == oM and len(bk) == len(obk) and bk == obk
+    # the index: bit offset of every 2048th key = length of the oracle's BK over the keys before it
+    for i, off in enumerate(index):
+        if i and i % 16 == 0 or i == len(index) - 1:
+            pre, _ = oracle.key_encode_paper(keys[:2048 * i], l) if i else ("", 0)
+            if i and oracle.key_encode_paper(keys[:2048 * i], l)[1] == oM:
+                assert int(off) == len(pre)
+
+
+def test_paper_key_stream_on_compressed_gradient_keys_and_wide_deltas():
+    # the kept keys of a compressed gradient, and keys spread over the whole 31-bit range (M = 31)
+    n = 600_000
+    v = workloads.student_t_layers(n, seed=4, blocks=9, lo=1e-4, hi=1e-1)
+    rc, keys, codes, S = oracle.value_encode(v, workloads.base_for_keep(v, n // 50), 128)
+    assert rc == 0 and keys.size > 5000
+    for l in (2, 3):
+        bk, M, _ = _gpu_bk(keys, l)
+        obk, oM = oracle.key_encode_paper(keys, l)
+        assert M == oM and bk == obk
+    wide = np.array([0, 1, 2 ** 30 + 5, 2 ** 31 - 1], np.uint64)
+    bk, M, _ = _gpu_bk(wide, 2)
+    obk, oM = oracle.key_encode_paper(wide, 2)
+    assert M == oM == 31 and bk == obk
+    import ctypes as C
+    assert binding.lib().fastsgd_key_encode_paper(None, 5, 2, None, 0, None) == binding.E_NULL
+    assert binding.key_encode_paper_bound(10, 9) == 0
