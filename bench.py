@@ -483,6 +483,31 @@ def main():
     ms_adam = timed_flushed(adam_all, sub) / sub
     assert binding.decode_status() == 0
     del theta, adam_m, adam_v, adam_g
+
+    # a gradient that is sparse before it is compressed (under 5 % non-zeros): worker 0 as key-value pairs (eager, flushed)
+    kv_info = None
+    nz = np.flatnonzero(wl.grads[0])
+    if 0 < nz.size <= n // 20:
+        kv_keys = torch.from_numpy(nz.astype(np.uint32).view(np.int32)).to(dev)
+        kv_vals = torch.from_numpy(wl.grads[0][nz]).to(dev)
+        kv_out = torch.zeros(cap, dtype=torch.uint8, device=dev)
+
+        def kv_one():
+            rc = binding.compress_kv(kv_keys, kv_vals, n, pg, kv_out)
+            if rc:
+                raise binding.FastSGDError(rc, "fastsgd_compress_kv")
+
+        def dense_one():
+            rc = binding.compress(grads[0], pg, kv_out)
+            if rc:
+                raise binding.FastSGDError(rc, "fastsgd_compress")
+
+        kv_one()
+        assert binding.stream_info(kv_out) == binding.stream_info(outs[0])
+        kv_info = {"pairs": int(nz.size), "ms": timed_flushed(kv_one, sub) / sub, "dense_call_ms": timed_flushed(dense_one, sub) / sub,
+                   "note": "fastsgd_compress_kv on worker 0's non-zero entries against fastsgd_compress on its dense vector; "
+                           "same stream; 256 MiB written before every call; not part of value / ms_per_step"}
+        del kv_keys, kv_vals, kv_out
     assert all(binding.stream_info(o)[2] == 0 for o in outs) and binding.decode_status() == 0
 
     # per-kernel durations from CUDA events recorded on the launching stream
@@ -558,6 +583,7 @@ def main():
         "sparse_adam_update": {"ms": ms_adam, "touched_bytes": float(sum(stream_bytes)) * 2.0 + 40.0 * float(sum(kept)),
                                "note": "decode + Adam step on decoded coordinates only; two launches per 8 streams; "
                                        "256 MiB written before every call; not part of value / ms_per_step"},
+        "compress_kv": kv_info,
         "stream": {"bytes_per_worker": float(sum(stream_bytes)) / W, "kept_per_worker": float(sum(kept)) / W,
                    "bits_per_kept_entry": 8.0 * sum(stream_bytes) / max(1, sum(kept)),
                    "ratio_vs_dense_fp32": in_bytes / max(1.0, float(sum(stream_bytes)))},

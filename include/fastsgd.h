@@ -126,6 +126,24 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
                            void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream);
 
 /*
+ * The encoder for a gradient given as key-value pairs (Sec. 2.2 states the
+ * problem on the D non-zero pairs (k_j, v_j) of a D_m-dimensional gradient;
+ * the sparse models of Sec. 5 produce it in this form).
+ *   keys    device, `count` strictly ascending 32-bit keys, each < n
+ *   values  device, the matching fp32 values (zeros allowed: never kept)
+ *   n       D_m; out, out_bytes, params, stream as for fastsgd_compress
+ * The stream is, byte for byte, the one fastsgd_compress writes for the dense
+ * vector that holds values[j] at keys[j] and zeros elsewhere: the sum is
+ * formed on the same tree (zeros add exactly nothing), the groups are the
+ * same.  Nothing of size n is read or written except the per-group tables of
+ * the workspace: cost in proportion to count and to n / 2^14.  Keys that do
+ * not ascend or reach n give an unspecified stream, never an access outside
+ * the buffers.  Two launches (tile boundaries; the fused kernel).
+ */
+int fastsgd_compress_kv(const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
+                        const fastsgd_params* params, void* out, uint64_t out_bytes, void* stream);
+
+/*
  * Decoder and aggregation (Sec. 3.1 decoder phases 1-4; Sec. 2.1 aggregation).
  *   stream_in  device, 16-byte aligned, a stream made by fastsgd_compress
  *   bytes      number of valid bytes at stream_in (>= header.total_bytes)

@@ -88,6 +88,8 @@ def lib():
         L.fsgo_parse.argtypes = [u8p, C.c_uint64, C.c_uint64, PP, u64p, i32p, u64p, f64p]
         L.fsgo_decompress_accumulate.restype = C.c_int
         L.fsgo_decompress_accumulate.argtypes = [u8p, C.c_uint64, C.c_uint64, PP, f32p]
+        L.fsgo_compress_kv.restype = C.c_int
+        L.fsgo_compress_kv.argtypes = [u64p, f32p, C.c_uint64, C.c_uint64, PP, u8p, C.c_uint64, u64p]
         L.fsgo_sparse_adam_update.restype = C.c_int
         L.fsgo_sparse_adam_update.argtypes = [C.POINTER(u8p), u64p, C.c_uint32, C.c_uint64, PP, C.POINTER(Adam), f32p, f32p, f32p]
         _lib = L
@@ -231,3 +233,16 @@ def sparse_adam_update(streams, n: int, p: Params, lr: float, beta1: float, beta
     h = Adam(lr, beta1, beta2, eps)
     return lib().fsgo_sparse_adam_update(ptrs, sizes, len(ss), n, C.byref(p), C.byref(h),
                                          _ptr(theta, C.c_float), _ptr(m, C.c_float), _ptr(v, C.c_float))
+
+
+def compress_kv(keys, values, n: int, p: Params, cap: int | None = None):
+    """Encoder on key-value pairs -> (status, stream bytes as uint8 array)."""
+    k = np.ascontiguousarray(keys, np.uint64)
+    v = _f32(values)
+    assert k.size == v.size
+    if cap is None:
+        cap = compress_bound(n, p)
+    out = np.zeros(max(cap, 64), np.uint8)
+    total = C.c_uint64(0)
+    rc = lib().fsgo_compress_kv(_ptr(k, C.c_uint64), _ptr(v, C.c_float), k.size, n, C.byref(p), _ptr(out, C.c_uint8), cap, C.byref(total))
+    return rc, out[:total.value].copy()

@@ -522,3 +522,20 @@ int fsgo_sparse_adam_update(const uint8_t *const *streams, const uint64_t *bytes
     free(g);
     return FSGO_OK;
 }
+
+/* ------------------------------------------------------- key-value input */
+
+int fsgo_compress_kv(const uint64_t *keys, const float *values, uint64_t count,
+                     uint64_t n, const fsgo_params *p, uint8_t *out, uint64_t cap,
+                     uint64_t *total)
+{
+    if (n == 0) return FSGO_BAD_PARAM;
+    for (uint64_t j = 0; j < count; ++j)
+        if (keys[j] >= n || (j && keys[j] <= keys[j - 1])) return FSGO_BAD_PARAM;
+    float *dense = (float *)calloc(n, sizeof(float));
+    if (!dense) return FSGO_BAD_PARAM;
+    for (uint64_t j = 0; j < count; ++j) dense[keys[j]] = values[j];
+    int rc = fsgo_compress(dense, n, p, out, cap, total);
+    free(dense);
+    return rc;
+}

@@ -127,6 +127,14 @@ int fsgo_parse(const uint8_t *stream, uint64_t bytes, uint64_t n,
 int fsgo_decompress_accumulate(const uint8_t *stream, uint64_t bytes,
                                uint64_t n, const fsgo_params *p, float *dense);
 
+/* The encoder on a gradient given as `count` key-value pairs (strictly ascending
+ * keys < n): by definition the stream of the dense vector that holds values[j]
+ * at keys[j] and zeros elsewhere.  FSGO_BAD_PARAM if the keys do not ascend or
+ * reach n. */
+int fsgo_compress_kv(const uint64_t *keys, const float *values, uint64_t count,
+                     uint64_t n, const fsgo_params *p, uint8_t *out, uint64_t cap,
+                     uint64_t *total);
+
 /* Model update on the decoded coordinates only (Adam as printed in the
  * experimental set-up: m = beta1 m + (1 - beta1) g, v = beta2 v + (1 - beta2) g^2,
  * theta = theta - lr / sqrt(v + eps) * m, no bias correction).  g is the sum, in

@@ -29,6 +29,7 @@ EXPORTS = [
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
     "fastsgd_sparse_adam_update_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
+    "fastsgd_compress_kv",
 ]
 
 
@@ -73,6 +74,8 @@ def lib():
         L.fastsgd_compress_batch.argtypes = [C.POINTER(vp), u64, PP, C.POINTER(vp), u64, C.c_uint32, vp]
         L.fastsgd_decompress_accumulate_batch.restype = C.c_int
         L.fastsgd_decompress_accumulate_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, vp, vp]
+        L.fastsgd_compress_kv.restype = C.c_int
+        L.fastsgd_compress_kv.argtypes = [vp, vp, u64, u64, PP, vp, u64, vp]
         L.fastsgd_key_encode_paper_bound.restype = C.c_uint64
         L.fastsgd_key_encode_paper_bound.argtypes = [u64, C.c_uint32]
         L.fastsgd_key_encode_paper.restype = C.c_int
@@ -210,6 +213,16 @@ def sparse_adam_update_batch(streams_in, nbytes, n: int, p: Params, hyper: Adam,
     sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
     return lib().fastsgd_sparse_adam_update_batch(ptrs, sizes, k, int(n), C.byref(p), C.byref(hyper), grad_scratch.data_ptr(),
                                                   theta.data_ptr(), m.data_ptr(), v.data_ptr(), _stream_handle(stream))
+
+
+def compress_kv(keys: torch.Tensor, values: torch.Tensor, n: int, p: Params, out: torch.Tensor, stream=None) -> int:
+    """fastsgd_compress_kv: the gradient as ascending keys (int32 tensor holding 32-bit keys) and their fp32 values."""
+    assert keys.is_cuda and keys.dtype == torch.int32 and keys.is_contiguous()
+    assert values.is_cuda and values.dtype == torch.float32 and values.is_contiguous() and values.numel() == keys.numel()
+    assert out.is_cuda and out.dtype == torch.uint8 and out.is_contiguous()
+    cnt = keys.numel()
+    return lib().fastsgd_compress_kv(keys.data_ptr() if cnt else None, values.data_ptr() if cnt else None, cnt, int(n),
+                                     C.byref(p), out.data_ptr(), out.numel(), _stream_handle(stream))
 
 
 def key_encode_paper_bound(d: int, flag_bits: int) -> int:

@@ -86,7 +86,8 @@ uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
 uint64_t ws_dense_offset(uint64_t n, uint32_t group_log2) {
     // partials, descriptors, prefixes, tile maxima, the list of tiles to encode and its bitmap for every gradient one launch can take
     const uint64_t G = groups_of(n, group_log2);
-    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 24ull * G + 4ull * ((G + 31ull) >> 5));
+    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 24ull * G + 4ull * ((G + 31ull) >> 5))
+                       + 4ull * (G + 2ull);
     return (b + 255ull) & ~255ull;
 }
 
@@ -105,6 +106,7 @@ WorkspaceView view(void* ws, uint64_t n) {
     v.tmax = reinterpret_cast<float*>(v.prefix + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
     v.nelist = reinterpret_cast<uint32_t*>(v.tmax + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
     v.nebits = v.nelist + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2);
+    v.kv_start = v.nebits + (uint64_t)kCmpMaxJobs * ((groups_of(n, kGroupLog2) + 31ull) >> 5);
     return v;
 }
 
@@ -121,6 +123,8 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_compress<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_compress<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
     int b1 = 0, b2 = 0, b3 = 0;
     {
         int b3b = 0;
@@ -128,6 +132,8 @@ int ensure_device_setup() {
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (b3b < b3) b3 = b3b;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<false, true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (b3b < b3) b3 = b3b;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<false, false, true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (b3b < b3) b3 = b3b;
     }
     g_state.cmp_blocks_per_sm = b3;
@@ -271,12 +277,19 @@ int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream
     return launch_sum(grad, n, 0u, 0u, pw, view(g_state.ws, n), sum_out, static_cast<cudaStream_t>(stream));
 }
 
-int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_params* params,
-                           void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream) {
-    if (!grads || !outs || !params) return FASTSGD_E_NULL;
+namespace {
+// The encoder's launches.  kv_keys == nullptr: num_grads dense gradients, up to 8 per launch.  Else one gradient
+// given as kv_count ascending keys with their values (grads is not used).
+int compress_launches(const float* const* grads, uint64_t n, const fastsgd_params* params,
+                      void* const* outs, uint64_t out_bytes, uint32_t num_grads,
+                      const uint32_t* kv_keys, const float* kv_vals, uint64_t kv_count, void* stream) {
+    const bool kv = kv_keys != nullptr || kv_vals != nullptr || grads == nullptr;
+    if (!outs || !params || (!kv && !grads)) return FASTSGD_E_NULL;
+    if (kv && kv_count && (!kv_keys || !kv_vals)) return FASTSGD_E_NULL;
+    if (kv && (!aligned(kv_keys, 4) || !aligned(kv_vals, 4))) return FASTSGD_E_ALIGN;
     for (uint32_t i = 0; i < num_grads; ++i) {
-        if (!grads[i] || !outs[i]) return FASTSGD_E_NULL;
-        if (!aligned(grads[i], 16) || !aligned(outs[i], 16)) return FASTSGD_E_ALIGN;
+        if ((!kv && !grads[i]) || !outs[i]) return FASTSGD_E_NULL;
+        if ((!kv && !aligned(grads[i], 16)) || !aligned(outs[i], 16)) return FASTSGD_E_ALIGN;
     }
     PowTable pw;
     int rc = check_params(params, &pw);
@@ -302,8 +315,15 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
         std::memset(&cb, 0, sizeof(cb));
         cb.jobs = num_grads - first < (uint32_t)kCmpMaxJobs ? num_grads - first : (uint32_t)kCmpMaxJobs;
         for (uint32_t i = 0; i < cb.jobs; ++i) {
-            cb.grad[i] = grads[first + i];
+            cb.grad[i] = kv ? nullptr : grads[first + i];
             cb.out[i] = static_cast<uint8_t*>(outs[first + i]);
+        }
+        if (kv) {
+            if (kv_count > n) return FASTSGD_E_BAD_N;
+            cb.kv_keys = kv_keys; cb.kv_vals = kv_vals; cb.kv_start = w.kv_start;
+            k_kv_bounds<<<(unsigned)((G + 1ull + 255ull) / 256ull), 256, 0, st>>>(kv_keys, (uint32_t)kv_count, (uint32_t)G, w.kv_start);
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;
         }
         cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc; cb.prefix = w.prefix; cb.tmax = w.tmax; cb.nelist = w.nelist; cb.nebits = w.nebits;
         cb.sm_slots = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kSmSlotOffset);
@@ -326,13 +346,32 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
         cudaError_t err;
         {
             LaunchTimer lt(1, st);
-            err = cudaLaunchCooperativeKernel(cb.jobs > 1u ? (const void*)k_compress<true> : (cb.G > kCmpBigTiles ? (const void*)k_compress<false, true> : (const void*)k_compress<false>), dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs,
-                                              sizeof(CmpSmem), st);
+            const void* fn = kv ? (const void*)k_compress<false, false, true>
+                                : cb.jobs > 1u ? (const void*)k_compress<true>
+                                : (cb.G > kCmpBigTiles ? (const void*)k_compress<false, true> : (const void*)k_compress<false>);
+            err = cudaLaunchCooperativeKernel(fn, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs, sizeof(CmpSmem), st);
         }
         if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     return FASTSGD_OK;
+}
+}  // namespace
+
+int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_params* params,
+                           void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream) {
+    if (!grads) return FASTSGD_E_NULL;
+    return compress_launches(grads, n, params, outs, out_bytes, num_grads, nullptr, nullptr, 0, stream);
+}
+
+int fastsgd_compress_kv(const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
+                        const fastsgd_params* params, void* out, uint64_t out_bytes, void* stream) {
+    if (!out) return FASTSGD_E_NULL;
+    static const uint32_t no_keys[1] = {0};
+    static const float no_vals[1] = {0.f};
+    void* o1[1] = {out};
+    // (an empty list still goes through the key-value kernel: the pointers only mark the mode then)
+    return compress_launches(nullptr, n, params, o1, out_bytes, 1u, count ? keys : no_keys, count ? values : no_vals, count, stream);
 }
 
 int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,

@@ -144,6 +144,11 @@ struct CmpBatch {
     uint32_t            l;
     uint32_t            teams;           // 1, or 2: the two blocks of every SM work on different gradients
     uint32_t            pad;
+    // key-value input (kernel variant KV, one gradient): the gradient is given as kv_count ascending keys with
+    // their values instead of grad[0]; kv_start[t] = index of the first entry with key >= t * 2^14, t = 0..G
+    const uint32_t*     kv_keys;
+    const float*        kv_vals;
+    const uint32_t*     kv_start;
 };
 
 __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
@@ -265,6 +270,35 @@ __device__ __forceinline__ void issue_half(CmpSmem& s, const CmpArgs& a, uint32_
         __syncthreads();
         // these were generic-proxy writes to a buffer that a later bulk copy (async proxy) overwrites
         if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+}
+
+// Key-value input: the tile is formed in the stage from the entries that fall into it (zeros
+// elsewhere), so that everything downstream sees what a bulk copy of the dense gradient would have
+// brought.  Called by the whole block; the stage must be free; complete when it returns.
+__device__ __forceinline__ void kv_fill_tile(CmpSmem& s, const CmpBatch& b, uint32_t tile, int tid) {
+    float4* st4 = reinterpret_cast<float4*>(&s.stage[0][0]);
+    for (uint32_t i = tid; i < kTile / 4u; i += kCmpThreads) st4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint32_t lo = __ldg(b.kv_start + tile), hi = __ldg(b.kv_start + tile + 1u);
+    __syncthreads();
+    const uint32_t base = tile << kGroupLog2;
+    for (uint32_t j = lo + (uint32_t)tid; j < hi; j += kCmpThreads) {
+        const uint32_t k = __ldg(b.kv_keys + j) - base;
+        if (k < kTile) s.stage[0][k] = __ldg(b.kv_vals + j);      // (keys that do not ascend cannot write outside the stage)
+    }
+    __syncthreads();
+}
+
+// The encode pass's "start bringing tile `tile` into the stage": a bulk copy in flight, or (key-value input) the
+// tile formed on the spot.
+template <bool KV>
+__device__ __forceinline__ void load_tile(CmpSmem& s, const CmpBatch& b, const CmpArgs& a, int stage, uint32_t tile,
+                                          uint32_t& pending, int tid) {
+    if constexpr (KV) {
+        kv_fill_tile(s, b, tile, tid);
+    } else {
+        issue_tile(s, a, stage, tile, tid);
+        pending |= 1u << stage;
     }
 }
 
@@ -829,6 +863,56 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
     }
 }
 
+// The sum pass for key-value input (one gradient): tiles above the grid by ticket from the last one down, the
+// block's own tile c last (it stays in the stage for the encode pass).  A tile without entries has partial 0 and
+// is not formed at all; the others are formed in the stage and reduced on the same tree as a copied tile (zeros
+// add exactly nothing), so the sum has the bits of the dense gradient's sum.
+__device__ __forceinline__ void sum_pass_kv(CmpSmem& s, const CmpBatch& b, const CmpArgs& a, uint32_t c, uint32_t grid,
+                                            int tid, int lane, int warp) {
+    for (;;) {
+        if (tid == 0) {
+            const unsigned int tk = atomicAdd(a.ctl->tickets1, 1u);
+            s.p1_next[0] = grid + tk < a.G ? a.G - 1u - tk : c;
+        }
+        __syncthreads();
+        const uint32_t tile = s.p1_next[0];
+        const bool last = tile == c;
+        const bool empty = __ldg(b.kv_start + tile) == __ldg(b.kv_start + tile + 1u);
+        if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }
+        if (empty && !last) {
+            if (tid == 0) { a.partials[tile] = 0.0; a.tmax[tile] = 0.0f; }
+            __syncthreads();                             // (p1_next is rewritten next)
+            continue;
+        }
+        kv_fill_tile(s, b, tile, tid);
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            double x[4];
+            float mx = 0.0f;
+            const float4* row = reinterpret_cast<const float4*>(&s.stage[0][part * (int)(kTile / 2) + warp * 512]) + lane;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float4 v4 = row[r * 32];
+                x[r] = abs_sum4(v4);
+                mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v4.x), fabsf(v4.y)), fmaxf(fabsf(v4.z), fabsf(v4.w))));
+            }
+            const double u = warp_halfslab_tree(x, lane);
+            const uint32_t wmx = __reduce_max_sync(kFullMask, __float_as_uint(mx));
+            if (lane == 0) { s.s_warp[0][part][warp] = u; s.s_wmax[0][part][warp] = wmx; }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            double t0 = lane < kCmpWarps ? s.s_warp[0][0][lane] : 0.0, t1 = lane < kCmpWarps ? s.s_warp[0][1][lane] : 0.0;
+            t0 = warp_tree(t0, kCmpWarps);
+            t1 = warp_tree(t1, kCmpWarps);
+            const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? max(s.s_wmax[0][0][lane], s.s_wmax[0][1][lane]) : 0u);
+            if (lane == 0) { a.partials[tile] = __dadd_rn(t0, t1); a.tmax[tile] = __uint_as_float(tm); }
+        }
+        __syncthreads();                                 // (s_warp and p1_next are rewritten next)
+        if (last) break;
+    }
+}
+
 // Run by one block when a gradient's sum S is known: which tiles does the encode pass have to read?
 // A tile whose largest |v| (recorded by the sum pass) is below the early-stop threshold B_tau holds
 // nothing to keep.  Such a tile gets its descriptor (0 entries, 0 words) here; its directory entry
@@ -983,7 +1067,9 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
 // BIG (one gradient only): the variant for gradients with very many tiles, where the steps that one
 // block does for everybody (reducing the partials, listing the tiles, scanning the descriptors) take
 // forms that cost less per tile and more to start with.
-template <bool SEVERAL, bool BIG = false>
+// KV (one gradient only): the gradient comes as ascending keys with their values; tiles are formed in the stage
+// from the entries (kv_fill_tile) instead of being copied, everything else is the same code.
+template <bool SEVERAL, bool BIG = false, bool KV = false>
 __global__ void __launch_bounds__(kCmpThreads, 2)
 k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
@@ -1043,8 +1129,12 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     if (nown) {
         a = job_view(b, team);
         if (tid == 0) btrace[8u * team + 0] = read_globaltimer();
-        const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
-        sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
+        if constexpr (KV) {
+            sum_pass_kv(s, b, a, c, grid, tid, lane, warp);
+        } else {
+            const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
+            sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
+        }
         if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
         barrier_arrive<BIG>(s, a, pw, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
     }
@@ -1096,10 +1186,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             __syncthreads();
             g = s.next_tile[1];
             have = g < a.G;
-            if (have) {
-                issue_tile(s, a, 0, g, tid);
-                pending |= 1u;
-            }
+            if (have) load_tile<KV>(s, b, a, 0, g, pending, tid);
         }
         const CmpArgs ap = job_view(b, prev_job);
         if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
@@ -1124,7 +1211,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // iteration's first barrier)
             uint32_t tile_ahead = kNoMore;
             if (tid == 0) tile_ahead = ticket_ahead == kNoTicket ? kNoTicket : (ticket_ahead < listed ? __ldcg(a.nelist + ticket_ahead) : kNoMore);
-            if (i > 0u || preloaded) {
+            if (!KV && (i > 0u || preloaded)) {
                 if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
@@ -1238,10 +1325,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             const uint32_t g_next = s.next_tile[par];
             const bool more = g_next < a.G;                  // (false for kNoTicket too)
             if (more) {
-                if (!overflow) {                 // (a tile too dense for the lists packs its blob in the stage first)
-                    issue_tile(s, a, st, g_next, tid);
-                    pending |= 1u << st;
-                }
+                if (!overflow) load_tile<KV>(s, b, a, st, g_next, pending, tid);      // (a tile too dense for the lists packs its blob in the stage first)
                 if (tid == 0) {
                     const bool stop_reserving = overflow || dense_pending ||
                         npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords;
@@ -1354,8 +1438,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 __syncthreads();                     // the stage is free
                 if (more) {                          // (generic-proxy writes before an async-proxy one)
                     if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue_tile(s, a, st, g_next, tid);
-                    pending |= 1u << st;
+                    load_tile<KV>(s, b, a, st, g_next, pending, tid);
                 }
             }
             if (tid == 0) {
@@ -1379,8 +1462,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 g = s.next_tile[par];
                 have = g < a.G;
                 if (have) {
-                    issue_tile(s, a, st, g, tid);
-                    pending |= 1u << st;
+                    load_tile<KV>(s, b, a, st, g, pending, tid);
                     if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
                 if (npend > 0) drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
@@ -1470,6 +1552,20 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             st_release_u32(&b.ctl->bar_gen, gen_next);
         }
     }
+}
+
+// Key-value input, first launch: kv_start[t] = number of entries with key < t * 2^14 (a binary search per
+// tile boundary), t = 0..G.
+__global__ void __launch_bounds__(256) k_kv_bounds(const uint32_t* __restrict__ keys, uint32_t count, uint32_t G, uint32_t* __restrict__ kv_start) {
+    const uint32_t t = blockIdx.x * 256u + threadIdx.x;
+    if (t > G) return;
+    const unsigned long long bound = (unsigned long long)t << kGroupLog2;
+    uint32_t lo = 0, hi = count;                      // first index whose key is >= bound
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if ((unsigned long long)__ldg(keys + mid) < bound) lo = mid + 1u; else hi = mid;
+    }
+    kv_start[t] = lo;
 }
 
 }  // namespace fsg

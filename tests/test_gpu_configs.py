@@ -152,3 +152,25 @@ def test_config2_sparse_adam_update_as_benchmarked():
     assert binding.decode_status() == 0 and not bool(scratch.any().item())
     assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
     assert 0 < int((ot != theta0).sum()) <= 4 * n // 100
+
+
+def test_config3_key_value_input_as_benchmarked():
+    # config 3 is sparse before it is compressed: its non-zero entries as key-value pairs give the dense call's stream
+    wl = workloads.make("c3")
+    n = wl.n
+    v = wl.grads[0]
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg)
+    keys = np.flatnonzero(v)
+    assert 0 < keys.size < n // 500
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    out = torch.full((cap,), 0x5A, dtype=torch.uint8, device="cuda")
+    dk = torch.from_numpy(keys.astype(np.uint32).view(np.int32)).cuda()
+    dv = torch.from_numpy(v[keys]).cuda()
+    orc, ostream = oracle.compress(v, po)
+    for rep in range(2):
+        assert binding.compress_kv(dk, dv, n, pg, out) == 0
+        total, d, status = binding.stream_info(out)
+        assert status == orc == 0 and total == ostream.size
+        assert np.array_equal(out[:total].cpu().numpy(), ostream)

@@ -678,3 +678,64 @@ def test_paper_key_stream_on_compressed_gradient_keys_and_wide_deltas():
     import ctypes as C
     assert binding.lib().fastsgd_key_encode_paper(None, 5, 2, None, 0, None) == binding.E_NULL
     assert binding.key_encode_paper_bound(10, 9) == 0
+
+
+def _check_kv(keys, vals, n, b, l=2, tau=128):
+    """fastsgd_compress_kv against the oracle's stream for the same pairs (= the dense vector's stream)."""
+    import torch
+    import gpu_util as G
+    pg, po = _params(b, tau, l)
+    binding.ensure_workspace(n, pg)
+    orc, ostream = oracle.compress_kv(keys, vals, n, po)
+    buf = G.Guarded(binding.compress_bound(n, pg), fill=0x6B)
+    dk = torch.from_numpy(np.ascontiguousarray(keys, np.uint32).view(np.int32)).to(G.dev())
+    dv = torch.from_numpy(np.ascontiguousarray(vals, np.float32)).to(G.dev())
+    for rep in range(2):
+        assert binding.compress_kv(dk, dv, n, pg, buf.view) == 0
+        total, d, status = binding.stream_info(buf.view)
+        assert status == orc and total == ostream.size and buf.intact(), (status, orc, total, ostream.size)
+        assert np.array_equal(buf.view[:total].cpu().numpy(), ostream), "stream differs"
+    return ostream
+
+
+@pytest.mark.parametrize("tiles", [1, 2, 7, 345, 700])
+@pytest.mark.parametrize("density", [0.0, 3e-5, 1e-3, 0.05])
+def test_key_value_input_equals_the_dense_path(tiles, density):
+    rng = np.random.default_rng(int(tiles * 1000 + density * 1e6))
+    n = tiles * 16384 - int(rng.integers(0, 16000)) if tiles > 1 else 9000
+    cnt = int(density * n)
+    if density == 0.0:
+        cnt = [0, 1, 2, 3][tiles % 4]
+    keys = np.sort(rng.choice(n, size=cnt, replace=False)).astype(np.uint64)
+    vals = (rng.standard_t(3, cnt) * 1e-2).astype(np.float32)
+    if cnt > 10:
+        vals[rng.integers(0, cnt, cnt // 10)] = 0.0                   # pairs with a zero value
+    dense = np.zeros(n, np.float32)
+    dense[keys.astype(np.int64)] = vals
+    b = workloads.base_for_keep(dense, max(1, int(0.7 * np.count_nonzero(dense)))) if np.count_nonzero(dense) else 1.1
+    s = _check_kv(keys, vals, n, b)
+    # and it is the dense call's stream
+    import gpu_util as G
+    pg, _ = _params(b)
+    rc, status, gstream, intact = G.gpu_compress(dense, pg)
+    assert rc == 0 and np.array_equal(gstream, s)
+
+
+def test_key_value_input_with_dense_runs_and_every_flag_size():
+    # runs of consecutive keys (tiles too dense for the per-warp lists), a first key of 0, a last key of n - 1
+    rng = np.random.default_rng(12)
+    n = 9 * 16384 + 77
+    parts = [np.arange(0, 3000), np.arange(16384 * 2 + 100, 16384 * 3 + 900), rng.choice(np.arange(16384 * 5, n - 1), 400, replace=False), [n - 1]]
+    keys = np.unique(np.concatenate(parts)).astype(np.uint64)
+    vals = rng.standard_normal(keys.size).astype(np.float32)
+    dense = np.zeros(n, np.float32)
+    dense[keys.astype(np.int64)] = vals
+    for l in (1, 3, 5):
+        b = workloads.base_for_keep(dense, int(0.9 * keys.size))
+        _check_kv(keys, vals, n, b, l=l)
+    import ctypes as C
+    import torch
+    pg, _ = _params(1.1)
+    out = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    assert binding.lib().fastsgd_compress_kv(None, None, 5, n, C.byref(pg), out.data_ptr(), out.numel(), None) == binding.E_NULL
+    assert binding.lib().fastsgd_compress_kv(None, None, 0, n, C.byref(pg), None, 0, None) == binding.E_NULL

@@ -83,3 +83,26 @@ def test_beta1_one_keeps_the_first_moment_and_errors_update_nothing():
     t2, m2, v2 = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.float32)
     assert oracle.sparse_adam_update([s, bad], n, po, 1.0, 0.5, 0.5, 0.0, t2, m2, v2) != 0
     assert not t2.any() and not m2.any() and not v2.any()
+
+
+def test_key_value_input_has_the_dense_vectors_stream_and_the_plain_sum():
+    # values that are powers of two: the sum is exact in any order, so the header's sum is the plain total
+    po = oracle.params(2.0, 16, 2, 14)
+    n = 3 * 16384 + 9
+    keys = np.array([0, 5, 16383, 16384, 40000, n - 1], np.uint64)
+    vals = np.array([0.5, -0.25, 2.0, 0.0, -8.0, 1.0], np.float32)
+    rc, s = oracle.compress_kv(keys, vals, n, po)
+    assert rc == 0
+    dense = np.zeros(n, np.float32)
+    dense[keys.astype(np.int64)] = vals
+    rc2, s2 = oracle.compress(dense, po)
+    assert rc2 == 0 and np.array_equal(s, s2)
+    rc3, pk, pc, S = oracle.parse(s, n, po)
+    assert rc3 == 0 and S == 11.75
+    assert set(pk.tolist()) <= set(keys[vals != 0].tolist())          # a zero value is never kept
+    # order and range of the keys are part of the contract
+    assert oracle.compress_kv(np.array([5, 5], np.uint64), np.ones(2, np.float32), n, po)[0] != 0
+    assert oracle.compress_kv(np.array([7, 3], np.uint64), np.ones(2, np.float32), n, po)[0] != 0
+    assert oracle.compress_kv(np.array([n], np.uint64), np.ones(1, np.float32), n, po)[0] != 0
+    rc4, s4 = oracle.compress_kv(np.zeros(0, np.uint64), np.zeros(0, np.float32), n, po)
+    assert rc4 == 0 and np.array_equal(s4, oracle.compress(np.zeros(n, np.float32), po)[1])
