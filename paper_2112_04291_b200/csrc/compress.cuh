@@ -871,19 +871,20 @@ __device__ __forceinline__ void sum_pass_kv(CmpSmem& s, const CmpBatch& b, const
                                             int tid, int lane, int warp) {
     for (;;) {
         if (tid == 0) {
-            const unsigned int tk = atomicAdd(a.ctl->tickets1, 1u);
-            s.p1_next[0] = grid + tk < a.G ? a.G - 1u - tk : c;
+            // thread 0 settles the tiles without entries by itself and comes back with the next one that has some
+            uint32_t tile;
+            for (;;) {
+                const unsigned int tk = atomicAdd(a.ctl->tickets1, 1u);
+                tile = grid + tk < a.G ? a.G - 1u - tk : c;
+                a.desc[tile] = 0ull; a.prefix[tile] = 0ull;
+                if (tile == c || __ldg(b.kv_start + tile) != __ldg(b.kv_start + tile + 1u)) break;
+                a.partials[tile] = 0.0; a.tmax[tile] = 0.0f;
+            }
+            s.p1_next[0] = tile;
         }
         __syncthreads();
         const uint32_t tile = s.p1_next[0];
         const bool last = tile == c;
-        const bool empty = __ldg(b.kv_start + tile) == __ldg(b.kv_start + tile + 1u);
-        if (tid == 0) { a.desc[tile] = 0ull; a.prefix[tile] = 0ull; }
-        if (empty && !last) {
-            if (tid == 0) { a.partials[tile] = 0.0; a.tmax[tile] = 0.0f; }
-            __syncthreads();                             // (p1_next is rewritten next)
-            continue;
-        }
         kv_fill_tile(s, b, tile, tid);
 #pragma unroll
         for (int part = 0; part < 2; ++part) {
