@@ -837,8 +837,14 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             s.g_count[tid] = count; s.g_M[tid] = M; s.g_off[tid] = off; s.g_nwords[tid] = nwords;
         }
         __syncthreads();
+        // Model update with the group's slice of the aggregated gradient in shared memory: the streams need not be
+        // parsed again -- the coordinates to update are the non-zeros of the slice.  Thread t looks at entries
+        // t, t + 256, ..., eight at a time, so that the loads of their moments and parameters are in flight together
+        // (neighbouring threads, neighbouring addresses).
+        const bool scan_tile = MODE == 1 && use_tile;
         // staging offsets; a blob that does not fit is parsed from global memory
         uint32_t used = 0;
+        if (!scan_tile)
         for (uint32_t w = 0; w < W; ++w) {
             const uint32_t nw = s.g_count[w] ? s.g_nwords[w] : 0u;
             const bool fits = used + nw <= kBlockStageWords;
@@ -860,6 +866,23 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 continue;
             }
         }
+        if (scan_tile) {
+            for (uint32_t i0 = 0; i0 < span; i0 += 8u * (uint32_t)kDecThreads) {
+                uint32_t kk[8]; float cur[8], vv[8], res[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t idx = i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid;
+                    cur[u] = idx < span ? s.u.tile[idx] : 0.0f;
+                    kk[u] = cur[u] != 0.0f ? lo + idx : 0xFFFFFFFFu;
+                    vv[u] = 0.0f;
+                }
+                apply_run<MODE, 8>(a, kk, cur, vv, res);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (kk[u] != 0xFFFFFFFFu) s.u.tile[i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid] = res[u];
+            }
+            __syncthreads();
+        } else
         for (uint32_t w = 0; w < W; ++w) {
             const uint32_t c = s.g_count[w];
             const uint32_t* blob = s.g_valid[w] ? s.bstage + s.g_base[w]
