@@ -739,3 +739,38 @@ def test_key_value_input_with_dense_runs_and_every_flag_size():
     out = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
     assert binding.lib().fastsgd_compress_kv(None, None, 5, n, C.byref(pg), out.data_ptr(), out.numel(), None) == binding.E_NULL
     assert binding.lib().fastsgd_compress_kv(None, None, 0, n, C.byref(pg), None, 0, None) == binding.E_NULL
+
+
+@pytest.mark.parametrize("keep_div", [500, 40, 3])
+def test_randomly_damaged_streams_report_the_oracles_status(keep_div):
+    # seeded random damage (one to three bytes anywhere in the stream, header and directory included) on sparse,
+    # medium and dense streams: the decoder reports exactly the oracle's status and never leaves its buffers
+    import gpu_util as G
+    n = 6 * 16384 + 321
+    rng = np.random.default_rng(900 + keep_div)
+    v = workloads.student_t_layers(n, seed=keep_div, blocks=5, lo=1e-3, hi=1e-1)
+    b = workloads.base_for_keep(v, n // keep_div)
+    pg, po = _params(b)
+    orc, st0 = oracle.compress(v, po)
+    assert orc == 0
+    fixed = 64 + 8 * 7
+    seen = set()
+    for case in range(60):
+        s = st0.copy()
+        region = case % 3                      # header, directory, blobs
+        for _ in range(int(rng.integers(1, 4))):
+            if region == 0:
+                pos = int(rng.integers(0, 64))
+            elif region == 1:
+                pos = int(rng.integers(64, fixed))
+            else:
+                pos = int(rng.integers(fixed, st0.size))
+            s[pos] ^= np.uint8(rng.integers(1, 256))
+        expect = oracle.decompress_accumulate(s, n, po, np.zeros(n, np.float32))
+        rc, st, dense, intact = G.gpu_decompress(s, n, pg)
+        assert rc == 0 and intact, case
+        assert st == expect, (case, st, expect)
+        seen.add(st)
+    assert len(seen) >= 3                      # several different outcomes, a sound decode among them or not
+    rc, st, dense, intact = G.gpu_decompress(st0, n, pg)
+    assert rc == 0 and st == 0 and intact
