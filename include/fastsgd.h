@@ -128,7 +128,7 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
 /*
  * The encoder for a gradient given as key-value pairs (Sec. 2.2 states the
  * problem on the D non-zero pairs (k_j, v_j) of a D_m-dimensional gradient;
- * the sparse models of Sec. 5 produce it in this form).
+ * the sparse models of Sec. 4 produce it in this form).
  *   keys    device, `count` strictly ascending 32-bit keys, each < n
  *   values  device, the matching fp32 values (zeros allowed: never kept)
  *   n       D_m; out, out_bytes, params, stream as for fastsgd_compress
@@ -175,9 +175,9 @@ int fastsgd_decompress_accumulate_batch(const void* const* streams_in, const uin
                                         float* dense_out, void* stream);
 
 /*
- * Model update on the decoded coordinates only (Sec. 5.1, "Implementation":
+ * Model update on the decoded coordinates only (Sec. 4.1, "Implementation":
  * the models are trained with Adam; Table of the running-time breakdown, part
- * "model updating").  Hyper-parameters of the two Adam equations of Sec. 5.1.
+ * "model updating").  Hyper-parameters of the two Adam equations of Sec. 4.1.
  */
 typedef struct fastsgd_adam {
     float lr;      /* eta */

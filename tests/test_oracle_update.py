@@ -1,4 +1,4 @@
-"""Pins of the oracle's model update on decoded coordinates (Sec. 5.1: the two Adam equations
+"""Pins of the oracle's model update on decoded coordinates (Sec. 4.1: the two Adam equations
 as printed, applied where the aggregated decoded gradient is non-zero).  Streams are built with
 b = 2 and sum = 1, so that a code L decodes to exactly 2^-L."""
 import numpy as np
