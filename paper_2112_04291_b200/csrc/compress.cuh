@@ -84,7 +84,7 @@ struct CmpSmem {
     uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
     double   job_sum[2];                     // by gradient parity: its sum
     double   s_nodes[256];                   // nodes of the final sum tree when a thread holds more than 8 partials
-    uint32_t pad5;
+    uint32_t pad5;                           // (scratch flag of the shared descriptor scan)
     uint32_t publisher;                      // this block was the last to finish the gradient's encode pass
     uint32_t team;                           // which of the two teams of blocks this one belongs to
     uint32_t last_arrival;                   // this block was the last to arrive at a grid barrier
@@ -759,6 +759,108 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
         }
         __syncthreads();
     }
+}
+
+// The same scan shared among the first blocks to finish the encode pass (kernel variant for very many tiles:
+// one block scanning 16384 descriptors or more takes tens of microseconds at the very end of the launch).
+// Block number `part` of `parts` takes a contiguous segment of the descriptors: it adds the segment up,
+// following descriptors that are not published yet (bounded polls), publishes the segment's total, takes
+// the totals of the segments before it (published the same way: bounded polls; nobody waits for a later
+// segment, so there is no cycle), then scans its segment once more from that base and writes the prefixes
+// and the directory entries of the groups without kept entries.  A descriptor that is not valid poisons
+// the prefixes of its segment and of every later one.
+constexpr uint32_t kScanParts = 16;
+__device__ __forceinline__ unsigned long long scan_segment(CmpSmem& s, const CmpArgs& a, uint32_t beg, uint32_t end, unsigned long long running,
+                                                          bool store, bool& bad, int tid, int lane, int warp) {
+    const uint32_t fixed_words = (kHeaderBytes + 8u * a.G) >> 2;
+    uint32_t* outw = reinterpret_cast<uint32_t*>(a.out);
+    for (uint32_t pos = beg; pos < end; pos += (uint32_t)kDrainChunks * kCmpThreads) {
+        unsigned long long own[kDrainChunks], excl[kDrainChunks];
+        bool bad_here = false;
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+            own[j] = idx < end ? ld_relaxed_u64(a.desc + idx) : desc_pack(kDescValid, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            if (!store && !bad) {
+                const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+                uint32_t spin = 0;
+                while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
+                    if (++spin > kWaitLimit) break;
+                    if (spin > 32u) __nanosleep(32);
+                    own[j] = ld_relaxed_u64(a.desc + idx);
+                }
+            }
+            if ((own[j] >> 62) != kDescValid) { bad_here = true; own[j] = 0ull; }
+            own[j] = ((unsigned long long)desc_count(own[j]) << 32) | desc_words(own[j]);
+            unsigned long long incl = own[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long u = __shfl_up_sync(kFullMask, incl, o);
+                if (lane >= o) incl += u;
+            }
+            if (lane == 31) s.scan64[j][warp] = incl;
+            excl[j] = incl - own[j];
+        }
+        if (__syncthreads_or(bad_here ? 1 : 0)) bad = true;
+#pragma unroll
+        for (int j = 0; j < kDrainChunks; ++j) {
+            unsigned long long before = running, all = 0ull;
+#pragma unroll
+            for (int w = 0; w < kCmpWarps; ++w) {
+                const unsigned long long u = s.scan64[j][w];
+                if (w < warp) before += u;
+                all += u;
+            }
+            excl[j] += before;
+            running += all;
+            const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
+            if (store && idx < end) {
+                st_relaxed_u64(a.prefix + idx, bad ? desc_pack(kDescPoison, 0, 0)
+                                                   : desc_pack(kDescValid, (uint32_t)(excl[j] >> 32), (uint32_t)excl[j]));
+                if (!bad && (own[j] >> 32) == 0ull) {
+                    outw[(kHeaderBytes >> 2) + 2u * idx]      = 0u;
+                    outw[(kHeaderBytes >> 2) + 2u * idx + 1u] = fixed_words + (uint32_t)excl[j];
+                }
+            }
+        }
+        __syncthreads();
+    }
+    return running;
+}
+
+__device__ __forceinline__ void publish_part(CmpSmem& s, const CmpArgs& a, unsigned long long* segtot, uint32_t part, uint32_t parts,
+                                             int tid, int lane, int warp) {
+    constexpr uint32_t kStepAll = (uint32_t)kDrainChunks * kCmpThreads;
+    const uint32_t seg = ((a.G + parts - 1u) / parts + kStepAll - 1u) / kStepAll * kStepAll;
+    const uint32_t beg = min(part * seg, a.G), end = min(beg + seg, a.G);
+    bool bad = false;
+    const unsigned long long total = scan_segment(s, a, beg, end, 0ull, false, bad, tid, lane, warp);
+    if (tid == 0) st_relaxed_u64(segtot + part, bad ? desc_pack(kDescPoison, 0, 0) : desc_pack(kDescValid, (uint32_t)(total >> 32), (uint32_t)total));
+    // the segments before this one
+    if (tid < (int)kScanParts) s.scan64[0][tid] = 0ull;
+    if (tid == 0) s.pad5 = 0u;                          // (set below if one of them is poisoned)
+    __syncthreads();
+    if (tid < (int)part) {
+        unsigned long long v = ld_relaxed_u64(segtot + tid);
+        uint32_t spin = 0;
+        while ((v >> 62) == kDescInvalid) {
+            if (++spin > kWaitLimit) break;
+            if (spin > 32u) __nanosleep(32);
+            v = ld_relaxed_u64(segtot + tid);
+        }
+        if ((v >> 62) != kDescValid) s.pad5 = 1u;
+        s.scan64[0][tid] = ((unsigned long long)desc_count(v) << 32) | desc_words(v);
+    }
+    __syncthreads();
+    unsigned long long base = 0ull;
+#pragma unroll
+    for (int w = 0; w < (int)kScanParts; ++w) base += s.scan64[0][w];
+    if (s.pad5) bad = true;
+    __syncthreads();
+    scan_segment(s, a, beg, end, base, true, bad, tid, lane, warp);
 }
 
 // Phase 1 for one gradient: fp64 partial sum of every 2^14-entry tile.  Tiles grid..G-1 are handed
@@ -1483,14 +1585,20 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 const unsigned int old = atom_add_acq_rel_u32(a.enc_done, 1u);      // this block's descriptors before its count
                 if (old == enc_expect - 1u) *a.enc_done = 0u;
                 // the launch's last gradient: the first block through follows the others; else the last one scans
-                s.publisher = (job == H ? old == 0u : old == enc_expect - 1u) ? 1u : 0u;
+                if constexpr (BIG) s.publisher = old < min(kScanParts, enc_expect) ? old + 1u : 0u;      // (one gradient: the first blocks through share the scan)
+                else s.publisher = (job == H ? old == 0u : old == enc_expect - 1u) ? 1u : 0u;
             }
         }
         __syncthreads();
         if (s.publisher) {
-            // (following the others: small steps, so that what is complete is published at once; with very many tiles large steps)
-            if (job == H) publish_prefixes<true, BIG ? kDrainChunks : 1>(s, a, tid, lane, warp);
-            else publish_prefixes<false, kDrainChunks>(s, a, tid, lane, warp);
+            if constexpr (BIG) {
+                // (the per-SM counters of the two-team launches are not in use here: their place holds the segment totals)
+                publish_part(s, a, reinterpret_cast<unsigned long long*>(b.sm_slots), s.publisher - 1u, min(kScanParts, enc_expect), tid, lane, warp);
+            } else {
+                // (following the others: small steps, so that what is complete is published at once)
+                if (job == H) publish_prefixes<true, 1>(s, a, tid, lane, warp);
+                else publish_prefixes<false, kDrainChunks>(s, a, tid, lane, warp);
+            }
         }
         // place what the previous gradient left behind; what this one leaves waits for the next turn
         if (!aborted && nprev > 0) {
@@ -1550,6 +1658,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         if (old == gridDim.x - 1u) {
             b.ctl->exit_count = 0u;
             if (b.teams == 2u) for (int i = 0; i < 256; ++i) b.sm_slots[i] = 0u;
+            if constexpr (BIG) for (int i = 0; i < 2 * (int)kScanParts; ++i) b.sm_slots[i] = 0u;
             st_release_u32(&b.ctl->bar_gen, gen_next);
         }
     }
