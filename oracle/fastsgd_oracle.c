@@ -87,31 +87,34 @@ uint32_t fsgo_quantise(double a, const double *B, uint32_t tau)
     return tau + 1;
 }
 
-/* ---------------------------------------------------------- Algorithm 1 */
+/* ------------------------------------------- gradient value encoder (Sec. 3.2)
+ * By the definitions: S is the sum of all magnitudes (numerator of Eq. 2); an
+ * entry is kept iff its code L = ceil(log_b(S/|v|)) (Eq. 3 on Eq. 2) does not
+ * exceed tau, which is the test |v| >= S / b^tau (the early-stop threshold);
+ * the kept code carries the sign of the value. */
 
 int fsgo_value_encode(const float *v, uint64_t n, double base, uint32_t tau,
                       uint64_t *keys, int32_t *codes, uint64_t *d, double *sum)
 {
     double P[129], B[129];
     *d = 0;
-    double s = fsgo_abs_sum(v, n);
-    *sum = s;
-    int rc = fsgo_tables(s, base, tau, P, B);
+    const double S = fsgo_abs_sum(v, n);
+    *sum = S;
+    int rc = fsgo_tables(S, base, tau, P, B);
     if (rc) return rc;
-    if (!isfinite(s)) return FSGO_ERR_NONFINITE;
-    double tau_e = B[tau];                       /* early-stop threshold */
-    uint64_t cnt = 0;
-    for (uint64_t j = 0; j < n; ++j) {
-        double a = (double)fabsf(v[j]);
-        if (a > 0.0 && a >= tau_e) {
-            uint32_t L = fsgo_quantise(a, B, tau);   /* <= tau here */
-            if (L == 0) L = 1;                       /* keeps the sign, still an underestimate */
-            keys[cnt]  = j;
-            codes[cnt] = (v[j] < 0.0f) ? -(int32_t)L : (int32_t)L;
-            ++cnt;
-        }
+    if (!isfinite(S)) return FSGO_ERR_NONFINITE;
+    uint64_t kept = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const double mag = (double)fabsf(v[i]);
+        if (!(mag > 0.0)) continue;                  /* zeros (and only zeros) have no reciprocal */
+        uint32_t L = fsgo_quantise(mag, B, tau);     /* tau + 1 when the entry falls below B[tau] */
+        if (L > tau) continue;                       /* threshold filter */
+        if (L < 1) L = 1;                            /* |v| = S: keeps the sign, still an underestimate */
+        keys[kept]  = i;
+        codes[kept] = (v[i] < 0.0f) ? -(int32_t)L : (int32_t)L;
+        ++kept;
     }
-    *d = cnt;
+    *d = kept;
     return FSGO_OK;
 }
 
@@ -160,24 +163,25 @@ static int64_t put_chars(char *bk, uint64_t cap, int64_t pos, uint64_t value, ui
     return pos + nbits;
 }
 
+/* Sec. 3.3 by its definitions: the delta keys are the adjacent differences of
+ * the ascending keys with the first taken from 0 (Eq. 4); M is the bit length of
+ * the largest of them; BK is, key after key, the length flag followed by the
+ * delta in the width that flag selects. */
 int64_t fsgo_key_encode_paper(const uint64_t *keys, uint64_t d, uint32_t l,
                               char *bk, uint64_t cap, uint32_t *M_out)
 {
     uint64_t *delta = (uint64_t *)malloc((d ? d : 1) * sizeof(uint64_t));
-    uint64_t preKey = 0, maxDelta = 0;
-    for (uint64_t j = 0; j < d; ++j) {
-        delta[j] = keys[j] - preKey;
-        preKey = keys[j];
-        if (maxDelta < delta[j]) maxDelta = delta[j];
-    }
-    uint32_t M = fsgo_bitlen(maxDelta);
+    for (uint64_t j = 0; j < d; ++j) delta[j] = keys[j] - (j ? keys[j - 1] : 0u);
+    uint64_t widest = 0;
+    for (uint64_t j = 0; j < d; ++j) if (delta[j] > widest) widest = delta[j];
+    uint32_t M = fsgo_bitlen(widest);
     if (M < 1) M = 1;
     *M_out = M;
     uint32_t widths[32];
     fsgo_widths(M, l, widths);
     int64_t pos = 0;
     for (uint64_t j = 0; j < d && pos >= 0; ++j) {
-        uint32_t flag = fsgo_length_flag(delta[j], widths, l);
+        const uint32_t flag = fsgo_length_flag(delta[j], widths, l);
         pos = put_chars(bk, cap, pos, flag, l);
         if (pos >= 0) pos = put_chars(bk, cap, pos, delta[j], widths[flag]);
     }

@@ -75,6 +75,62 @@ def _run_batched(wl):
     assert np.array_equal(got, odense)
 
 
+def _run_batched_checked(wl, check_workers):
+    """All W gradients in ONE fastsgd_compress_batch launch and all W streams in ONE
+    fastsgd_decompress_accumulate_batch launch (what bench.py times); the streams of `check_workers` are
+    compared byte for byte with the oracle's, the dense sum with the oracle's over all W workers."""
+    n, W = wl.n, wl.workers
+    pg = binding.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    po = oracle.params(wl.base, wl.tau, wl.flag_bits, wl.group_log2)
+    binding.ensure_workspace(n, pg)
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    grads = [torch.from_numpy(g).cuda() for g in wl.grads]
+    outs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(W)]
+    for o in outs:
+        o.fill_(0x3C)
+    assert binding.compress_batch(grads, pg, outs) == 0
+    dense = torch.zeros(n, dtype=torch.float32, device="cuda")
+    assert binding.decompress_accumulate_batch(outs, [cap] * W, n, pg, dense) == 0
+    assert binding.decode_status() == 0
+    del grads
+    odense = np.zeros(n, np.float32)
+    for w in range(W):
+        total, d, status = binding.stream_info(outs[w])
+        orc, ostream = oracle.compress(wl.grads[w], po)
+        assert status == orc == 0 and total == ostream.size, f"worker {w}"
+        assert d == int(np.frombuffer(ostream[24:32].tobytes(), np.uint64)[0])
+        if w in check_workers:
+            assert np.array_equal(outs[w][:total].cpu().numpy(), ostream), f"worker {w}: stream differs"
+        assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+    got = dense.cpu().numpy()
+    assert np.allclose(got, odense, rtol=RTOL, atol=ATOL)
+    assert np.array_equal(got, odense)
+
+
+_C4_GRADS = {}
+
+
+def _config4_eight_workers(keep):
+    """Config 4 with its 8 workers; the gradients are drawn once per test session and shared by the keep ratios."""
+    if "grads" not in _C4_GRADS:
+        _C4_GRADS["grads"] = workloads.make("c4", workers=8, keep=1e-3).grads
+    grads = _C4_GRADS["grads"]
+    n = grads[0].size
+    base = workloads.base_for_keep(grads[0], int(round(keep * n)))
+    return workloads.Workload("c4", n, 8, float(keep), grads, base)
+
+
+@pytest.mark.parametrize("keep", [1e-4, 1e-2])
+def test_config4_eight_workers_one_launch_as_benchmarked(keep):
+    # the launch bench.py times for config 4: 8 gradients of 335 M entries in one k_compress launch, 8 streams in one
+    # decoder launch; three streams compared byte for byte, the dense sum over all eight
+    wl = _config4_eight_workers(keep)
+    assert wl.n == 335_141_888 and wl.workers == 8
+    _run_batched_checked(wl, check_workers=(0, 3, 7))
+    if keep == 1e-2:
+        _C4_GRADS.clear()
+
+
 def test_config1_full():
     wl = workloads.make("c1")
     kept = _run(wl)
@@ -121,8 +177,16 @@ def test_config5_sweep(log2n, keep):
     _run(wl)
 
 
-def test_config5_sweep_largest():
-    wl = workloads.make("c5", n=1 << 30, keep=1e-3)
+@pytest.mark.parametrize("keep", [1e-4, 1e-3, 1e-2, 1e-1])
+def test_config5_sweep_2_28(keep):
+    # n = 2^28: the kernel variant for gradients with more than 8192 tiles, at all four keep ratios
+    # (10 %: every tile of the launch goes through the dense-tile packer)
+    _run(workloads.make("c5", n=1 << 28, keep=keep))
+
+
+@pytest.mark.parametrize("keep", [1e-3, 1e-1])
+def test_config5_sweep_largest(keep):
+    wl = workloads.make("c5", n=1 << 30, keep=keep)
     _run(wl)
 
 

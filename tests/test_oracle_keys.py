@@ -103,10 +103,10 @@ def test_single_group_stream_is_algorithm2_with_planes(l):
 
 @pytest.mark.parametrize("glog", [2, 3, 4])
 def test_round_trip_all_subsets(glog):
-    # Keys must come back exactly (Sec. 3.3: the key codec is lossless): every subset of
-    # {0..n-1} for n <= 12 (n = 16 sampled), groups of 4, 8 and 16 indices.
+    # Keys must come back exactly (Sec. 3.3: the key codec is lossless): every non-empty subset of
+    # {0..n-1} for n = 1, 5, 12 and 16 (65,535 subsets), groups of 4, 8 and 16 indices.
     p = oracle.params(1.1, 128, 2, glog)
-    for n in (1, 5, 12):
+    for n in (1, 5, 12, 16):
         for mask in range(1, 1 << n):
             keys = [i for i in range(n) if mask >> i & 1]
             codes = [(-1) ** i * (1 + (i * 37) % 128) for i in keys]
@@ -114,12 +114,6 @@ def test_round_trip_all_subsets(glog):
             assert rc == 0
             rc, k2, c2, S = oracle.parse(stream, n, p)
             assert rc == 0 and k2.tolist() == keys and c2.tolist() == codes and S == 2.5
-    rng = np.random.default_rng(glog)
-    for mask in rng.integers(1, 1 << 16, 3000).tolist():
-        keys = [i for i in range(16) if mask >> i & 1]
-        rc, stream = oracle.write_stream(keys, [1] * len(keys), 16, 1.0, p)
-        rc, k2, c2, S = oracle.parse(stream, 16, p)
-        assert rc == 0 and k2.tolist() == keys
 
 
 @pytest.mark.parametrize("l", [1, 2, 3, 4, 5])

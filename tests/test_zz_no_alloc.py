@@ -5,7 +5,9 @@ cudaMalloc (device-wide synchronisation, failure under memory pressure) and own 
 so they cannot register a workspace either.  For them the entry point keeps its scratch in a
 fixed array inside the library.  This test calls it through the C ABI, twice in a row with
 different inputs, and checks each result against the regular entry point (which uses the
-caller's workspace): the sums must be the same fp64 bits, as everywhere else in this suite.
+caller's workspace) and against the CPU oracle's tree sum: the sums must be the same fp64 bits,
+as everywhere else in this suite.  The largest accepted size (every partial of the built-in
+array in use) and a single-chunk input are covered too.
 
 Collected last (file name) so that a run that stops at the first failure has run everything else.
 It does not depend on any other test: it passes alone in a fresh process too.
@@ -14,6 +16,9 @@ import ctypes as C
 
 import numpy as np
 import pytest
+
+import oracle
+from paper_2112_04291_b200 import binding
 
 pytestmark = pytest.mark.gpu
 
@@ -45,7 +50,19 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
         v = (rng.standard_normal(n) * 10.0 ** rng.integers(-6, 3, n)).astype(np.float32)
         new, old = _sum_both_ways(v)
         assert new == old                       # same fp64 value, bit for bit
+        assert new == oracle.abs_sum(v)         # ... and the oracle's tree sum, directly
         assert abs(new - float(np.abs(v).astype(np.float64).sum())) <= 1e-9 * new
+
+
+def test_largest_accepted_size_and_a_single_chunk():
+    # n = 2^28 uses all 16384 partials of the built-in array; n <= 2^14 is one chunk (a grid of one block)
+    rng = np.random.default_rng(77)
+    for n in (binding.NOALLOC_MAX_N, 16_384, 9_001):
+        v = rng.standard_normal(n, dtype=np.float32)
+        v[::7] *= np.float32(1e-4)
+        new, old = _sum_both_ways(v)
+        assert new == old == oracle.abs_sum(v)
+        del v
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
@@ -61,3 +78,10 @@ def test_sizes_beyond_the_built_in_scratch_are_refused():
     assert "2^28" in binding.strerror(rc)
     assert lib.fastsgd_abs_sum_noalloc(None, C.c_uint64(16), C.c_void_p(out.data_ptr()), stream) == binding.E_NULL
     assert lib.fastsgd_abs_sum_noalloc(C.c_void_p(g.data_ptr() + 4), C.c_uint64(8), C.c_void_p(out.data_ptr()), stream) == binding.E_ALIGN
+    # a refused call leaves nothing behind: the next accepted call on the same stream is exact
+    v = np.linspace(-3.0, 5.0, 40_003, dtype=np.float32)
+    gv = torch.from_numpy(v).cuda()
+    rc = lib.fastsgd_abs_sum_noalloc(C.c_void_p(gv.data_ptr()), C.c_uint64(v.size), C.c_void_p(out.data_ptr()), stream)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert out.item() == oracle.abs_sum(v)
