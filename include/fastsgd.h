@@ -52,7 +52,7 @@ typedef struct fastsgd_params {
     double   base;        /* b > 1, with b^tau finite (Eq. 3)                        */
     uint32_t tau;         /* threshold, 1..128: kept codes L satisfy 1 <= L <= tau    */
     uint32_t flag_bits;   /* l, 1..5: size of the length flag (Sec. 3.3, Phase 5)     */
-    uint32_t group_log2;  /* log2 of the group size T; this build supports 14        */
+    uint32_t group_log2;  /* log2 of the group size T, 8..20 (see fastsgd_compress); 14 is the fast path */
     uint32_t reserved;    /* must be 0                                               */
 } fastsgd_params;
 
@@ -73,7 +73,7 @@ typedef struct fastsgd_params {
 #define FASTSGD_ST_OK              0
 #define FASTSGD_ST_NONFINITE       1     /* compress: sum of |v| is Inf or NaN                               */
 #define FASTSGD_ST_CAPACITY        2     /* compress: stream does not fit in out_bytes                       */
-#define FASTSGD_ST_TIMEOUT         3     /* compress: a bounded wait between thread blocks ran out (see below) */
+#define FASTSGD_ST_TIMEOUT         3     /* a bounded wait between thread blocks ran out (see fastsgd_compress) */
 #define FASTSGD_ST_BAD_MAGIC      16
 #define FASTSGD_ST_BAD_VERSION    17
 #define FASTSGD_ST_BAD_STATUS     18     /* decompress: the stream's own status is not OK                    */
@@ -102,11 +102,21 @@ typedef struct fastsgd_params {
  * If the stream does not fit, or the sum is not finite, only a 64-byte header
  * carrying the status is written.  Nothing outside out[0, out_bytes) is
  * written.
+ * Group sizes: T = 2^14 is what the fused kernel is built for (its tile is the
+ * group).  Any other group_log2 in 8..20 takes a general path -- the sum kernel,
+ * then the list encoder of fastsgd_compress_kv run over the dense gradient, two
+ * launches per gradient and three reads of it -- with the same stream as the
+ * definition gives (the paper's Algorithm 2 has no groups: it is the case
+ * T >= n).  Below 2^8: FASTSGD_E_NOT_IMPLEMENTED.  The decoder takes the same
+ * range as long as the stream has at most 2^17 groups.
  * The kernel is launched cooperatively (all its thread blocks resident at
  * once, two per SM) and its blocks wait for one another with bounded waits; if
  * one of them runs out (it should not on a GPU the kernel has to itself) every
  * stream of that launch reports FASTSGD_ST_TIMEOUT, and the workspace must be
- * registered again before the next call.
+ * registered again before the next call: once fastsgd_stream_info or
+ * fastsgd_decode_status has returned that status, every compress and
+ * decompress call fails with FASTSGD_E_NO_WORKSPACE until
+ * fastsgd_set_workspace is called again.
  */
 int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
                      void* out, uint64_t out_bytes, void* stream);
@@ -135,10 +145,13 @@ int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_
  * The stream is, byte for byte, the one fastsgd_compress writes for the dense
  * vector that holds values[j] at keys[j] and zeros elsewhere: the sum is
  * formed on the same tree (zeros add exactly nothing), the groups are the
- * same.  Nothing of size n is read or written except the per-group tables of
- * the workspace: cost in proportion to count and to n / 2^14.  Keys that do
- * not ascend or reach n give an unspecified stream, never an access outside
- * the buffers.  Two launches (tile boundaries; the fused kernel).
+ * same.  Nothing of size n is read, formed or written except the directory
+ * (8 bytes per group) and one pass over the per-chunk sums (8 bytes per 2^14
+ * indices): cost in proportion to count and to n / 2^14.  Any group_log2 in
+ * 1..20.  Keys that do not ascend or reach n give an unspecified stream, never
+ * an access outside the buffers.  One cooperative launch (a warp per 32 pairs;
+ * two grid barriers with bounded waits, FASTSGD_ST_TIMEOUT as for
+ * fastsgd_compress).
  */
 int fastsgd_compress_kv(const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
                         const fastsgd_params* params, void* out, uint64_t out_bytes, void* stream);
@@ -316,17 +329,6 @@ int fastsgd_decompress_accumulate_host(const void* const* streams_host, const ui
                                        uint32_t num_streams, uint64_t n, const fastsgd_params* params,
                                        float* dense_host, int accumulate, int* status,
                                        void* dev_scratch, uint64_t dev_scratch_bytes, void* stream);
-
-/* Profiling aid.  While enabled, every kernel launch is bracketed by a pair of
- * CUDA events recorded on its stream.  fastsgd_kernel_timing_read synchronises
- * those events, adds up the elapsed milliseconds and the launches per kernel
- * (index 0 abs-sum, 1 encode, 2 decode-accumulate) since the last read, and
- * forgets them.  Off by default; the events add a little launch overhead. */
-int fastsgd_kernel_timing_enable(int enable);
-int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]);
-
-/* number of kernels the library has launched since it was loaded */
-uint64_t fastsgd_launch_count(void);
 
 const char* fastsgd_strerror(int code);
 int fastsgd_version(void);

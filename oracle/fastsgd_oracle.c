@@ -107,8 +107,8 @@ int fsgo_value_encode(const float *v, uint64_t n, double base, uint32_t tau,
     for (uint64_t i = 0; i < n; ++i) {
         const double mag = (double)fabsf(v[i]);
         if (!(mag > 0.0)) continue;                  /* zeros (and only zeros) have no reciprocal */
-        uint32_t L = fsgo_quantise(mag, B, tau);     /* tau + 1 when the entry falls below B[tau] */
-        if (L > tau) continue;                       /* threshold filter */
+        if (!(mag >= B[tau])) continue;              /* threshold filter: L <= tau iff |v| >= S / b^tau */
+        uint32_t L = fsgo_quantise(mag, B, tau);
         if (L < 1) L = 1;                            /* |v| = S: keeps the sign, still an underestimate */
         keys[kept]  = i;
         codes[kept] = (v[i] < 0.0f) ? -(int32_t)L : (int32_t)L;

@@ -30,6 +30,7 @@ EXPORTS = [
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
     "fastsgd_sparse_adam_update_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
     "fastsgd_compress_kv",
+    "fastsgd_debug_set_wait_limits", "fastsgd_debug_layout", "fastsgd_debug_trace_compiled",
 ]
 
 
@@ -112,6 +113,12 @@ def lib():
         L.fastsgd_kernel_timing_enable.argtypes = [C.c_int]
         L.fastsgd_kernel_timing_read.restype = C.c_int
         L.fastsgd_kernel_timing_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+        L.fastsgd_debug_set_wait_limits.restype = C.c_int
+        L.fastsgd_debug_set_wait_limits.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32]
+        L.fastsgd_debug_layout.restype = C.c_int
+        L.fastsgd_debug_layout.argtypes = [u64p, C.c_uint32]
+        L.fastsgd_debug_trace_compiled.restype = C.c_int
+        L.fastsgd_debug_trace_compiled.argtypes = []
         _lib = L
     return _lib
 
@@ -310,25 +317,48 @@ def kernel_timing_read():
     return {k: (ms[i], int(cnt[i])) for i, k in enumerate(KERNELS)}
 
 
-def debug_trace():
-    """Block 0's %globaltimer stamps (ns) for the first gradient of the last compress launch: start,
-    end of the sum pass, grid barrier passed, boundary table ready, end of the encode pass.
-    Profiling aid read straight from the registered workspace tensor; synchronises."""
-    t = debug_trace_blocks(1)
-    if t is None:
-        return None
-    r = t[0, 0]
-    return [int(r[0]), int(r[1]), int(r[3]), int(r[4]), int(r[5])]
+def debug_set_wait_limits(block_polls: int = 0, copy_tries: int = 0, queue_polls: int = 0) -> None:
+    """fastsgd_debug_set_wait_limits: shorten (or, with zeros, restore) the kernels' bounded waits.  Test aid."""
+    _check(lib().fastsgd_debug_set_wait_limits(int(block_polls), int(copy_tries), int(queue_polls)),
+           "fastsgd_debug_set_wait_limits")
+
+
+LAYOUT_FIELDS = ("bar_count", "ne_count", "error", "decoder_trace", "encoder_trace", "encoder_trace_bytes",
+                 "queue_slots", "queue_counters")
+
+
+def debug_layout() -> dict:
+    """fastsgd_debug_layout: byte offsets of a few fields inside the registered workspace."""
+    v = (C.c_uint64 * len(LAYOUT_FIELDS))()
+    _check(lib().fastsgd_debug_layout(v, len(LAYOUT_FIELDS)), "fastsgd_debug_layout")
+    return {k: int(v[i]) for i, k in enumerate(LAYOUT_FIELDS)}
+
+
+def workspace_u32(field: str, count: int):
+    """`count` 32-bit words of the registered workspace at a field of debug_layout(), as a torch view
+    (reads and writes go to device memory; synchronise before relying on them)."""
+    ws = _workspace_keepalive
+    assert ws is not None, "no workspace registered through this module"
+    off = debug_layout()[field]
+    return ws[off:off + 4 * count].view(torch.int32)
+
+
+def listed_tiles(jobs: int):
+    """Tiles the encode pass of the last fastsgd_compress(_batch) launch read a second time, per gradient
+    (the others held nothing to keep, or were still in shared memory).  Synchronises."""
+    torch.cuda.synchronize()
+    return [int(x) for x in workspace_u32("ne_count", 8)[:jobs].cpu().tolist()]
 
 
 def debug_trace_blocks(blocks: int = 148):
     """Per-block stamps (ns, %globaltimer) of the last compress launch, shape (blocks, 8, 8): for
     each block and each gradient of the launch: start, end of the sum pass, previous gradient's
     pending tiles placed, grid barrier passed, table ready, end of the encode loop; slot 6 of
-    gradient 0 holds the end of the launch's last drain.  Profiling aid; synchronises."""
+    gradient 0 holds the end of the launch's last drain.  Only a library built with -DFASTSGD_TRACE
+    writes them (None otherwise); synchronises."""
     ws = _workspace_keepalive
-    if ws is None:
+    if ws is None or not lib().fastsgd_debug_trace_compiled():
         return None
     torch.cuda.synchronize()
-    off = 32768 + (4 << 17)
+    off = debug_layout()["encoder_trace"]
     return ws[off:off + 512 * blocks].cpu().numpy().view("<u8").reshape(blocks, 8, 8).astype("int64")

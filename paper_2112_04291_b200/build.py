@@ -29,11 +29,15 @@ def _deps():
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    """Compiles the library if it is missing or older than its sources.  With FASTSGD_TRACE=1 in the
+    environment the kernels are built with their %globaltimer phase stamps (a profiling build: force it,
+    and force a plain build afterwards)."""
     stale = (not os.path.exists(LIB_PATH)) or any(
         os.path.getmtime(d) > os.path.getmtime(LIB_PATH) for d in _deps())
     if force or stale:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", LIB_PATH, *sources()]
+        trace = ["-DFASTSGD_TRACE"] if os.environ.get("FASTSGD_TRACE") == "1" else []
+        cmd = [nvcc, *NVCC_FLAGS, *trace, *(["-Xptxas", "-v"] if verbose else []), "-o", LIB_PATH, *sources()]
         subprocess.check_call(cmd)
     return LIB_PATH
 

@@ -1,6 +1,7 @@
 // C-ABI shim: argument checks, workspace bookkeeping and kernel launches on the caller's
 // stream.  No computation of the path happens here except the parameter-only table b^k.
 #include "../../include/fastsgd.h"
+#include "../../include/fastsgd_debug.h"
 
 #include <atomic>
 #include <cmath>
@@ -13,6 +14,7 @@
 #include "bits.cuh"
 #include "compress.cuh"
 #include "keys_paper.cuh"
+#include "kv.cuh"
 #include "decode.cuh"
 
 namespace {
@@ -28,7 +30,12 @@ struct State {
     int        sum_blocks_per_sm = 0;
     int        dec_blocks_per_sm = 0;
     int        cmp_blocks_per_sm = 0;
+    int        kv_blocks_per_sm = 0;
     bool       attrs_set = false;
+    bool       timed_out = false;          // a status query saw FASTSGD_ST_TIMEOUT: the workspace's counters are not at rest
+    uint32_t   wait_limit = kWaitLimit;    // bounded waits of the kernels (shortened only by fastsgd_debug_set_wait_limits)
+    uint32_t   try_limit = kTryLimit;
+    uint32_t   dec_spin_limit = kDecSpinLimit;
 };
 State g_state;
 std::atomic<uint64_t> g_launches{0};
@@ -68,7 +75,6 @@ int check_params(const fastsgd_params* p, PowTable* pw) {
         else t.P[k] = t.P[p->tau];
     }
     if (!std::isfinite(t.P[p->tau])) return FASTSGD_E_BAD_PARAM;
-    if (p->group_log2 != (uint32_t)kGroupLog2) return FASTSGD_E_NOT_IMPLEMENTED;
     return FASTSGD_OK;
 }
 
@@ -86,8 +92,7 @@ uint64_t bound_bytes(uint64_t n, const fastsgd_params* p) {
 uint64_t ws_dense_offset(uint64_t n, uint32_t group_log2) {
     // partials, descriptors, prefixes, tile maxima, the list of tiles to encode and its bitmap for every gradient one launch can take
     const uint64_t G = groups_of(n, group_log2);
-    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 24ull * G + 4ull * ((G + 31ull) >> 5))
-                       + 4ull * (G + 2ull);
+    const uint64_t b = kPartialsOffset + (uint64_t)kCmpMaxJobs * (8ull * chunks_of(n) + 24ull * G + 4ull * ((G + 31ull) >> 5));
     return (b + 255ull) & ~255ull;
 }
 
@@ -95,18 +100,17 @@ uint64_t ws_bytes_for(uint64_t n, uint32_t group_log2) {
     return ws_dense_offset(n, group_log2) + (uint64_t)kMaxCtas * kDenseScratchBytes;
 }
 
-WorkspaceView view(void* ws, uint64_t n) {
+WorkspaceView view(void* ws, uint64_t n, uint32_t group_log2 = kGroupLog2) {
     WorkspaceView v;
     unsigned char* base = static_cast<unsigned char*>(ws);
     v.ctl = reinterpret_cast<Control*>(base);
     v.thr = reinterpret_cast<float*>(base + kThrOffset);
     v.partials = reinterpret_cast<double*>(base + kPartialsOffset);
     v.desc = reinterpret_cast<unsigned long long*>(base + kPartialsOffset + (uint64_t)kCmpMaxJobs * 8ull * chunks_of(n));
-    v.prefix = v.desc + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2);
-    v.tmax = reinterpret_cast<float*>(v.prefix + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
-    v.nelist = reinterpret_cast<uint32_t*>(v.tmax + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2));
-    v.nebits = v.nelist + (uint64_t)kCmpMaxJobs * groups_of(n, kGroupLog2);
-    v.kv_start = v.nebits + (uint64_t)kCmpMaxJobs * ((groups_of(n, kGroupLog2) + 31ull) >> 5);
+    v.prefix = v.desc + (uint64_t)kCmpMaxJobs * groups_of(n, group_log2);
+    v.tmax = reinterpret_cast<float*>(v.prefix + (uint64_t)kCmpMaxJobs * groups_of(n, group_log2));
+    v.nelist = reinterpret_cast<uint32_t*>(v.tmax + (uint64_t)kCmpMaxJobs * groups_of(n, group_log2));
+    v.nebits = v.nelist + (uint64_t)kCmpMaxJobs * groups_of(n, group_log2);
     return v;
 }
 
@@ -123,7 +127,9 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_compress<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
-    if (cudaFuncSetAttribute(k_compress<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
+    if (cudaFuncSetAttribute(k_compress_kv<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(KvSmem)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_compress_kv<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(KvSmem)) != cudaSuccess)
         return FASTSGD_E_CUDA;
     int b1 = 0, b2 = 0, b3 = 0;
     {
@@ -133,8 +139,10 @@ int ensure_device_setup() {
         if (b3b < b3) b3 = b3b;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<false, true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (b3b < b3) b3 = b3b;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress<false, false, true>, kCmpThreads, sizeof(CmpSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
-        if (b3b < b3) b3 = b3b;
+        int b3c = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3b, k_compress_kv<false>, kKvThreads, sizeof(KvSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b3c, k_compress_kv<true>, kKvThreads, sizeof(KvSmem)) != cudaSuccess) return FASTSGD_E_CUDA;
+        g_state.kv_blocks_per_sm = b3b < b3c ? b3b : b3c;
     }
     g_state.cmp_blocks_per_sm = b3;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, k_abs_sum, kSumThreads, 0) != cudaSuccess) return FASTSGD_E_CUDA;
@@ -206,6 +214,31 @@ int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]) {
 
 uint64_t fastsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+int fastsgd_debug_set_wait_limits(uint32_t block_polls, uint32_t copy_tries, uint32_t queue_polls) {
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    g_state.wait_limit = block_polls ? block_polls : kWaitLimit;
+    g_state.try_limit = copy_tries ? copy_tries : kTryLimit;
+    g_state.dec_spin_limit = queue_polls == 0xFFFFFFFFu ? 0u : (queue_polls ? queue_polls : kDecSpinLimit);
+    return FASTSGD_OK;
+}
+
+int fastsgd_debug_layout(uint64_t* offsets, uint32_t count) {
+    if (!offsets) return FASTSGD_E_NULL;
+    const uint64_t v[FASTSGD_DEBUG_LAYOUT_FIELDS] = {
+        offsetof(Control, bar_count), offsetof(Control, ne_count), offsetof(Control, error),
+        kTraceOffset, kJobTraceOffset, kJobTraceBytes, kQueueOffset, offsetof(Control, dq)};
+    for (uint32_t i = 0; i < count && i < (uint32_t)FASTSGD_DEBUG_LAYOUT_FIELDS; ++i) offsets[i] = v[i];
+    return FASTSGD_OK;
+}
+
+int fastsgd_debug_trace_compiled(void) {
+#ifdef FASTSGD_TRACE
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 const char* fastsgd_strerror(int code) {
     switch (code) {
         case FASTSGD_OK: return "ok";
@@ -237,13 +270,13 @@ const char* fastsgd_strerror(int code) {
 
 uint64_t fastsgd_compress_bound(uint64_t n, const fastsgd_params* params) {
     int rc = check_params(params, nullptr);
-    if ((rc != FASTSGD_OK && rc != FASTSGD_E_NOT_IMPLEMENTED) || n == 0) return 0;
+    if (rc != FASTSGD_OK || n == 0) return 0;
     return bound_bytes(n, params);
 }
 
 uint64_t fastsgd_workspace_bytes(uint64_t n, const fastsgd_params* params) {
     int rc = check_params(params, nullptr);
-    if ((rc != FASTSGD_OK && rc != FASTSGD_E_NOT_IMPLEMENTED) || n == 0) return 0;
+    if (rc != FASTSGD_OK || n == 0) return 0;
     return ws_bytes_for(n, params->group_log2);
 }
 
@@ -260,6 +293,7 @@ int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
         return FASTSGD_E_CUDA;
     g_state.ws = dev_ptr;
     g_state.ws_bytes = bytes;
+    g_state.timed_out = false;
     return FASTSGD_OK;
 }
 
@@ -278,18 +312,56 @@ int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream
 }
 
 namespace {
-// The encoder's launches.  kv_keys == nullptr: num_grads dense gradients, up to 8 per launch.  Else one gradient
-// given as kv_count ascending keys with their values (grads is not used).
+// The list encoder (kv.cuh).  dense = false: `count` key-value pairs.  dense = true: the gradient `values` of n
+// entries itself, read as the list (i, v_i), with its sum already in the workspace.  Caller holds g_state.mu.
+int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
+                        const fastsgd_params* params, const PowTable& pw, void* out, uint64_t out_bytes, cudaStream_t st) {
+    if (g_state.kv_blocks_per_sm < 1) return FASTSGD_E_CUDA;
+    const uint64_t G = groups_of(n, params->group_log2);
+    WorkspaceView w = view(g_state.ws, n, params->group_log2);
+    KvArgs ka;
+    std::memset(&ka, 0, sizeof(ka));
+    ka.keys = keys; ka.vals = values; ka.count = dense ? n : count; ka.n = n;
+    ka.out = static_cast<uint8_t*>(out); ka.out_bytes = out_bytes; ka.ctl = w.ctl;
+    ka.partials = reinterpret_cast<double*>(static_cast<unsigned char*>(g_state.ws) + kKvPartialsOffset);
+    ka.meta = w.desc;
+    ka.blk_agg = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(g_state.ws) + kKvAggOffset);
+    ka.base = params->base; ka.G = (uint32_t)G; ka.chunks = (uint32_t)chunks_of(n);
+    ka.tau = params->tau; ka.l = params->flag_bits; ka.group_log2 = params->group_log2;
+    ka.wait_limit = g_state.wait_limit; ka.given_sum = dense ? 1u : 0u;
+    // a warp per 32 list entries (dense: per group) until the GPU is full; all blocks are resident: they meet at grid barriers
+    const uint64_t units = dense ? G : count;
+    const uint64_t per_warp = dense ? 1ull : 32ull;
+    uint64_t grid = (units + per_warp * kKvWarps - 1) / (per_warp * kKvWarps);
+    const uint64_t cap = (uint64_t)g_state.sm_count * (uint64_t)(g_state.kv_blocks_per_sm > 2 ? 2 : g_state.kv_blocks_per_sm);
+    if (grid > cap) grid = cap;
+    if (grid > kKvMaxGrid) grid = kKvMaxGrid;
+    if (grid < 1) grid = 1;
+    const uint64_t warps = grid * kKvWarps;
+    uint64_t slice = (units + warps - 1) / warps;
+    if (!dense) slice = (slice + 31ull) & ~31ull;
+    if (slice < per_warp) slice = per_warp;
+    ka.slice = (uint32_t)slice;
+    PowTable pwc = pw;
+    void* kargs[] = {&ka, &pwc};
+    cudaError_t err;
+    {
+        LaunchTimer lt(1, st);
+        err = cudaLaunchCooperativeKernel(dense ? (const void*)k_compress_kv<true> : (const void*)k_compress_kv<false>,
+                                          dim3((unsigned)grid), dim3(kKvThreads), kargs, sizeof(KvSmem), st);
+    }
+    if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return FASTSGD_OK;
+}
+
+// The encoder's launches: num_grads dense gradients, up to 8 per launch.
 int compress_launches(const float* const* grads, uint64_t n, const fastsgd_params* params,
-                      void* const* outs, uint64_t out_bytes, uint32_t num_grads,
-                      const uint32_t* kv_keys, const float* kv_vals, uint64_t kv_count, void* stream) {
-    const bool kv = kv_keys != nullptr || kv_vals != nullptr || grads == nullptr;
-    if (!outs || !params || (!kv && !grads)) return FASTSGD_E_NULL;
-    if (kv && kv_count && (!kv_keys || !kv_vals)) return FASTSGD_E_NULL;
-    if (kv && (!aligned(kv_keys, 4) || !aligned(kv_vals, 4))) return FASTSGD_E_ALIGN;
+                      void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream) {
+    if (!outs || !params || !grads) return FASTSGD_E_NULL;
     for (uint32_t i = 0; i < num_grads; ++i) {
-        if ((!kv && !grads[i]) || !outs[i]) return FASTSGD_E_NULL;
-        if ((!kv && !aligned(grads[i], 16)) || !aligned(outs[i], 16)) return FASTSGD_E_ALIGN;
+        if (!grads[i] || !outs[i]) return FASTSGD_E_NULL;
+        if (!aligned(grads[i], 16) || !aligned(outs[i], 16)) return FASTSGD_E_ALIGN;
     }
     PowTable pw;
     int rc = check_params(params, &pw);
@@ -300,10 +372,23 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
     if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
     if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;   // descriptor fields are 31 bits
     std::lock_guard<std::mutex> lock(g_state.mu);
-    if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
+    if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (params->group_log2 != (uint32_t)kGroupLog2) {
+        // Any other group size: the sum kernel, then the list encoder over the dense gradient (the fused kernel's
+        // tile is the group of 2^14).  Two launches per gradient, the gradient read three times.
+        if (params->group_log2 < 8u) return FASTSGD_E_NOT_IMPLEMENTED;
+        for (uint32_t i = 0; i < num_grads; ++i) {
+            double* S = reinterpret_cast<double*>(static_cast<unsigned char*>(g_state.ws) + kJobSumOffset);
+            rc = launch_sum(grads[i], n, 0u, params->tau, pw, view(g_state.ws, n, params->group_log2), S, st);
+            if (rc) return rc;
+            rc = launch_list_encoder(true, nullptr, grads[i], n, n, params, pw, outs[i], out_bytes, st);
+            if (rc) return rc;
+        }
+        return FASTSGD_OK;
+    }
     WorkspaceView w = view(g_state.ws, n);
     if (g_state.cmp_blocks_per_sm < 1) return FASTSGD_E_CUDA;
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
@@ -315,20 +400,14 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
         std::memset(&cb, 0, sizeof(cb));
         cb.jobs = num_grads - first < (uint32_t)kCmpMaxJobs ? num_grads - first : (uint32_t)kCmpMaxJobs;
         for (uint32_t i = 0; i < cb.jobs; ++i) {
-            cb.grad[i] = kv ? nullptr : grads[first + i];
+            cb.grad[i] = grads[first + i];
             cb.out[i] = static_cast<uint8_t*>(outs[first + i]);
-        }
-        if (kv) {
-            if (kv_count > n) return FASTSGD_E_BAD_N;
-            cb.kv_keys = kv_keys; cb.kv_vals = kv_vals; cb.kv_start = w.kv_start;
-            k_kv_bounds<<<(unsigned)((G + 1ull + 255ull) / 256ull), 256, 0, st>>>(kv_keys, (uint32_t)kv_count, (uint32_t)G, w.kv_start);
-            g_launches.fetch_add(1, std::memory_order_relaxed);
-            if (cudaGetLastError() != cudaSuccess) return FASTSGD_E_CUDA;
         }
         cb.out_bytes = out_bytes; cb.n = n; cb.ctl = w.ctl; cb.partials = w.partials; cb.desc = w.desc; cb.prefix = w.prefix; cb.tmax = w.tmax; cb.nelist = w.nelist; cb.nebits = w.nebits;
         cb.sm_slots = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kSmSlotOffset);
         cb.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
         cb.base = params->base; cb.G = (uint32_t)G; cb.tau = params->tau; cb.l = params->flag_bits;
+        cb.wait_limit = g_state.wait_limit; cb.try_limit = g_state.try_limit;
         // Two or more gradients, two resident blocks per SM and enough tiles: the two blocks of an SM
         // form two teams that work on different gradients.  One gradient: the tiles below the grid
         // size are assigned statically, so every block gets an equal share.
@@ -346,9 +425,8 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
         cudaError_t err;
         {
             LaunchTimer lt(1, st);
-            const void* fn = kv ? (const void*)k_compress<false, false, true>
-                                : cb.jobs > 1u ? (const void*)k_compress<true>
-                                : (cb.G > kCmpBigTiles ? (const void*)k_compress<false, true> : (const void*)k_compress<false>);
+            const void* fn = cb.jobs > 1u ? (const void*)k_compress<true>
+                                          : (cb.G > kCmpBigTiles ? (const void*)k_compress<false, true> : (const void*)k_compress<false>);
             err = cudaLaunchCooperativeKernel(fn, dim3((unsigned)launch_grid), dim3(kCmpThreads), kargs, sizeof(CmpSmem), st);
         }
         if (err != cudaSuccess) { cudaGetLastError(); return FASTSGD_E_CUDA; }
@@ -361,17 +439,28 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
 int fastsgd_compress_batch(const float* const* grads, uint64_t n, const fastsgd_params* params,
                            void* const* outs, uint64_t out_bytes, uint32_t num_grads, void* stream) {
     if (!grads) return FASTSGD_E_NULL;
-    return compress_launches(grads, n, params, outs, out_bytes, num_grads, nullptr, nullptr, 0, stream);
+    return compress_launches(grads, n, params, outs, out_bytes, num_grads, stream);
 }
 
 int fastsgd_compress_kv(const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
                         const fastsgd_params* params, void* out, uint64_t out_bytes, void* stream) {
-    if (!out) return FASTSGD_E_NULL;
-    static const uint32_t no_keys[1] = {0};
-    static const float no_vals[1] = {0.f};
-    void* o1[1] = {out};
-    // (an empty list still goes through the key-value kernel: the pointers only mark the mode then)
-    return compress_launches(nullptr, n, params, o1, out_bytes, 1u, count ? keys : no_keys, count ? values : no_vals, count, stream);
+    if (!out || !params) return FASTSGD_E_NULL;
+    if (count && (!keys || !values)) return FASTSGD_E_NULL;
+    if (!aligned(keys, 4) || !aligned(values, 4) || !aligned(out, 16)) return FASTSGD_E_ALIGN;
+    PowTable pw;
+    int rc = check_params(params, &pw);
+    if (rc) return rc;
+    rc = check_n(n);
+    if (rc) return rc;
+    if (count > n) return FASTSGD_E_BAD_N;
+    const uint64_t G = groups_of(n, params->group_log2);
+    if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
+    if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
+    rc = ensure_device_setup();
+    if (rc) return rc;
+    return launch_list_encoder(false, keys, values, count, n, params, pw, out, out_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params,
@@ -395,13 +484,15 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
     if (rc) return rc;
     rc = check_n(n);
     if (rc) return rc;
+    // (the queue of groups that whole blocks decode has 2^17 slots)
+    if (params->group_log2 < 8u || groups_of(n, params->group_log2) > (kQueueBytes >> 2)) return FASTSGD_E_NOT_IMPLEMENTED;
     for (uint32_t i = 0; i < num_streams; ++i) {
         if (!streams_in[i]) return FASTSGD_E_NULL;
         if (!aligned(streams_in[i], 16)) return FASTSGD_E_ALIGN;
         if (bytes[i] < kHeaderBytes) return FASTSGD_E_TRUNCATED;
     }
     std::lock_guard<std::mutex> lock(g_state.mu);
-    if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
+    if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
     const uint64_t G = groups_of(n, params->group_log2);
@@ -432,6 +523,7 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
         da.q_list = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kQueueOffset);
         da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
         da.group_log2 = params->group_log2;
+        da.spin_limit = g_state.dec_spin_limit; da.try_limit = g_state.try_limit;
         if (adam) {
             da.theta = theta; da.m = m; da.v = v;
             da.lr = adam->lr; da.beta1 = adam->beta1; da.beta2 = adam->beta2; da.eps = adam->eps;
@@ -525,7 +617,12 @@ int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_byt
     if (cudaMemcpyAsync(h, stream_in, kHeaderBytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
     uint32_t s32; uint64_t v;
-    if (status) { std::memcpy(&s32, h + 8, 4); *status = (int)s32; }
+    std::memcpy(&s32, h + 8, 4);
+    if (status) *status = (int)s32;
+    if (s32 == (uint32_t)FASTSGD_ST_TIMEOUT) {        // the launch that wrote this stream left the workspace's counters mid-way
+        std::lock_guard<std::mutex> lock(g_state.mu);
+        g_state.timed_out = true;
+    }
     if (d) { std::memcpy(&v, h + 24, 8); *d = v; }
     if (total_bytes) { std::memcpy(&v, h + 32, 8); *total_bytes = v; }
     return FASTSGD_OK;
@@ -541,6 +638,7 @@ int fastsgd_decode_status(void* stream, int* status) {
     if (cudaMemcpyAsync(&v, p, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;
     *status = (v == ~0ull) ? FASTSGD_ST_OK : (int)(v & 0xFFull);
+    if (*status == FASTSGD_ST_TIMEOUT) g_state.timed_out = true;
     if (v != ~0ull) {
         if (cudaMemsetAsync(p, 0xFF, 8, st) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return FASTSGD_E_CUDA;

@@ -56,7 +56,11 @@ constexpr uint64_t kJobTraceOffset = kQueueOffset + kQueueBytes;  // u64 [320 bl
 constexpr uint64_t kJobTraceBytes  = 320ull * 8ull * 8ull * 8ull;
 constexpr uint64_t kSmSlotOffset   = kJobTraceOffset + kJobTraceBytes;  // u32 [256]: blocks of the running launch seen on each SM (zero between launches)
 constexpr uint64_t kSmSlotBytes    = 1024;
-constexpr uint64_t kPartialsOffset = kSmSlotOffset + kSmSlotBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]; then float tmax[G]; then u32 nelist[G]; then u32 nebits[ceil(G / 32)]; after the 8 gradients: u32 kv_start[G + 2] (key-value input)
+constexpr uint64_t kKvPartialsOffset = kSmSlotOffset + kSmSlotBytes;   // double [2^17]: chunk nodes of the key-value encoder's sum (zero between launches)
+constexpr uint64_t kKvPartialsBytes  = 8ull << 17;
+constexpr uint64_t kKvAggOffset    = kKvPartialsOffset + kKvPartialsBytes;   // u64 [512]: per-block totals of the key-value encoder
+constexpr uint64_t kKvAggBytes     = 8ull * 512ull;
+constexpr uint64_t kPartialsOffset = kKvAggOffset + kKvAggBytes;  // per gradient of a launch: double partial[chunks]; then u64 desc[G]; then u64 prefix[G]; then float tmax[G]; then u32 nelist[G]; then u32 nebits[ceil(G / 32)]
 
 struct WorkspaceView {
     Control*            ctl;
@@ -67,7 +71,6 @@ struct WorkspaceView {
     float*              tmax;
     uint32_t*           nelist;
     uint32_t*           nebits;
-    uint32_t*           kv_start;
 };
 
 __host__ __device__ inline uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }

@@ -75,10 +75,10 @@ struct CmpSmem {
     uint32_t max_delta;
     uint32_t abort_flag;
     uint32_t poison_seen;
-    uint32_t pad;
+    uint32_t wait_limit;                     // polls before a wait on another block gives up (from the launch arguments)
     uint32_t next_tile[2];                   // by tile parity: the tile this block works on next
     uint32_t ne_count;                       // tiles the gradient's encode pass hands out by ticket
-    uint32_t pad6;
+    uint32_t try_limit;                      // tries before a wait on a bulk copy gives up (from the launch arguments)
     uint32_t held[2];                        // tiles this block has taken and not yet published (for the give-up path)
     uint32_t sc_pos, sc_count, sc_words;     // running exclusive scan of the descriptors: [0, pos) included
     uint32_t job_skip[2];                    // by gradient parity: 0 encode, 1 sum == 0, 2 sum not finite
@@ -144,11 +144,8 @@ struct CmpBatch {
     uint32_t            l;
     uint32_t            teams;           // 1, or 2: the two blocks of every SM work on different gradients
     uint32_t            pad;
-    // key-value input (kernel variant KV, one gradient): the gradient is given as kv_count ascending keys with
-    // their values instead of grad[0]; kv_start[t] = index of the first entry with key >= t * 2^14, t = 0..G
-    const uint32_t*     kv_keys;
-    const float*        kv_vals;
-    const uint32_t*     kv_start;
+    uint32_t            wait_limit;      // polls before a wait on another block gives up (kWaitLimit unless a test shortens it)
+    uint32_t            try_limit;       // tries before a wait on a bulk copy gives up (kTryLimit likewise)
 };
 
 __device__ __forceinline__ CmpArgs job_view(const CmpBatch& b, uint32_t w) {
@@ -181,9 +178,9 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
 // wait costs a handful of instructions; false when every try ran out.
 constexpr uint32_t kTryHintNs = 10000u;
 constexpr uint32_t kTryLimit  = 1u << 18;
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, uint32_t tries = kTryLimit) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t t = 0; t < kTryLimit; ++t) {
+    for (uint32_t t = 0; t < tries; ++t) {
         uint32_t ok;
         asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
                      : "=r"(ok) : "r"(addr), "r"(parity), "r"(kTryHintNs) : "memory");
@@ -219,11 +216,17 @@ __device__ __forceinline__ unsigned int atom_add_acq_rel_u32(unsigned int* p, un
     asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
     return old;
 }
+// Phase stamps (%globaltimer, thread 0 of every block) are compiled in only with -DFASTSGD_TRACE.
+#ifdef FASTSGD_TRACE
 __device__ __forceinline__ unsigned long long read_globaltimer() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+#define FSG_STAMP(slot) do { if (tid == 0) btrace[(slot)] = read_globaltimer(); } while (0)
+#else
+#define FSG_STAMP(slot) do { } while (0)
+#endif
 
 // Starts the copy of tile `tile` into `stage` (thread 0), and, for the one tile that reaches past
 // n, fills the rest of the buffer (all threads).  Called by the whole block.
@@ -270,35 +273,6 @@ __device__ __forceinline__ void issue_half(CmpSmem& s, const CmpArgs& a, uint32_
         __syncthreads();
         // these were generic-proxy writes to a buffer that a later bulk copy (async proxy) overwrites
         if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-}
-
-// Key-value input: the tile is formed in the stage from the entries that fall into it (zeros
-// elsewhere), so that everything downstream sees what a bulk copy of the dense gradient would have
-// brought.  Called by the whole block; the stage must be free; complete when it returns.
-__device__ __forceinline__ void kv_fill_tile(CmpSmem& s, const CmpBatch& b, uint32_t tile, int tid) {
-    float4* st4 = reinterpret_cast<float4*>(&s.stage[0][0]);
-    for (uint32_t i = tid; i < kTile / 4u; i += kCmpThreads) st4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const uint32_t lo = __ldg(b.kv_start + tile), hi = __ldg(b.kv_start + tile + 1u);
-    __syncthreads();
-    const uint32_t base = tile << kGroupLog2;
-    for (uint32_t j = lo + (uint32_t)tid; j < hi; j += kCmpThreads) {
-        const uint32_t k = __ldg(b.kv_keys + j) - base;
-        if (k < kTile) s.stage[0][k] = __ldg(b.kv_vals + j);      // (keys that do not ascend cannot write outside the stage)
-    }
-    __syncthreads();
-}
-
-// The encode pass's "start bringing tile `tile` into the stage": a bulk copy in flight, or (key-value input) the
-// tile formed on the spot.
-template <bool KV>
-__device__ __forceinline__ void load_tile(CmpSmem& s, const CmpBatch& b, const CmpArgs& a, int stage, uint32_t tile,
-                                          uint32_t& pending, int tid) {
-    if constexpr (KV) {
-        kv_fill_tile(s, b, tile, tid);
-    } else {
-        issue_tile(s, a, stage, tile, tid);
-        pending |= 1u << stage;
     }
 }
 
@@ -527,11 +501,12 @@ __device__ __forceinline__ void place_pending(CmpSmem& s, const CmpArgs& a, uint
         }
         if (mine && g == a.G - 1 && lane == 0) {
             int status = kStOk;
-            if (skip == 2u) status = kStNonfinite;
+            if (ld_acquire_u32(&a.ctl->error) != 0u) status = kStTimeout;      // some block of the launch gave up: its tiles are missing
+            else if (skip == 2u) status = kStNonfinite;
             else if (end_bytes > a.out_bytes) status = kStCapacity;
             const uint64_t d_total = status == kStOk ? (pre >> 32) + (cm & 0xFFFFFFu) : 0ull;
             const uint64_t total = status == kStOk ? end_bytes : (uint64_t)kHeaderBytes;
-            const double Sh = status == kStNonfinite ? 0.0 : S;
+            const double Sh = (status == kStNonfinite || status == kStTimeout) ? 0.0 : S;
             outw[0] = kMagic;
             outw[1] = kVersion;
             outw[2] = (uint32_t)status;
@@ -568,7 +543,7 @@ __device__ __forceinline__ void fetch_prefixes(CmpSmem& s, const CmpArgs& a, int
         unsigned long long v = ld_relaxed_u64(p);
         uint32_t spin = 0;
         while ((v >> 62) == kDescInvalid) {
-            if (++spin > kWaitLimit) { s.poison_seen = 2u; break; }
+            if (++spin > s.wait_limit) { s.poison_seen = 2u; break; }
             if (spin > 32u) __nanosleep(32);
             v = ld_relaxed_u64(p);
         }
@@ -609,7 +584,7 @@ __device__ __forceinline__ bool drain_wait(CmpSmem& s, const CmpArgs& a, const C
             const uint32_t idx = sc.pos + (uint32_t)j * kCmpThreads + tid;
             uint32_t spin = 0;
             while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
-                if (++spin > kWaitLimit) { s.poison_seen = 2u; own[j] = 0ull; break; }
+                if (++spin > s.wait_limit) { s.poison_seen = 2u; own[j] = 0ull; break; }
                 __nanosleep(64);
                 own[j] = ld_relaxed_u64(a.desc + idx);
             }
@@ -718,7 +693,7 @@ __device__ __forceinline__ void publish_prefixes(CmpSmem& s, const CmpArgs& a, i
                 const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
                 uint32_t spin = 0;
                 while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
-                    if (++spin > kWaitLimit) break;
+                    if (++spin > s.wait_limit) break;
                     if (spin > 32u) __nanosleep(32);
                     own[j] = ld_relaxed_u64(a.desc + idx);
                 }
@@ -788,7 +763,7 @@ __device__ __forceinline__ unsigned long long scan_segment(CmpSmem& s, const Cmp
                 const uint32_t idx = pos + (uint32_t)j * kCmpThreads + tid;
                 uint32_t spin = 0;
                 while ((own[j] >> 62) == kDescInvalid) {         // not published yet: bounded poll
-                    if (++spin > kWaitLimit) break;
+                    if (++spin > s.wait_limit) break;
                     if (spin > 32u) __nanosleep(32);
                     own[j] = ld_relaxed_u64(a.desc + idx);
                 }
@@ -847,7 +822,7 @@ __device__ __forceinline__ void publish_part(CmpSmem& s, const CmpArgs& a, unsig
         unsigned long long v = ld_relaxed_u64(segtot + tid);
         uint32_t spin = 0;
         while ((v >> 62) == kDescInvalid) {
-            if (++spin > kWaitLimit) break;
+            if (++spin > s.wait_limit) break;
             if (spin > 32u) __nanosleep(32);
             v = ld_relaxed_u64(segtot + tid);
         }
@@ -861,6 +836,22 @@ __device__ __forceinline__ void publish_part(CmpSmem& s, const CmpArgs& a, unsig
     if (s.pad5) bad = true;
     __syncthreads();
     scan_segment(s, a, beg, end, base, true, bad, tid, lane, warp);
+}
+
+// Every stream of the launch reports the timeout: a header with that status and nothing else (identical words from
+// every block that writes them).  One thread.
+__device__ __forceinline__ void write_timeout_headers(const CmpBatch& b) {
+    for (uint32_t w = 0; w < b.jobs; ++w) {
+        uint32_t* outw = reinterpret_cast<uint32_t*>(b.out[w]);
+        outw[0] = kMagic; outw[1] = kVersion; outw[2] = (uint32_t)kStTimeout; outw[3] = b.tau;
+        outw[4] = (uint32_t)b.n; outw[5] = (uint32_t)(b.n >> 32);
+        outw[6] = 0u; outw[7] = 0u; outw[8] = kHeaderBytes; outw[9] = 0u;
+        outw[10] = 0u; outw[11] = 0u;
+        const unsigned long long bb = (unsigned long long)__double_as_longlong(b.base);
+        outw[12] = (uint32_t)bb; outw[13] = (uint32_t)(bb >> 32);
+        outw[14] = b.l | ((uint32_t)kGroupLog2 << 8);
+        outw[15] = b.G;
+    }
 }
 
 // Phase 1 for one gradient: fp64 partial sum of every 2^14-entry tile.  Tiles grid..G-1 are handed
@@ -917,7 +908,7 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         uint32_t nxt = kNoTicket;
 #pragma unroll
         for (int part = 0; part < 2; ++part) {
-            if (!mbar_wait(&s.mbar[part], (parity >> part) & 1u)) s.abort_flag = 1u;
+            if (!mbar_wait(&s.mbar[part], (parity >> part) & 1u, s.try_limit)) s.abort_flag = 1u;
             parity ^= 1u << part;
             pending &= ~(1u << part);
             double x[4];
@@ -962,57 +953,6 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
         t1 = warp_tree(t1, kCmpWarps);
         const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? max(s.s_wmax[qp][0][lane], s.s_wmax[qp][1][lane]) : 0u);
         if (lane == 0) { a.partials[prev_tile] = __dadd_rn(t0, t1); a.tmax[prev_tile] = __uint_as_float(tm); }
-    }
-}
-
-// The sum pass for key-value input (one gradient): tiles above the grid by ticket from the last one down, the
-// block's own tile c last (it stays in the stage for the encode pass).  A tile without entries has partial 0 and
-// is not formed at all; the others are formed in the stage and reduced on the same tree as a copied tile (zeros
-// add exactly nothing), so the sum has the bits of the dense gradient's sum.
-__device__ __forceinline__ void sum_pass_kv(CmpSmem& s, const CmpBatch& b, const CmpArgs& a, uint32_t c, uint32_t grid,
-                                            int tid, int lane, int warp) {
-    for (;;) {
-        if (tid == 0) {
-            // thread 0 settles the tiles without entries by itself and comes back with the next one that has some
-            uint32_t tile;
-            for (;;) {
-                const unsigned int tk = atomicAdd(a.ctl->tickets1, 1u);
-                tile = grid + tk < a.G ? a.G - 1u - tk : c;
-                a.desc[tile] = 0ull; a.prefix[tile] = 0ull;
-                if (tile == c || __ldg(b.kv_start + tile) != __ldg(b.kv_start + tile + 1u)) break;
-                a.partials[tile] = 0.0; a.tmax[tile] = 0.0f;
-            }
-            s.p1_next[0] = tile;
-        }
-        __syncthreads();
-        const uint32_t tile = s.p1_next[0];
-        const bool last = tile == c;
-        kv_fill_tile(s, b, tile, tid);
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            double x[4];
-            float mx = 0.0f;
-            const float4* row = reinterpret_cast<const float4*>(&s.stage[0][part * (int)(kTile / 2) + warp * 512]) + lane;
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const float4 v4 = row[r * 32];
-                x[r] = abs_sum4(v4);
-                mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v4.x), fabsf(v4.y)), fmaxf(fabsf(v4.z), fabsf(v4.w))));
-            }
-            const double u = warp_halfslab_tree(x, lane);
-            const uint32_t wmx = __reduce_max_sync(kFullMask, __float_as_uint(mx));
-            if (lane == 0) { s.s_warp[0][part][warp] = u; s.s_wmax[0][part][warp] = wmx; }
-        }
-        __syncthreads();
-        if (warp == 0) {
-            double t0 = lane < kCmpWarps ? s.s_warp[0][0][lane] : 0.0, t1 = lane < kCmpWarps ? s.s_warp[0][1][lane] : 0.0;
-            t0 = warp_tree(t0, kCmpWarps);
-            t1 = warp_tree(t1, kCmpWarps);
-            const uint32_t tm = __reduce_max_sync(kFullMask, lane < kCmpWarps ? max(s.s_wmax[0][0][lane], s.s_wmax[0][1][lane]) : 0u);
-            if (lane == 0) { a.partials[tile] = __dadd_rn(t0, t1); a.tmax[tile] = __uint_as_float(tm); }
-        }
-        __syncthreads();                                 // (s_warp and p1_next are rewritten next)
-        if (last) break;
     }
 }
 
@@ -1125,7 +1065,7 @@ __device__ __forceinline__ void barrier_wait(CmpSmem& s, Control* ctl, uint32_t 
     if (tid == 0 && !s.abort_flag) {
         uint32_t spin = 0;
         while (ld_acquire_u32(&ctl->bar_flag[job]) != gen_next) {
-            if (++spin > kWaitLimit) { s.abort_flag = 1u; break; }
+            if (++spin > s.wait_limit) { s.abort_flag = 1u; break; }
             if (spin > 64u) __nanosleep(32);
         }
     }
@@ -1170,16 +1110,16 @@ __device__ __forceinline__ void make_table(CmpSmem& s, const CmpArgs& a, const P
 // BIG (one gradient only): the variant for gradients with very many tiles, where the steps that one
 // block does for everybody (reducing the partials, listing the tiles, scanning the descriptors) take
 // forms that cost less per tile and more to start with.
-// KV (one gradient only): the gradient comes as ascending keys with their values; tiles are formed in the stage
-// from the entries (kv_fill_tile) instead of being copied, everything else is the same code.
-template <bool SEVERAL, bool BIG = false, bool KV = false>
+template <bool SEVERAL, bool BIG = false>
 __global__ void __launch_bounds__(kCmpThreads, 2)
 k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char cmp_smem_raw[];
     CmpSmem& s = *reinterpret_cast<CmpSmem*>(cmp_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t c = blockIdx.x;
+#ifdef FASTSGD_TRACE
     unsigned long long* btrace = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(b.ctl) + kJobTraceOffset) + 64u * c;
+#endif
 
     constexpr bool full = SEVERAL;            // several gradients: every tile of every pass is handed out by ticket
     unsigned int gen_next = 0u;
@@ -1188,6 +1128,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         for (int st = 0; st < 2; ++st) mbar_init(&s.mbar[st], 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s.abort_flag = 0u;
+        s.wait_limit = b.wait_limit; s.try_limit = b.try_limit;
         s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
         uint32_t team = 0u;
         if (b.teams == 2u) {                  // (the host launches exactly two blocks per SM then)
@@ -1223,7 +1164,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     CmpArgs a = job_view(b, 0u);
 
     if (step == 2u && team == 1u) {
-        if (tid == 0) btrace[8u * 7u + 0] = read_globaltimer();
+        FSG_STAMP(8u * 7u + 0);
         const SumCursor cur = sum_begin(s, a, 0u, full, c, grid, 2u, pending, tid);
         sum_rest(s, a, 0u, full, c, grid, 2u, cur, parity, pending, tid, lane, warp);
         barrier_arrive<BIG>(s, a, pw, 0u, full, grid, gridDim.x, gen_next, tid, lane, warp);
@@ -1231,14 +1172,12 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     }
     if (nown) {
         a = job_view(b, team);
-        if (tid == 0) btrace[8u * team + 0] = read_globaltimer();
-        if constexpr (KV) {
-            sum_pass_kv(s, b, a, c, grid, tid, lane, warp);
-        } else {
+        FSG_STAMP(8u * team + 0);
+        {
             const SumCursor cur = sum_begin(s, a, team, full, c, grid, 0xFFFFFFFFu, pending, tid);
             sum_rest(s, a, team, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
         }
-        if (tid == 0) btrace[8u * team + 1] = read_globaltimer();
+        FSG_STAMP(8u * team + 1);
         barrier_arrive<BIG>(s, a, pw, team, full, grid, (step == 2u && team == 0u) ? gridDim.x : grid, gen_next, tid, lane, warp);
     }
 
@@ -1252,20 +1191,20 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         // next gradient's sum pass; this gradient's table while the first copy is in flight
         const uint32_t nj = job + step;
         const CmpArgs an = job_view(b, nj);
-        if (tid == 0) btrace[8u * nj + 0] = read_globaltimer();
+        FSG_STAMP(8u * nj + 0);
         const SumCursor cur = sum_begin(s, an, nj, full, c, grid, 0xFFFFFFFFu, pending, tid);
         barrier_wait(s, b.ctl, job, gen_next, tid);
-        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
+        FSG_STAMP(8u * job + 3);
         if (!s.abort_flag) make_table(s, a, pw, job, jp, tid, lane, warp);
-        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
+        FSG_STAMP(8u * job + 4);
         sum_rest(s, an, nj, full, c, grid, 0xFFFFFFFFu, cur, parity, pending, tid, lane, warp);
-        if (tid == 0) btrace[8u * nj + 1] = read_globaltimer();
+        FSG_STAMP(8u * nj + 1);
         barrier_arrive<BIG>(s, an, pw, nj, full, grid, grid, gen_next, tid, lane, warp);
     } else {
         barrier_wait(s, b.ctl, job, gen_next, tid);
-        if (tid == 0) btrace[8u * job + 3] = read_globaltimer();
+        FSG_STAMP(8u * job + 3);
         if (!s.abort_flag) make_table(s, a, pw, job, jp, tid, lane, warp);
-        if (tid == 0) btrace[8u * job + 4] = read_globaltimer();
+        FSG_STAMP(8u * job + 4);
     }
     __syncthreads();
     aborted = s.abort_flag != 0u;
@@ -1289,10 +1228,10 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             __syncthreads();
             g = s.next_tile[1];
             have = g < a.G;
-            if (have) load_tile<KV>(s, b, a, 0, g, pending, tid);
+            if (have) { issue_tile(s, a, 0, g, tid); pending |= 1u; }
         }
         const CmpArgs ap = job_view(b, prev_job);
-        if (tid == 0) btrace[8u * job + 2] = read_globaltimer();
+        FSG_STAMP(8u * job + 2);
 
         // =============================== encode pass ===============================
         // Every warp owns one slab of 1024 consecutive entries of the tile in the stage: it filters
@@ -1314,8 +1253,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             // iteration's first barrier)
             uint32_t tile_ahead = kNoMore;
             if (tid == 0) tile_ahead = ticket_ahead == kNoTicket ? kNoTicket : (ticket_ahead < listed ? __ldcg(a.nelist + ticket_ahead) : kNoMore);
-            if (!KV && (i > 0u || preloaded)) {
-                if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u)) s.abort_flag = 1u;
+            if (i > 0u || preloaded) {
+                if (!mbar_wait(&s.mbar[st], (parity >> st) & 1u, s.try_limit)) s.abort_flag = 1u;
                 parity ^= 1u << st;
                 pending &= ~(1u << st);
             }
@@ -1428,7 +1367,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             const uint32_t g_next = s.next_tile[par];
             const bool more = g_next < a.G;                  // (false for kNoTicket too)
             if (more) {
-                if (!overflow) load_tile<KV>(s, b, a, st, g_next, pending, tid);      // (a tile too dense for the lists packs its blob in the stage first)
+                if (!overflow) { issue_tile(s, a, st, g_next, tid); pending |= 1u << st; }      // (a tile too dense for the lists packs its blob in the stage first)
                 if (tid == 0) {
                     const bool stop_reserving = overflow || dense_pending ||
                         npend + 3 >= kPendMax || arena_used + worst_now + 2u * kArenaReserve > kArenaWords;
@@ -1541,7 +1480,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 __syncthreads();                     // the stage is free
                 if (more) {                          // (generic-proxy writes before an async-proxy one)
                     if (tid == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    load_tile<KV>(s, b, a, st, g_next, pending, tid);
+                    issue_tile(s, a, st, g_next, tid); pending |= 1u << st;
                 }
             }
             if (tid == 0) {
@@ -1565,7 +1504,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 g = s.next_tile[par];
                 have = g < a.G;
                 if (have) {
-                    load_tile<KV>(s, b, a, st, g, pending, tid);
+                    issue_tile(s, a, st, g, tid); pending |= 1u << st;
                     if (tid == 0) ticket_ahead = atomicAdd(a.ticket, 1u);
                 }
                 if (npend > 0) drain_place(s, a, ap, jp, nprev, npend, tid, lane, warp);
@@ -1576,7 +1515,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
                 have = more;
             }
         }
-        if (tid == 0) btrace[8u * job + 5] = read_globaltimer();
+        FSG_STAMP(8u * job + 5);
         // this block's tiles of the gradient are published: count it; the last block through computes
         // the prefixes for everybody
         if (tid == 0) {
@@ -1623,7 +1562,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         __syncthreads();                           // pending list written by thread 0
         if (!drain_final(s, job_view(b, prev_job), (niter - 1u) & 1u, nprev, tid, lane, warp)) aborted = true;
     }
-    if (tid == 0) btrace[6] = read_globaltimer();   // (slot 6 of the first gradient: end of the launch's last drain)
+    FSG_STAMP(6);   // (slot 6 of the first gradient: end of the launch's last drain)
 
     if (aborted) {
         // give up: record it, unblock the others, wait for this block's copies, mark every stream of
@@ -1635,19 +1574,8 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
             if (s.held[0] < a.G) st_relaxed_u64(a.desc + s.held[0], desc_pack(kDescPoison, 0, 0));
             if (s.held[1] < a.G) st_relaxed_u64(a.desc + s.held[1], desc_pack(kDescPoison, 0, 0));
             for (int st = 0; st < 2; ++st)
-                if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u);
-            // every stream of the launch reports the timeout (identical words from every block that gives up)
-            for (uint32_t w = 0; w < b.jobs; ++w) {
-                uint32_t* outw = reinterpret_cast<uint32_t*>(b.out[w]);
-                outw[0] = kMagic; outw[1] = kVersion; outw[2] = (uint32_t)kStTimeout; outw[3] = a.tau;
-                outw[4] = (uint32_t)a.n; outw[5] = (uint32_t)(a.n >> 32);
-                outw[6] = 0u; outw[7] = 0u; outw[8] = kHeaderBytes; outw[9] = 0u;
-                outw[10] = 0u; outw[11] = 0u;
-                const unsigned long long bb = (unsigned long long)__double_as_longlong(a.base);
-                outw[12] = (uint32_t)bb; outw[13] = (uint32_t)(bb >> 32);
-                outw[14] = a.l | ((uint32_t)kGroupLog2 << 8);
-                outw[15] = a.G;
-            }
+                if (pending & (1u << st)) mbar_wait(&s.mbar[st], (parity >> st) & 1u, s.try_limit);
+            write_timeout_headers(b);
         }
         __syncthreads();
     }
@@ -1656,26 +1584,15 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
     if (tid == 0) {
         const unsigned int old = atom_add_acq_rel_u32(&b.ctl->exit_count, 1u);
         if (old == gridDim.x - 1u) {
+            // a block that did not give up may have written an OK header after the others marked the streams: the
+            // last block out (it sees every other block's writes) has the final word
+            if (ld_acquire_u32(&b.ctl->error) != 0u) write_timeout_headers(b);
             b.ctl->exit_count = 0u;
             if (b.teams == 2u) for (int i = 0; i < 256; ++i) b.sm_slots[i] = 0u;
             if constexpr (BIG) for (int i = 0; i < 2 * (int)kScanParts; ++i) b.sm_slots[i] = 0u;
             st_release_u32(&b.ctl->bar_gen, gen_next);
         }
     }
-}
-
-// Key-value input, first launch: kv_start[t] = number of entries with key < t * 2^14 (a binary search per
-// tile boundary), t = 0..G.
-__global__ void __launch_bounds__(256) k_kv_bounds(const uint32_t* __restrict__ keys, uint32_t count, uint32_t G, uint32_t* __restrict__ kv_start) {
-    const uint32_t t = blockIdx.x * 256u + threadIdx.x;
-    if (t > G) return;
-    const unsigned long long bound = (unsigned long long)t << kGroupLog2;
-    uint32_t lo = 0, hi = count;                      // first index whose key is >= bound
-    while (lo < hi) {
-        const uint32_t mid = lo + ((hi - lo) >> 1);
-        if ((unsigned long long)__ldg(keys + mid) < bound) lo = mid + 1u; else hi = mid;
-    }
-    kv_start[t] = lo;
 }
 
 }  // namespace fsg

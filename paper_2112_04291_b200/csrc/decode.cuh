@@ -42,13 +42,15 @@ struct DecArgs {
     unsigned long long* status;     // sticky minimum of (group << 32 | key index << 8 | status)
     unsigned int*       q_ctl;      // {pushed, taken, done, exited, reserved}: queue of groups for whole blocks, shared by the grid
     unsigned int*       q_list;     // its G slots
-    unsigned long long* trace;      // per-block stamps (profiling aid)
+    unsigned long long* trace;      // per-block stamps (only written by builds with -DFASTSGD_TRACE)
     double              base;
     uint32_t            W;          // streams in this launch
     uint32_t            G;
     uint32_t            tau;
     uint32_t            l;
     uint32_t            group_log2;
+    uint32_t            spin_limit; // polls before a wait on the queue of large groups gives up (kDecSpinLimit unless a test shortens it)
+    uint32_t            try_limit;  // tries before a wait on a bulk copy gives up
     // model update on the decoded coordinates (second pass; `dense` then holds the aggregated gradient)
     float*              theta;
     float*              m;
@@ -93,11 +95,16 @@ __device__ __forceinline__ void apply_run(const DecArgs& a, const uint32_t (&kk)
     }
 }
 
+#ifdef FASTSGD_TRACE
 __device__ __forceinline__ unsigned long long read_globaltimer_dec() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+#define FSG_DEC_STAMP(var) do { if (tid == 0) var = read_globaltimer_dec(); } while (0)
+#else
+#define FSG_DEC_STAMP(var) do { } while (0)
+#endif
 
 __device__ __forceinline__ void dec_fail(const DecArgs& a, uint32_t g, uint32_t j, int st) {
     atomicMin(a.status, ((unsigned long long)g << 32) | ((unsigned long long)(j & 0xFFFFFFu) << 8) | (unsigned)st);
@@ -605,9 +612,11 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     DecShared& s = *reinterpret_cast<DecShared*>(dec_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t W = a.W;
-    // per-block %globaltimer stamps (profiling aid): start, tables ready, own groups done, end; groups taken from the queue
+#ifdef FASTSGD_TRACE
+    // per-block %globaltimer stamps: start, tables ready, own groups done, end; groups taken from the queue
     unsigned long long T0 = 0, T1 = 0, T2 = 0; unsigned int taken = 0;
-    if (tid == 0) T0 = read_globaltimer_dec();
+#endif
+    FSG_DEC_STAMP(T0);
 
     if (tid == 0) {
         mbar_init(&s.tile_bar, 1u);
@@ -636,7 +645,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     }
     __syncthreads();
 
-    if (tid == 0) T1 = read_globaltimer_dec();
+    FSG_DEC_STAMP(T1);
     // ---- this block owns groups blockIdx.x, blockIdx.x + gridDim.x, ...; warp w takes every 8th of them
     // (a warp applies the streams of a group one after the other: with many streams the whole block is the better choice sooner)
     const uint32_t warp_max = W <= 2u ? kDecWarpMax : kDecWarpSide;
@@ -784,7 +793,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     }
     __syncthreads();
 
-    if (tid == 0) T2 = read_globaltimer_dec();
+    FSG_DEC_STAMP(T2);
     // ---- groups with many keys sit in a queue shared by all blocks, so that a block that found
     //      several of them does not hold the others up.  Slots are filled as the groups are found;
     //      a taker waits (bounded) for its slot, or leaves once every block is past its own groups
@@ -809,7 +818,11 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                     }
                     if (*reinterpret_cast<volatile unsigned int*>(q_done) >= gridDim.x &&
                         i >= *reinterpret_cast<volatile unsigned int*>(q_reserved)) break;      // nothing will fill it
-                    if (i >= a.G || ++spin > kDecSpinLimit) break;
+                    if (i >= a.G) break;
+                    if (++spin > a.spin_limit) {         // the slot was reserved and never filled in time: the group it stands for is lost
+                        dec_fail(a, 0u, 0u, kStTimeout);
+                        break;
+                    }
                     __nanosleep(100);
                 }
                 s.big[0] = got;
@@ -818,7 +831,9 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             g = s.big[0];
             if (g == 0xFFFFFFFFu) break;
         }
+#ifdef FASTSGD_TRACE
         ++taken;
+#endif
         const uint64_t lo64 = (uint64_t)g << a.group_log2;
         const uint64_t hi64 = lo64 + (1ull << a.group_log2);
         const uint32_t lo = (uint32_t)lo64, span = (uint32_t)((hi64 < a.n ? hi64 : a.n) - lo64);
@@ -857,7 +872,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         }
         __syncthreads();
         if (use_tile) {
-            if (tid == 0) s.big[1] = mbar_wait(&s.tile_bar, tile_parity) ? 1u : 0u;     // bounded wait, one thread
+            if (tid == 0) s.big[1] = mbar_wait(&s.tile_bar, tile_parity, a.try_limit) ? 1u : 0u;     // bounded wait, one thread
             __syncthreads();
             tile_parity ^= 1u;
             if (s.big[1] == 0u) {                                 // ran out: the group is skipped
@@ -918,14 +933,22 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         __syncthreads();
     }
     if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // write-backs complete before the block leaves
+#ifdef FASTSGD_TRACE
     if (tid == 0 && blockIdx.x < 480u) {
         a.trace[8u * blockIdx.x + 0] = T0; a.trace[8u * blockIdx.x + 1] = T1; a.trace[8u * blockIdx.x + 2] = T2;
         a.trace[8u * blockIdx.x + 3] = read_globaltimer_dec(); a.trace[8u * blockIdx.x + 4] = taken;
     }
-    // the last block to leave clears the counters for the next launch (the slots were cleared as they were taken)
+#endif
+    // the last block to leave clears the counters for the next launch.  The slots were cleared as they were taken; a
+    // slot whose taker gave up (status TIMEOUT) was filled afterwards with nobody to take it: cleared here, so that
+    // the queue is back in its resting state whatever happened.
     if (tid == 0) {
         __threadfence();
         if (atomicAdd(q_exited, 1u) == gridDim.x - 1u) {
+            if (*reinterpret_cast<volatile unsigned long long*>(a.status) != ~0ull) {
+                const uint32_t reserved = *reinterpret_cast<volatile unsigned int*>(q_reserved);
+                for (uint32_t i = 0; i < reserved && i < a.G; ++i) a.q_list[i] = 0u;
+            }
             a.q_ctl[0] = 0u; *q_taken = 0u; *q_done = 0u; *q_reserved = 0u;
             __threadfence();
             *q_exited = 0u;

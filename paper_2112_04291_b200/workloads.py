@@ -119,6 +119,32 @@ def base_for_keep(v: np.ndarray, keep: int, tau: int = TAU) -> float:
     return float(max(b, 1.0 + 1e-9))
 
 
+def bases_for_keeps(v: np.ndarray, keeps, tau: int = TAU) -> list:
+    """base_for_keep for several kept counts at once (one selection pass over |v|); the same values."""
+    a = np.abs(v)
+    ks = [int(max(1, min(int(k), a.size))) for k in keeps]
+    a.partition(sorted(set(a.size - k for k in ks)))
+    s = float(np.abs(v).sum(dtype=np.float64))
+    out = []
+    for k in ks:
+        q = float(a[a.size - k])
+        if not (q > 0.0) or not (s > q):
+            out.append(1.1)
+        else:
+            out.append(float(max((s / q) ** (1.0 / tau), 1.0 + 1e-9)))
+    return out
+
+
+def _draw_workers(fn, n: int, seeds, threads: int) -> list:
+    """One gradient per seed; with threads > 1 the workers are drawn side by side (numpy's generators
+    release the interpreter lock), which changes nothing in the values."""
+    if threads <= 1 or len(seeds) <= 1:
+        return [fn(n, s) for s in seeds]
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=min(threads, len(seeds))) as ex:
+        return list(ex.map(lambda s: fn(n, s), seeds))
+
+
 @dataclass
 class Workload:
     name: str
@@ -133,31 +159,38 @@ class Workload:
 
 
 def make(name: str, n: int | None = None, workers: int | None = None, keep: float | None = None,
-         seed: int = 0) -> Workload:
+         seed: int = 0, threads: int = 1) -> Workload:
     """The five benchmark configurations (optionally at a reduced n for tests)."""
     if name == "c1":
         n = n or 1_048_576; workers = workers or 1; keep = keep if keep is not None else 0.01
-        grads = [normal(n, seed + w) for w in range(workers)]
-        kcount = keep * n
+        fn = normal
     elif name == "c2":
         n = n or 25_557_032; workers = workers or 4; keep = keep if keep is not None else 0.005
-        grads = [student_t_layers(n, seed + w) for w in range(workers)]
-        kcount = keep * n
+        fn = student_t_layers
     elif name == "c3":
         n = n or 50_000_000; workers = workers or 1
-        grads = [clustered_sparse(n, seed + w) for w in range(workers)]
+        fn = clustered_sparse
+    elif name == "c4":
+        n = n or 335_141_888; workers = workers or 8; keep = keep if keep is not None else 0.001
+        fn = normal_layers
+    elif name == "c5":
+        n = n or (1 << 20); workers = workers or 1; keep = keep if keep is not None else 0.01
+        fn = normal_outliers
+    else:
+        raise ValueError(name)
+    grads = _draw_workers(fn, n, [seed + w for w in range(workers)], threads)
+    if name == "c3":
         nnz = int(np.count_nonzero(grads[0]))
         kcount = (keep if keep is not None else 0.8) * nnz      # keep is a fraction of the nonzeros here
         keep = kcount / n
-    elif name == "c4":
-        n = n or 335_141_888; workers = workers or 8; keep = keep if keep is not None else 0.001
-        grads = [normal_layers(n, seed + w) for w in range(workers)]
-        kcount = keep * n
-    elif name == "c5":
-        n = n or (1 << 20); workers = workers or 1; keep = keep if keep is not None else 0.01
-        grads = [normal_outliers(n, seed + w) for w in range(workers)]
-        kcount = keep * n
     else:
-        raise ValueError(name)
+        kcount = keep * n
     b = base_for_keep(grads[0], int(round(kcount)))
     return Workload(name, n, workers, float(keep), grads, b)
+
+
+def with_keeps(wl: Workload, keeps) -> list:
+    """The same gradients at several keep ratios (fractions of n): one Workload per ratio, sharing the arrays."""
+    bases = bases_for_keeps(wl.grads[0], [int(round(k * wl.n)) for k in keeps])
+    return [Workload(wl.name, wl.n, wl.workers, float(k), wl.grads, b, wl.tau, wl.flag_bits, wl.group_log2)
+            for k, b in zip(keeps, bases)]

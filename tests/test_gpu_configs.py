@@ -238,3 +238,26 @@ def test_config3_key_value_input_as_benchmarked():
         total, d, status = binding.stream_info(out)
         assert status == orc == 0 and total == ostream.size
         assert np.array_equal(out[:total].cpu().numpy(), ostream)
+
+
+def test_key_value_input_scattered_pairs_bert_size():
+    # pairs scattered uniformly over n = 335 M (about 16 per chunk, every chunk touched): the stream of the dense call
+    n = 335_141_888
+    rng = np.random.default_rng(31)
+    keys = np.unique(rng.integers(0, n, 340_000)).astype(np.uint64)
+    vals = rng.laplace(0.0, 1e-2, keys.size).astype(np.float32)
+    v = np.zeros(n, np.float32)
+    v[keys.astype(np.int64)] = vals
+    b = workloads.base_for_keep(v, int(0.8 * keys.size))
+    pg, po = binding.params(b), oracle.params(b)
+    binding.ensure_workspace(n, pg)
+    cap = (min(binding.compress_bound(n, pg), max(4 * n, 1 << 20)) + 255) & ~255
+    out = torch.full((cap,), 0x5A, dtype=torch.uint8, device="cuda")
+    dk = torch.from_numpy(keys.astype(np.uint32).view(np.int32)).cuda()
+    dv = torch.from_numpy(vals).cuda()
+    orc, ostream = oracle.compress(v, po)
+    for rep in range(2):
+        assert binding.compress_kv(dk, dv, n, pg, out) == 0
+        total, d, status = binding.stream_info(out)
+        assert status == orc == 0 and total == ostream.size
+        assert np.array_equal(out[:total].cpu().numpy(), ostream)

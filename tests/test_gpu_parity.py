@@ -680,14 +680,14 @@ def test_paper_key_stream_on_compressed_gradient_keys_and_wide_deltas():
     assert binding.key_encode_paper_bound(10, 9) == 0
 
 
-def _check_kv(keys, vals, n, b, l=2, tau=128):
+def _check_kv(keys, vals, n, b, l=2, tau=128, glog=14, cap=None):
     """fastsgd_compress_kv against the oracle's stream for the same pairs (= the dense vector's stream)."""
     import torch
     import gpu_util as G
-    pg, po = _params(b, tau, l)
+    pg, po = binding.params(b, tau, l, glog), oracle.params(b, tau, l, glog)
     binding.ensure_workspace(n, pg)
-    orc, ostream = oracle.compress_kv(keys, vals, n, po)
-    buf = G.Guarded(binding.compress_bound(n, pg), fill=0x6B)
+    orc, ostream = oracle.compress_kv(keys, vals, n, po, cap)
+    buf = G.Guarded(binding.compress_bound(n, pg) if cap is None else cap, fill=0x6B)
     dk = torch.from_numpy(np.ascontiguousarray(keys, np.uint32).view(np.int32)).to(G.dev())
     dv = torch.from_numpy(np.ascontiguousarray(vals, np.float32)).to(G.dev())
     for rep in range(2):
@@ -739,6 +739,80 @@ def test_key_value_input_with_dense_runs_and_every_flag_size():
     out = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
     assert binding.lib().fastsgd_compress_kv(None, None, 5, n, C.byref(pg), out.data_ptr(), out.numel(), None) == binding.E_NULL
     assert binding.lib().fastsgd_compress_kv(None, None, 0, n, C.byref(pg), None, 0, None) == binding.E_NULL
+
+
+@pytest.mark.parametrize("glog", [4, 8, 12, 16, 20])
+@pytest.mark.parametrize("l", [2, 5])
+def test_key_value_input_other_group_sizes(glog, l):
+    # the key-value encoder takes the group size as a parameter: runs, scattered pairs, a group that spans many chunks
+    rng = np.random.default_rng(100 * glog + l)
+    n = 2_500_003 if glog >= 12 else 300_007
+    parts = [np.arange(5, 2600), rng.choice(n, n // 200, replace=False), np.arange(n - 40_000, n - 1, 3), [n - 1]]
+    keys = np.unique(np.concatenate(parts)).astype(np.uint64)
+    vals = (rng.standard_t(3, keys.size) * 1e-2).astype(np.float32)
+    dense = np.zeros(n, np.float32)
+    dense[keys.astype(np.int64)] = vals
+    b = workloads.base_for_keep(dense, int(0.8 * keys.size))
+    _check_kv(keys, vals, n, b, l=l, glog=glog)
+
+
+@pytest.mark.parametrize("glog", [8, 12, 16, 20])
+@pytest.mark.parametrize("keep_div", [300, 12])
+def test_other_group_sizes_dense_input_and_decoder(glog, keep_div):
+    # group sizes other than the fused encoder's 2^14: streams byte-equal to the oracle's, decoded sums bit-equal
+    import gpu_util as G
+    rng = np.random.default_rng(glog * 7 + keep_div)
+    n = 3_000_017
+    v = workloads.student_t_layers(n, seed=glog, blocks=11)
+    v[rng.integers(0, n, n // 3)] = 0.0
+    b = workloads.base_for_keep(v, n // keep_div)
+    for l in (2, 3):
+        pg, po = binding.params(b, 128, l, glog), oracle.params(b, 128, l, glog)
+        orc, ostream = oracle.compress(v, po)
+        rc, status, gstream, intact = G.gpu_compress(v, pg, fill=0x77)
+        assert rc == 0 and intact and status == orc == 0
+        assert gstream.size == ostream.size and np.array_equal(gstream, ostream)
+        dense0 = rng.standard_normal(n).astype(np.float32)
+        odense = dense0.copy()
+        assert oracle.decompress_accumulate(ostream, n, po, odense) == 0
+        rc, st, gdense, intact = G.gpu_decompress(gstream, n, pg, dense0)
+        assert rc == 0 and st == 0 and intact
+        assert np.allclose(gdense, odense, rtol=RTOL, atol=ATOL) and np.array_equal(gdense, odense)
+
+
+def test_key_value_input_status_words_and_hostile_keys():
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(5)
+    n = 6 * 16384 + 5
+    keys = np.sort(rng.choice(n, 3000, replace=False)).astype(np.uint64)
+    vals = rng.standard_normal(3000).astype(np.float32)
+    dense = np.zeros(n, np.float32)
+    dense[keys.astype(np.int64)] = vals
+    b = workloads.base_for_keep(dense, 2500)
+    pg, po = _params(b)
+    # a capacity that holds header and directory but not the blobs; then one byte short of the stream; then exact
+    full = _check_kv(keys, vals, n, b)
+    for cap in (64 + 8 * 7, full.size - 4, full.size):
+        s = _check_kv(keys, vals, n, b, cap=cap)
+        assert (s.size == full.size) == (cap == full.size)
+    # a value that is not finite; all values zero
+    bad = vals.copy(); bad[17] = np.inf
+    _check_kv(keys, bad, n, b)
+    bad[17] = np.nan
+    _check_kv(keys, bad, n, b)
+    _check_kv(keys, np.zeros_like(vals), n, b)
+    # keys that do not ascend, repeat, or reach beyond n: any stream, but nothing outside the buffers, and the next call is exact
+    binding.ensure_workspace(n, pg)
+    buf = G.Guarded(binding.compress_bound(n, pg), fill=0x6B)
+    for hostile in (keys[::-1].copy(), np.repeat(keys[:1500], 2), np.concatenate([keys[:2990], np.arange(n, n + 10)]),
+                    np.full(3000, 2 ** 32 - 1), rng.integers(0, 2 ** 32, 3000)):
+        dk = torch.from_numpy(np.ascontiguousarray(hostile, np.uint64).astype(np.uint32).view(np.int32)).to(G.dev())
+        dv = torch.from_numpy(vals).to(G.dev())
+        assert binding.compress_kv(dk, dv, n, pg, buf.view) == 0
+        torch.cuda.synchronize()
+        assert buf.intact()
+    _check_kv(keys, vals, n, b)
 
 
 @pytest.mark.parametrize("keep_div", [500, 40, 3])
