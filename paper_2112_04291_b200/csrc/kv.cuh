@@ -171,10 +171,13 @@ __device__ __forceinline__ unsigned long long kv_group_sizes(KvWarp& ws, const K
     uint32_t M = maxd ? 32u - (uint32_t)__clz((int)maxd) : 1u;
     M = min(M, 20u);                                      // (more only with keys that do not ascend)
     __syncwarp();
+    // payload bits exactly as pass 3 lays them out: a delta of bit length bl takes the width of its (clamped) level;
+    // bit length 32 (only with keys that do not ascend) takes the top level, like every length above M
     const uint32_t f = kv_flag_of_bl((uint32_t)lane, a.l, c_inv_m[M]);
     const uint32_t w = ((min(f, (1u << a.l) - 1u) + 1u) * M + (1u << a.l) - 1u) >> a.l;
-    const uint32_t bits = __reduce_add_sync(kFullMask, ws.hist[lane] * w);
+    const uint32_t bits = __reduce_add_sync(kFullMask, ws.hist[lane] * w + (lane == 0 ? ws.hist[32] * M : 0u));
     __syncwarp();
+    if (count > (1u << 20)) count = 0u;                   // more entries than a group has indices (keys that repeat): an empty group
     const uint32_t words = count ? (count * (8u + a.l) + bits + 31u) >> 5 : 0u;
     return (unsigned long long)(count ? (count | (M << 24)) : 0u) | ((unsigned long long)words << 32);
 }
@@ -200,8 +203,10 @@ __device__ __forceinline__ void kv_group_pack(KvWarp& ws, const KvArgs& a, const
             w = ((f + 1u) * M + round_up) >> a.l;
         }
         const uint32_t w_incl = warp_incl_scan(w, lane);
-        if (b.kept) {
-            const uint32_t q = rank + (uint32_t)__popc(b.km & ((1u << lane) - 1u));
+        // (count, M and words come from the workspace entry of the group; with keys that do not ascend a group can have
+        // several first entries and the entry may be another one's: no field is written outside [0, 32 words))
+        const uint32_t q = rank + (uint32_t)__popc(b.km & ((1u << lane) - 1u));
+        if (b.kept && q < count && dpos + w_incl <= 32u * words) {
             const uint32_t code = code_byte_of(thr, a.tau, b.val);
             const uint32_t d = w >= 32u ? b.delta : (b.delta & ((1u << w) - 1u));
             if (in_smem) {
@@ -226,7 +231,7 @@ __device__ __forceinline__ void kv_group_pack(KvWarp& ws, const KvArgs& a, const
             }
         }
         rank += (uint32_t)__popc(b.km);
-        dpos += __shfl_sync(kFullMask, w_incl, 31);
+        dpos = min(dpos + __shfl_sync(kFullMask, w_incl, 31), 32u * words + 1u);      // (beyond the blob only on inconsistent input: stays there)
         if (b.vm != kFullMask) break;
     }
     __syncwarp();
@@ -424,8 +429,10 @@ k_compress_kv(const KvArgs a, const __grid_constant__ PowTable pw) {
                 outw[(kHeaderBytes >> 2) + 2u * g] = cm;
                 outw[(kHeaderBytes >> 2) + 2u * g + 1u] = off;
             }
-            if (count && write_blobs) kv_group_pack<DENSE>(ws, a, s.thr, head_e, g, count, M, words, outw + off, lane);
-            off += words;
+            if (count && write_blobs && M >= 1u && M <= 20u && (uint64_t)count * (8u + a.l) <= 32ull * words &&
+                (uint64_t)off + words <= (uint64_t)fixed_words + words_total)
+                kv_group_pack<DENSE>(ws, a, s.thr, head_e, g, count, M, words, outw + off, lane);
+            off = (uint32_t)min((uint64_t)off + words, (uint64_t)fixed_words + words_total);
         });
         // block 0: the groups after the last one with entries (they start where the stream ends), and the header
         if (blockIdx.x == 0) {
