@@ -218,188 +218,154 @@ __device__ __forceinline__ bool read_dir(const DecArgs& a, const uint32_t* sw, u
     return true;
 }
 
-// One group of one stream, decoded by a warp (BLOCK = false, `t` = lane, `nthreads` = 32) or by the
-// block from `blob` (shared memory copy, or global memory for very large blobs).  A thread owns a
-// run of K consecutive keys; for K <= 8 (up to 2048 keys per block) everything it parses stays in
-// registers between the passes.  With `tile` the values go into the group's slice of dense_out held
-// in shared memory (block path), else straight into dense_out.
-template <int MODE, bool BLOCK>
-__device__ __forceinline__ void decode_group(const DecArgs& a, DecShared& s, const uint32_t* blob, uint32_t nwords,
-                                             uint32_t g, uint32_t count, uint32_t M, const float* val, float* tile,
-                                             int t, int nthreads, int lane, int warp) {
+// Sequential reader of a most-significant-bit-first sequence held as little-endian 32-bit words: fields of up to 32
+// bits, one after the other, from a 64-bit window that is topped up a word at a time (beyond nwords: zeros).
+struct BitReader {
+    const uint32_t*    w;
+    uint32_t           nwords, next;
+    unsigned long long buf;          // the next `avail` bits of the sequence, left-aligned; avail > 32 between calls
+    int                avail;
+    __device__ __forceinline__ void init(const uint32_t* words, uint32_t nw, uint32_t pos) {
+        w = words; nwords = nw;
+        const uint32_t wi = pos >> 5, sh = pos & 31u;
+        const uint32_t w0 = wi < nw ? bswap32(words[wi]) : 0u, w1 = (wi + 1u) < nw ? bswap32(words[wi + 1u]) : 0u;
+        buf = ((((unsigned long long)w0) << 32) | w1) << sh;
+        avail = 64 - (int)sh;
+        next = wi + 2u;
+    }
+    __device__ __forceinline__ uint32_t take(uint32_t nb) {
+        const uint32_t v = nb ? (uint32_t)(buf >> (64u - nb)) : 0u;
+        buf <<= nb;
+        avail -= (int)nb;
+        if (avail <= 32) {
+            const uint32_t x = next < nwords ? bswap32(w[next]) : 0u;
+            buf |= (unsigned long long)x << (32 - avail);
+            avail += 32;
+            ++next;
+        }
+        return v;
+    }
+};
+
+// The four code bytes j, j+1, j+2, j+3 of a blob (byte i in bits 8i.. of the result); two word loads.
+__device__ __forceinline__ uint32_t codes4(const uint32_t* blob, uint32_t nwords, uint32_t j) {
+    const uint32_t wi = j >> 2;
+    const uint32_t w0 = wi < nwords ? blob[wi] : 0u, w1 = (wi + 1u) < nwords ? blob[wi + 1u] : 0u;
+    return __funnelshift_r(w0, w1, 8u * (j & 3u));
+}
+
+// One group of one stream with any number of keys, decoded by the whole block in rounds of 8 keys per thread: a
+// round's flags, widths, deltas and keys stay in registers (one block scan of the widths and one of the deltas per
+// round); the bit position of the next delta and the last key carry over.  A round is validated in full before it is
+// applied; the blob's length, which the flags of ALL rounds imply, is checked when the last round is done.  With
+// `tile` the values go into the group's slice of dense_out held in shared memory, else straight into dense_out.
+template <int MODE>
+__device__ __forceinline__ void decode_long(const DecArgs& a, DecShared& s, const uint32_t* blob, uint32_t nwords,
+                                            uint32_t g, uint32_t count, uint32_t M, const float* val, float* tile,
+                                            int t, int nthreads, int lane, int warp) {
+    constexpr int KMAX = 8;
     const uint64_t lo64 = (uint64_t)g << a.group_log2;
     const uint64_t hi64 = lo64 + (1ull << a.group_log2);
     const uint32_t lo = (uint32_t)lo64;
     const uint32_t hi = (uint32_t)(hi64 < a.n ? hi64 : a.n);
-    const bool lead = (t == 0);
+    const uint32_t levels_m1 = (1u << a.l) - 1u;
     const uint32_t flag_pos0 = 8u * count;
     const uint32_t delta_pos0 = flag_pos0 + a.l * count;
-    const uint32_t levels_m1 = (1u << a.l) - 1u;
-
-    // this thread's run of consecutive keys [jb, je)
-    const uint32_t K = (count + nthreads - 1) / nthreads;
-    const uint32_t jb = min(count, (uint32_t)t * K), je = min(count, jb + K);
-    const bool small = K <= 8u;                       // uniform over the group
-    uint32_t wv[8], dv[8];
-
-    // phase 1: widths from the flags; their sum fixes the blob's length, which must be the directory's
-    uint32_t wsum = 0;
-    if (small) {
+    const uint32_t per_round = (uint32_t)KMAX * (uint32_t)nthreads;
+    uint32_t bitpos = delta_pos0, keybase = lo;
+    bool failed = false;                                  // uniform over the block
+    for (uint32_t r0 = 0; r0 < count; r0 += per_round) {
+        const uint32_t rc = min(per_round, count - r0);
+        const uint32_t K = (rc + nthreads - 1) / nthreads;
+        const uint32_t jb = r0 + min(rc, (uint32_t)t * K), je = r0 + min(rc, (uint32_t)t * K + K);
+        uint32_t wv[KMAX], dv[KMAX], codes[2], wsum = 0u;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            wv[k] = 0u;
-            if (jb + k < je) {
-                const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * (jb + k), a.l);
-                wv[k] = ((f + 1u) * M + levels_m1) >> a.l;
-            }
-            wsum += wv[k];
-        }
-    } else {
-        for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-            wsum += ((f + 1u) * M + levels_m1) >> a.l;
-        }
-    }
-    uint32_t wtotal;
-    const uint32_t pos0 = delta_pos0 + excl_scan<BLOCK>(wsum, &wtotal, s, lane, warp, 0);
-    if ((((uint64_t)delta_pos0 + wtotal + 31ull) >> 5) != nwords) {
-        if (lead) dec_fail(a, g, 0u, kStBadDirectory);
-        return;
-    }
-
-    // phase 2: this thread's deltas and their sum, then the key before its first one
-    uint32_t dsum = 0;
-    if (small) {
-        uint32_t pos = pos0;
+        for (int k0 = 0; k0 < KMAX; k0 += 4) {
+            const uint32_t fb = (jb + k0 < je) ? get_bits(blob, nwords, flag_pos0 + a.l * (jb + k0), a.l * 4u) : 0u;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            dv[k] = get_bits(blob, nwords, pos, wv[k]);       // width 0 beyond the run: reads as 0
-            pos += wv[k];
-            dsum = min(dsum + dv[k], 1u << 21);                // saturates only when already invalid
-        }
-    } else {
-        uint32_t pos = pos0;
-        for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            dsum = min(dsum + get_bits(blob, nwords, pos, w), 1u << 21);
-            pos += w;
-        }
-    }
-    uint32_t dtotal;
-    const uint32_t key0 = lo + excl_scan<BLOCK>(dsum, &dtotal, s, lane, warp, 1);
-
-    // validation of the whole group before anything is applied: first key index that repeats,
-    // leaves the group, or carries a code beyond tau
-    unsigned long long bad = ~0ull;
-    if (small) {
-        uint32_t key = key0;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t j = jb + k;
-            if (j < je && bad == ~0ull) {
-                key += dv[k];
-                const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
-                if ((j > 0 && dv[k] == 0u) || key >= hi) bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
-                else if ((code & 0x7Fu) + 1u > a.tau) bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode;
+            for (int k = k0; k < k0 + 4; ++k) {
+                const uint32_t f = (fb >> (a.l * (uint32_t)(k0 + 3 - k))) & levels_m1;
+                wv[k] = (jb + k < je) ? ((f + 1u) * M + levels_m1) >> a.l : 0u;
+                wsum += wv[k];
             }
         }
-    } else {
-        uint32_t pos = pos0, key = key0;
-        for (uint32_t j = jb; j < je; ++j) {
-            const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-            const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-            const uint32_t delta = get_bits(blob, nwords, pos, w);
-            pos += w;
-            key += delta;
-            const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
-            if ((j > 0 && delta == 0u) || key >= hi) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey; break; }
-            if ((code & 0x7Fu) + 1u > a.tau) { bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode; break; }
+        codes[0] = codes4(blob, nwords, jb);
+        codes[1] = codes4(blob, nwords, jb + 4u);
+        uint32_t wtotal, dtotal;
+        const uint32_t pos0 = bitpos + excl_scan<true>(wsum, &wtotal, s, lane, warp, 0);
+        if (failed) {                                     // only the blob's length is still of interest
+            bitpos = min(bitpos + wtotal, 0xFFF00000u);
+            __syncthreads();                              // (the scan's scratch is rewritten next round)
+            continue;
         }
-    }
-    if (BLOCK) {
-        if (__syncthreads_or(bad != ~0ull)) {             // one barrier when the group is sound
+        BitReader rd;
+        rd.init(blob, nwords, pos0);
+        uint32_t dsum = 0u;
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            dv[k] = rd.take(wv[k]);
+            dsum = min(dsum + dv[k], 1u << 21);
+        }
+        const uint32_t key0 = keybase + excl_scan<true>(dsum, &dtotal, s, lane, warp, 1);
+        unsigned long long bad = ~0ull;
+        {
+            uint32_t key = key0;
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) {
+                const uint32_t j = jb + k;
+                if (j < je && bad == ~0ull) {
+                    key += dv[k];
+                    const uint32_t code = (codes[k >> 2] >> (8u * (uint32_t)(k & 3))) & 0xFFu;
+                    if ((j > 0 && dv[k] == 0u) || key >= hi || key < lo) bad = ((unsigned long long)j << 8) | (unsigned)kStBadKey;
+                    else if ((code & 0x7Fu) + 1u > a.tau) bad = ((unsigned long long)j << 8) | (unsigned)kStBadCode;
+                }
+            }
+        }
+        if (__syncthreads_or(bad != ~0ull)) {             // one barrier when the round is sound
             if (t == 0) s.first_bad = ~0ull;
             __syncthreads();
             if (bad != ~0ull) atomicMin(&s.first_bad, bad);
             __syncthreads();
             bad = s.first_bad;
             __syncthreads();
+            if (t == 0) dec_fail(a, g, (uint32_t)(bad >> 8), (int)(bad & 0xFFull));
+            // nothing more is applied; the remaining rounds only add up the widths, since a blob whose length disagrees
+            // with its flags is reported as that (key index 0: it takes precedence in the status word)
+            failed = true;
+            bitpos = min(bitpos + wtotal, 0xFFF00000u);
+            continue;
         }
-    } else {
-        const uint32_t blo = __reduce_min_sync(kFullMask, (uint32_t)(bad < 0xFFFFFFFFull ? bad : 0xFFFFFFFFull));
-        bad = blo == 0xFFFFFFFFu ? ~0ull : (unsigned long long)blo;
-    }
-    if (bad != ~0ull) {
-        if (lead) dec_fail(a, g, (uint32_t)(bad >> 8), (int)(bad & 0xFFull));
-        return;
-    }
-
-    // phases 3-4 and the aggregation
-    if (small) {
-        uint32_t key = key0;
-        uint32_t kk[8]; float vv[8];
+        {
+            uint32_t key = key0;
+            uint32_t kk[KMAX]; float vv[KMAX], dd[KMAX], res[KMAX];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t j = jb + k;
-            kk[k] = 0xFFFFFFFFu; vv[k] = 0.f;
-            if (j < je) {
-                key += dv[k];
-                const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
-                const float mag = val[(code & 0x7Fu) + 1u];
-                kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
-            }
-        }
-        float dd[8], res[8];                                   // distinct keys: all loads, then all stores
-        if (BLOCK && tile != nullptr) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo] : 0.f;
-            apply_run<MODE, 8>(a, kk, dd, vv, res);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = res[k];
-        } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
-            apply_run<MODE, 8>(a, kk, dd, vv, res);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
-        }
-        return;
-    }
-    {
-        // longer runs: four keys at a time (their loads in flight together)
-        uint32_t pos = pos0, key = key0;
-        for (uint32_t j0 = jb; j0 < je; j0 += 4u) {
-            uint32_t kk[4]; float vv[4], dd[4], res[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t j = j0 + (uint32_t)u;
-                kk[u] = 0xFFFFFFFFu; vv[u] = 0.f;
-                if (j < je) {
-                    const uint32_t f = get_bits(blob, nwords, flag_pos0 + a.l * j, a.l);
-                    const uint32_t w = ((f + 1u) * M + levels_m1) >> a.l;
-                    key += get_bits(blob, nwords, pos, w);
-                    pos += w;
-                    const uint32_t code = (blob[j >> 2] >> (8u * (j & 3u))) & 0xFFu;
+            for (int k = 0; k < KMAX; ++k) {
+                kk[k] = 0xFFFFFFFFu; vv[k] = 0.f;
+                if (jb + k < je) {
+                    key += dv[k];
+                    const uint32_t code = (codes[k >> 2] >> (8u * (uint32_t)(k & 3))) & 0xFFu;
                     const float mag = val[(code & 0x7Fu) + 1u];
-                    kk[u] = key; vv[u] = (code & 0x80u) ? -mag : mag;
+                    kk[k] = key; vv[k] = (code & 0x80u) ? -mag : mag;
                 }
             }
-            if (BLOCK && tile != nullptr) {
+            if (tile != nullptr) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) dd[u] = kk[u] != 0xFFFFFFFFu ? tile[kk[u] - lo] : 0.f;
-                apply_run<MODE, 4>(a, kk, dd, vv, res);
+                for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo] : 0.f;
+                apply_run<MODE, KMAX>(a, kk, dd, vv, res);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) if (kk[u] != 0xFFFFFFFFu) tile[kk[u] - lo] = res[u];
+                for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo] = res[k];
             } else {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) dd[u] = kk[u] != 0xFFFFFFFFu ? a.dense[kk[u]] : 0.f;
-                apply_run<MODE, 4>(a, kk, dd, vv, res);
+                for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
+                apply_run<MODE, KMAX>(a, kk, dd, vv, res);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) if (kk[u] != 0xFFFFFFFFu) a.dense[kk[u]] = res[u];
+                for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
             }
         }
+        bitpos = min(bitpos + wtotal, 0xFFF00000u);
+        keybase = min(keybase + dtotal, 0xFFF00000u);     // (saturate only when already invalid)
     }
+    if ((((uint64_t)bitpos + 31ull) >> 5) != nwords && t == 0) dec_fail(a, g, 0u, kStBadDirectory);
 }
 
 // Exclusive scans of NS values per thread at once (one barrier for all of them in a block).
@@ -919,8 +885,8 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 const float* v1[1] = {s.val[w]};
                 decode_multi<MODE, true, 1, 4>(a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
             } else {
-                decode_group<MODE, true>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
-                                   tid, kDecThreads, lane, warp);
+                decode_long<MODE>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                                  tid, kDecThreads, lane, warp);
             }
             __syncthreads();       // these streams' updates before the next stream's
         }
