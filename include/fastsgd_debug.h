@@ -36,6 +36,12 @@ uint64_t fastsgd_launch_count(void);
  * milliseconds; production code never calls this. */
 int fastsgd_debug_set_wait_limits(uint32_t block_polls, uint32_t copy_tries, uint32_t queue_polls);
 
+/* Caps the number of thread blocks of the encoders' launches (fastsgd_compress,
+ * _batch, _kv) that follow; 0 restores the default (as many as are resident at
+ * once).  With a cap the batch encoder does not split its blocks into two
+ * teams.  The stream never depends on the grid: tests use this to show it. */
+int fastsgd_debug_set_grid(uint32_t blocks);
+
 /* Byte offsets inside the registered workspace (all of them in its fixed first
  * part): [0] u32 bar_count[8], arrivals at each gradient's grid barrier;
  * [1] u32 ne_count[8], tiles the last encoder launch read a second time, per

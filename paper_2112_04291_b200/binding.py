@@ -30,7 +30,7 @@ EXPORTS = [
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
     "fastsgd_sparse_adam_update_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
     "fastsgd_compress_kv",
-    "fastsgd_debug_set_wait_limits", "fastsgd_debug_layout", "fastsgd_debug_trace_compiled",
+    "fastsgd_debug_set_wait_limits", "fastsgd_debug_layout", "fastsgd_debug_trace_compiled", "fastsgd_debug_set_grid",
 ]
 
 
@@ -115,6 +115,8 @@ def lib():
         L.fastsgd_kernel_timing_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         L.fastsgd_debug_set_wait_limits.restype = C.c_int
         L.fastsgd_debug_set_wait_limits.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32]
+        L.fastsgd_debug_set_grid.restype = C.c_int
+        L.fastsgd_debug_set_grid.argtypes = [C.c_uint32]
         L.fastsgd_debug_layout.restype = C.c_int
         L.fastsgd_debug_layout.argtypes = [u64p, C.c_uint32]
         L.fastsgd_debug_trace_compiled.restype = C.c_int
@@ -321,6 +323,11 @@ def debug_set_wait_limits(block_polls: int = 0, copy_tries: int = 0, queue_polls
     """fastsgd_debug_set_wait_limits: shorten (or, with zeros, restore) the kernels' bounded waits.  Test aid."""
     _check(lib().fastsgd_debug_set_wait_limits(int(block_polls), int(copy_tries), int(queue_polls)),
            "fastsgd_debug_set_wait_limits")
+
+
+def debug_set_grid(blocks: int = 0) -> None:
+    """fastsgd_debug_set_grid: cap the encoders' thread blocks (0: default).  Test aid."""
+    _check(lib().fastsgd_debug_set_grid(int(blocks)), "fastsgd_debug_set_grid")
 
 
 LAYOUT_FIELDS = ("bar_count", "ne_count", "error", "decoder_trace", "encoder_trace", "encoder_trace_bytes",

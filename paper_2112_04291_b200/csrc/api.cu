@@ -33,6 +33,7 @@ struct State {
     int        kv_blocks_per_sm = 0;
     bool       attrs_set = false;
     bool       timed_out = false;          // a status query saw FASTSGD_ST_TIMEOUT: the workspace's counters are not at rest
+    uint32_t   grid_override = 0;          // blocks of the encoders' launches (0: as many as are resident); tests only
     uint32_t   wait_limit = kWaitLimit;    // bounded waits of the kernels (shortened only by fastsgd_debug_set_wait_limits)
     uint32_t   try_limit = kTryLimit;
     uint32_t   dec_spin_limit = kDecSpinLimit;
@@ -222,6 +223,12 @@ int fastsgd_debug_set_wait_limits(uint32_t block_polls, uint32_t copy_tries, uin
     return FASTSGD_OK;
 }
 
+int fastsgd_debug_set_grid(uint32_t blocks) {
+    std::lock_guard<std::mutex> lock(g_state.mu);
+    g_state.grid_override = blocks;
+    return FASTSGD_OK;
+}
+
 int fastsgd_debug_layout(uint64_t* offsets, uint32_t count) {
     if (!offsets) return FASTSGD_E_NULL;
     const uint64_t v[FASTSGD_DEBUG_LAYOUT_FIELDS] = {
@@ -336,6 +343,7 @@ int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, u
     const uint64_t cap = (uint64_t)g_state.sm_count * (uint64_t)(g_state.kv_blocks_per_sm > 2 ? 2 : g_state.kv_blocks_per_sm);
     if (grid > cap) grid = cap;
     if (grid > kKvMaxGrid) grid = kKvMaxGrid;
+    if (g_state.grid_override && g_state.grid_override < grid) grid = g_state.grid_override;
     if (grid < 1) grid = 1;
     const uint64_t warps = grid * kKvWarps;
     uint64_t slice = (units + warps - 1) / warps;
@@ -394,6 +402,7 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
     if (grid > kMaxCtas) grid = kMaxCtas;
     const uint64_t grid_full = grid;
+    if (g_state.grid_override && g_state.grid_override < grid) grid = g_state.grid_override;      // (never two teams then)
     if (grid > G) grid = G;
     for (uint32_t first = 0; first < num_grads; first += kCmpMaxJobs) {
         CmpBatch cb;
@@ -414,7 +423,7 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
         uint64_t launch_grid = grid;
         cb.teams = 1u;
         if (cb.jobs >= 2u && g_state.cmp_blocks_per_sm >= 2 && grid_full == 2ull * (uint64_t)g_state.sm_count &&
-            g_state.sm_count <= 256 && G >= grid_full) {
+            g_state.sm_count <= 256 && G >= grid_full && !g_state.grid_override) {
             cb.teams = 2u;
             launch_grid = grid_full;
         } else if (cb.jobs == 1u) {

@@ -359,9 +359,11 @@ k_compress_kv(const KvArgs a, const __grid_constant__ PowTable pw) {
     const bool finite = isfinite(S);
     if (tid <= (int)a.tau)
         s.thr[tid] = (finite && S != 0.0) ? fmaxf(__double2float_ru(__ddiv_rn(S, pw.P[tid])), __int_as_float(1)) : __int_as_float(0x7f800000);
-    if (tid == 0) {
-        s.thr[130] = (float)log2(S);
-        s.thr[131] = (float)(1.0 / log2(a.base));
+    if (tid == 0) {                                       // (estimates that only steer the table search: see make_table)
+        const unsigned long long sb = (unsigned long long)__double_as_longlong(S);
+        const float mant = __uint_as_float(0x3F800000u | (uint32_t)((sb >> 29) & 0x7FFFFFull));
+        s.thr[130] = (float)((int)((sb >> 52) & 0x7FFull) - 1023) + __log2f(mant);
+        s.thr[131] = 1.0f / __log2f((float)a.base);
     }
     __syncthreads();
     const float thr_e = s.thr[a.tau];

@@ -185,6 +185,42 @@ def _damage(stream, pos, value, width=4):
     return s
 
 
+@pytest.mark.parametrize("blocks", [1, 7, 37, 148, 211])
+def test_same_bytes_whatever_the_grid(blocks):
+    # the fixed sum tree and the order-preserving offsets make the stream a function of the input alone: one gradient,
+    # three gradients in one launch and key-value input, each with the launch capped at `blocks` thread blocks
+    import torch
+    import gpu_util as G
+    n = 2_000_003
+    host = [workloads.student_t_layers(n, seed=70 + w, blocks=5) for w in range(3)]
+    b = workloads.base_for_keep(host[0], n // 150)
+    pg, po = _params(b)
+    binding.ensure_workspace(n, pg)
+    want = [oracle.compress(v, po)[1] for v in host]
+    grads = [torch.from_numpy(v).cuda() for v in host]
+    cap = binding.compress_bound(n, pg)
+    outs = [torch.zeros(cap, dtype=torch.uint8, device="cuda") for _ in range(3)]
+    keys = np.flatnonzero(np.abs(host[0]) > 1e-3)
+    dk = torch.from_numpy(keys.astype(np.uint32).view(np.int32)).cuda()
+    dv = torch.from_numpy(host[0][keys]).cuda()
+    sparse = np.zeros(n, np.float32); sparse[keys] = host[0][keys]
+    want_kv = oracle.compress(sparse, po)[1]
+    try:
+        binding.debug_set_grid(blocks)
+        assert binding.compress(grads[0], pg, outs[0]) == 0
+        total, d, status = binding.stream_info(outs[0])
+        assert status == 0 and np.array_equal(outs[0][:total].cpu().numpy(), want[0])
+        assert binding.compress_batch(grads, pg, outs) == 0
+        for w in range(3):
+            total, d, status = binding.stream_info(outs[w])
+            assert status == 0 and np.array_equal(outs[w][:total].cpu().numpy(), want[w]), w
+        assert binding.compress_kv(dk, dv, n, pg, outs[1]) == 0
+        total, d, status = binding.stream_info(outs[1])
+        assert status == 0 and np.array_equal(outs[1][:total].cpu().numpy(), want_kv)
+    finally:
+        binding.debug_set_grid(0)
+
+
 def test_damaged_streams_report_the_oracles_status_and_stay_in_bounds():
     import gpu_util as G
     n = 5 * 16384 + 100
