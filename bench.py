@@ -344,7 +344,7 @@ def series_stats(ts):
     return {"median": statistics.median(ts), "min": min(ts)}
 
 
-def measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs=None, dense=None):
+def measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs=None, dense=None, use_graph=True):
     """One compact entry of the `configs` table: compress-only, decompress-only and combined, every repetition
     timed by its own pair of CUDA events after 256 MiB were written (L2-cold); median and min."""
     n, W = wl.n, wl.workers
@@ -379,6 +379,23 @@ def measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs=None,
     kept = [d for _, d, _ in infos]
     listed = binding.listed_tiles(W)
 
+    # the same C-ABI calls replayed from CUDA graphs, as the headline step is (eager calls if capture fails)
+    def graph_of(fn):
+        if not use_graph:
+            return fn
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            g.replay()
+            torch.cuda.synchronize()
+            return g.replay
+        except Exception as exc:
+            print(f"[bench] CUDA graph capture failed, launching eagerly: {exc}", file=sys.stderr)
+            return fn
+
+    comp_run, dec_run, both_run = graph_of(comp), graph_of(dec), graph_of(both)
+
     def series(fn, cold):
         ts = []
         for it in range(reps + 3):
@@ -393,7 +410,7 @@ def measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs=None,
                 ts.append(e0.elapsed_time(e1))
         return ts
 
-    tc, td, tb = series(comp, True), series(dec, True), series(both, True)
+    tc, td, tb = series(comp_run, True), series(dec_run, True), series(both_run, True)
     in_bytes = 4.0 * n * W
     alg_c = 8.0 * n * W + float(sum(stream_bytes))
     alg_d = float(sum(stream_bytes)) + 8.0 * float(sum(kept))
@@ -412,13 +429,13 @@ def measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs=None,
     if entry["frac"] > 1.2:
         entry["note"] = "frac counts two full reads of every gradient; the kernel skipped most tiles: dram_frac is the hardware figure"
     if in_bytes < L2_BYTES:
-        tw = series(both, False)
+        tw = series(both_run, False)
         entry["combined_ms_l2_warm"] = series_stats(tw)
     assert all(binding.stream_info(o)[2] == 0 for o in outs) and binding.decode_status() == 0
     return entry
 
 
-def configs_table(torch, binding, workloads, dev, peak, reps, c2_entry):
+def configs_table(torch, binding, workloads, dev, peak, reps, c2_entry, use_graph=True):
     """Every benchmark configuration besides the headline: c1, c3, c4 at three keep ratios with its 8 workers, c5 at
     n = 2^26, 2^28, 2^30 at four keep ratios.  Inputs are drawn on the host (the same seeded generators as the
     parity tests), the next workload while the current one is being timed."""
@@ -447,7 +464,7 @@ def configs_table(torch, binding, workloads, dev, peak, reps, c2_entry):
             dense = torch.zeros(n, dtype=torch.float32, device=dev)
             for wl in wls:
                 key = name if len(wls) == 1 else "%s_keep_%g" % (name, wl.keep_fraction)
-                table[key] = measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs, dense)
+                table[key] = measure_config(torch, binding, dev, wl, grads, peak, reps, flush, outs, dense, use_graph)
             del grads, outs, dense, wls
             torch.cuda.empty_cache()
     return table
@@ -875,7 +892,8 @@ def main():
         del grads, outs, dense, host_grads, wl
         torch.cuda.empty_cache()
         try:
-            line["configs"] = configs_table(torch, binding, workloads, dev, peak, 20, c2_entry)
+            line["configs"] = configs_table(torch, binding, workloads, dev, peak, 20, c2_entry, use_graph=not args.no_graph)
+            line["configs_launch"] = "every leg a CUDA graph replay of its C-ABI calls, each repetition timed by its own pair of events after 256 MiB were written" if not args.no_graph else "eager C-ABI calls"
         except Exception as exc:          # the headline stands by itself
             line["configs"] = {"c2": c2_entry}
             line["configs_error"] = repr(exc)

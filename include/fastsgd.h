@@ -15,9 +15,11 @@
  *   - The caller owns every buffer.  The library allocates nothing; its scratch
  *     memory is the workspace the caller registers with fastsgd_set_workspace.
  *   - fastsgd_compress and fastsgd_decompress_accumulate only enqueue kernels
- *     on `stream` (a cudaStream_t passed as void*) and return at once.  All
- *     calls that share a workspace must be issued on one stream (or otherwise
- *     serialised): they share the workspace.
+ *     on `stream` (a cudaStream_t passed as void*) and return at once.  The
+ *     library keeps one workspace per device (the one registered while that
+ *     device was current); all calls on a device must be issued on one stream
+ *     (or otherwise serialised): they share that workspace.  Different devices
+ *     of one process are independent of each other.
  *   - Return value: 0 or a negative FASTSGD_E_* for what the host can see.
  *     What only the device can see is reported in a status word: the stream
  *     header's for compress (fastsgd_stream_info), the workspace's for

@@ -21,11 +21,10 @@ namespace {
 
 using namespace fsg;
 
+// Per device: the registered workspace and what the launches need to know about the GPU.
 struct State {
-    std::mutex mu;
     void*      ws = nullptr;
     uint64_t   ws_bytes = 0;
-    int        device = -1;
     int        sm_count = 0;
     int        sum_blocks_per_sm = 0;
     int        dec_blocks_per_sm = 0;
@@ -33,12 +32,28 @@ struct State {
     int        kv_blocks_per_sm = 0;
     bool       attrs_set = false;
     bool       timed_out = false;          // a status query saw FASTSGD_ST_TIMEOUT: the workspace's counters are not at rest
+};
+// Process-wide test settings (fastsgd_debug_*).
+struct Tunables {
     uint32_t   grid_override = 0;          // blocks of the encoders' launches (0: as many as are resident); tests only
     uint32_t   wait_limit = kWaitLimit;    // bounded waits of the kernels (shortened only by fastsgd_debug_set_wait_limits)
     uint32_t   try_limit = kTryLimit;
     uint32_t   dec_spin_limit = kDecSpinLimit;
 };
-State g_state;
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;                           // guards everything below (host side only: the calls of one device share its workspace)
+State      g_states[kMaxDevices];
+Tunables   g_tun;
+
+// the state of the current device (caller holds g_mu)
+State* device_state() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); dev = 0; }      // (no device at all: the argument checks still answer)
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
+    return &g_states[dev];
+}
+#define FSG_DEVICE_STATE() State* sp_ = device_state(); if (!sp_) return FASTSGD_E_CUDA; State& g_state = *sp_
+
 std::atomic<uint64_t> g_launches{0};
 
 // optional per-kernel timing (profiling aid)
@@ -116,10 +131,11 @@ WorkspaceView view(void* ws, uint64_t n, uint32_t group_log2 = kGroupLog2) {
 }
 
 int ensure_device_setup() {
-    // caller holds g_state.mu
+    // caller holds g_mu; once per device
+    FSG_DEVICE_STATE();
+    if (g_state.attrs_set) return FASTSGD_OK;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return FASTSGD_E_CUDA;
-    if (g_state.attrs_set && g_state.device == dev) return FASTSGD_OK;
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_compress<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CmpSmem)) != cudaSuccess)
@@ -164,7 +180,6 @@ int ensure_device_setup() {
         b2 = b2x[0];
         for (int i = 1; i < 4; ++i) if (b2x[i] < b2) b2 = b2x[i];
     }
-    g_state.device = dev;
     g_state.sm_count = sms;
     g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
     g_state.dec_blocks_per_sm = b2 > 0 ? b2 : 1;
@@ -176,6 +191,7 @@ bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p
 
 int launch_sum(const float* grad, uint64_t n, uint32_t groups, uint32_t tau, const PowTable& pw,
                const WorkspaceView& w, double* sum_out, cudaStream_t st) {
+    FSG_DEVICE_STATE();
     SumArgs sa;
     sa.grad = grad; sa.n = n; sa.chunks = (uint32_t)chunks_of(n); sa.groups = groups; sa.tau = tau;
     sa.ctl = w.ctl; sa.thr = w.thr; sa.partials = w.partials; sa.desc = w.desc; sa.sum_out = sum_out;
@@ -193,14 +209,14 @@ extern "C" {
 int fastsgd_version(void) { return 1; }
 
 int fastsgd_kernel_timing_enable(int enable) {
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
     g_timing = enable != 0;
     return FASTSGD_OK;
 }
 
 int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]) {
     if (!ms_total || !launches) return FASTSGD_E_NULL;
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
     for (int i = 0; i < 3; ++i) { ms_total[i] = 0.0; launches[i] = 0; }
     int rc = FASTSGD_OK;
     for (const TimedLaunch& t : g_timed) {
@@ -216,16 +232,16 @@ int fastsgd_kernel_timing_read(double ms_total[3], uint64_t launches[3]) {
 uint64_t fastsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int fastsgd_debug_set_wait_limits(uint32_t block_polls, uint32_t copy_tries, uint32_t queue_polls) {
-    std::lock_guard<std::mutex> lock(g_state.mu);
-    g_state.wait_limit = block_polls ? block_polls : kWaitLimit;
-    g_state.try_limit = copy_tries ? copy_tries : kTryLimit;
-    g_state.dec_spin_limit = queue_polls == 0xFFFFFFFFu ? 0u : (queue_polls ? queue_polls : kDecSpinLimit);
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_tun.wait_limit = block_polls ? block_polls : kWaitLimit;
+    g_tun.try_limit = copy_tries ? copy_tries : kTryLimit;
+    g_tun.dec_spin_limit = queue_polls == 0xFFFFFFFFu ? 0u : (queue_polls ? queue_polls : kDecSpinLimit);
     return FASTSGD_OK;
 }
 
 int fastsgd_debug_set_grid(uint32_t blocks) {
-    std::lock_guard<std::mutex> lock(g_state.mu);
-    g_state.grid_override = blocks;
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_tun.grid_override = blocks;
     return FASTSGD_OK;
 }
 
@@ -291,7 +307,8 @@ int fastsgd_set_workspace(void* dev_ptr, uint64_t bytes, void* stream) {
     if (!dev_ptr) return FASTSGD_E_NULL;
     if (!aligned(dev_ptr, 256)) return FASTSGD_E_ALIGN;
     if (bytes < kPartialsOffset) return FASTSGD_E_NO_WORKSPACE;   // control block, tables, trace, decoder queue
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     int rc = ensure_device_setup();
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -309,7 +326,8 @@ int fastsgd_abs_sum(const float* grad, uint64_t n, double* sum_out, void* stream
     if (!aligned(grad, 16) || !aligned(sum_out, 8)) return FASTSGD_E_ALIGN;
     int rc = check_n(n);
     if (rc) return rc;
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     if (!g_state.ws || g_state.ws_bytes < ws_bytes_for(n, kGroupLog2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
@@ -323,6 +341,7 @@ namespace {
 // entries itself, read as the list (i, v_i), with its sum already in the workspace.  Caller holds g_state.mu.
 int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
                         const fastsgd_params* params, const PowTable& pw, void* out, uint64_t out_bytes, cudaStream_t st) {
+    FSG_DEVICE_STATE();
     if (g_state.kv_blocks_per_sm < 1) return FASTSGD_E_CUDA;
     const uint64_t G = groups_of(n, params->group_log2);
     WorkspaceView w = view(g_state.ws, n, params->group_log2);
@@ -335,7 +354,7 @@ int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, u
     ka.blk_agg = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(g_state.ws) + kKvAggOffset);
     ka.base = params->base; ka.G = (uint32_t)G; ka.chunks = (uint32_t)chunks_of(n);
     ka.tau = params->tau; ka.l = params->flag_bits; ka.group_log2 = params->group_log2;
-    ka.wait_limit = g_state.wait_limit; ka.given_sum = dense ? 1u : 0u;
+    ka.wait_limit = g_tun.wait_limit; ka.given_sum = dense ? 1u : 0u;
     // a warp per 32 list entries (dense: per group) until the GPU is full; all blocks are resident: they meet at grid barriers
     const uint64_t units = dense ? G : count;
     const uint64_t per_warp = dense ? 1ull : 32ull;
@@ -343,7 +362,7 @@ int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, u
     const uint64_t cap = (uint64_t)g_state.sm_count * (uint64_t)(g_state.kv_blocks_per_sm > 2 ? 2 : g_state.kv_blocks_per_sm);
     if (grid > cap) grid = cap;
     if (grid > kKvMaxGrid) grid = kKvMaxGrid;
-    if (g_state.grid_override && g_state.grid_override < grid) grid = g_state.grid_override;
+    if (g_tun.grid_override && g_tun.grid_override < grid) grid = g_tun.grid_override;
     if (grid < 1) grid = 1;
     const uint64_t warps = grid * kKvWarps;
     uint64_t slice = (units + warps - 1) / warps;
@@ -379,7 +398,8 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
     const uint64_t G = groups_of(n, params->group_log2);
     if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
     if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;   // descriptor fields are 31 bits
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
@@ -402,7 +422,7 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
     uint64_t grid = (uint64_t)g_state.sm_count * g_state.cmp_blocks_per_sm;
     if (grid > kMaxCtas) grid = kMaxCtas;
     const uint64_t grid_full = grid;
-    if (g_state.grid_override && g_state.grid_override < grid) grid = g_state.grid_override;      // (never two teams then)
+    if (g_tun.grid_override && g_tun.grid_override < grid) grid = g_tun.grid_override;      // (never two teams then)
     if (grid > G) grid = G;
     for (uint32_t first = 0; first < num_grads; first += kCmpMaxJobs) {
         CmpBatch cb;
@@ -416,14 +436,14 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
         cb.sm_slots = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kSmSlotOffset);
         cb.dense_scratch = static_cast<unsigned char*>(g_state.ws) + ws_dense_offset(n, params->group_log2);
         cb.base = params->base; cb.G = (uint32_t)G; cb.tau = params->tau; cb.l = params->flag_bits;
-        cb.wait_limit = g_state.wait_limit; cb.try_limit = g_state.try_limit;
+        cb.wait_limit = g_tun.wait_limit; cb.try_limit = g_tun.try_limit;
         // Two or more gradients, two resident blocks per SM and enough tiles: the two blocks of an SM
         // form two teams that work on different gradients.  One gradient: the tiles below the grid
         // size are assigned statically, so every block gets an equal share.
         uint64_t launch_grid = grid;
         cb.teams = 1u;
         if (cb.jobs >= 2u && g_state.cmp_blocks_per_sm >= 2 && grid_full == 2ull * (uint64_t)g_state.sm_count &&
-            g_state.sm_count <= 256 && G >= grid_full && !g_state.grid_override) {
+            g_state.sm_count <= 256 && G >= grid_full && !g_tun.grid_override) {
             cb.teams = 2u;
             launch_grid = grid_full;
         } else if (cb.jobs == 1u) {
@@ -465,7 +485,8 @@ int fastsgd_compress_kv(const uint32_t* keys, const float* values, uint64_t coun
     const uint64_t G = groups_of(n, params->group_log2);
     if (out_bytes < kHeaderBytes + 8ull * G) return FASTSGD_E_CAPACITY;
     if (bound_bytes(n, params) / 4ull >= (1ull << 31)) return FASTSGD_E_BAD_N;
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
@@ -500,7 +521,8 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
         if (!aligned(streams_in[i], 16)) return FASTSGD_E_ALIGN;
         if (bytes[i] < kHeaderBytes) return FASTSGD_E_TRUNCATED;
     }
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     if (!g_state.ws || g_state.timed_out || g_state.ws_bytes < ws_bytes_for(n, params->group_log2)) return FASTSGD_E_NO_WORKSPACE;
     rc = ensure_device_setup();
     if (rc) return rc;
@@ -532,7 +554,7 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
         da.q_list = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(g_state.ws) + kQueueOffset);
         da.base = params->base; da.G = (uint32_t)G; da.tau = params->tau; da.l = params->flag_bits;
         da.group_log2 = params->group_log2;
-        da.spin_limit = g_state.dec_spin_limit; da.try_limit = g_state.try_limit;
+        da.spin_limit = g_tun.dec_spin_limit; da.try_limit = g_tun.try_limit;
         if (adam) {
             da.theta = theta; da.m = m; da.v = v;
             da.lr = adam->lr; da.beta1 = adam->beta1; da.beta2 = adam->beta2; da.eps = adam->eps;
@@ -586,10 +608,13 @@ int fastsgd_key_encode_paper(const uint32_t* keys, uint64_t d, uint32_t flag_bit
     const uint64_t need = fastsgd_key_encode_paper_bound(d, flag_bits);
     if (!need) return FASTSGD_E_BAD_PARAM;
     if (out_bytes < need) return FASTSGD_E_CAPACITY;
+    int sm_count = 0;
     {
-        std::lock_guard<std::mutex> lock(g_state.mu);
+        std::lock_guard<std::mutex> lock(g_mu);
+        FSG_DEVICE_STATE();
         const int rc = ensure_device_setup();
         if (rc) return rc;
+        sm_count = g_state.sm_count;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     BkArgs a;
@@ -600,7 +625,7 @@ int fastsgd_key_encode_paper(const uint32_t* keys, uint64_t d, uint32_t flag_bit
     a.bk = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(out) + 16 + 8ull * a.blocks);
     if (cudaMemsetAsync(out, 0, 16, st) != cudaSuccess) return FASTSGD_E_CUDA;
     if (a.blocks) {
-        const unsigned cap = 8u * (unsigned)g_state.sm_count;
+        const unsigned cap = 8u * (unsigned)sm_count;
         const unsigned want = (unsigned)((d + kBkThreads - 1) / kBkThreads);
         k_bk_maxdelta<<<want < cap ? want : cap, kBkThreads, 0, st>>>(a);
         k_bk_sizes<<<a.blocks, kBkThreads, 0, st>>>(a);
@@ -629,7 +654,8 @@ int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_byt
     std::memcpy(&s32, h + 8, 4);
     if (status) *status = (int)s32;
     if (s32 == (uint32_t)FASTSGD_ST_TIMEOUT) {        // the launch that wrote this stream left the workspace's counters mid-way
-        std::lock_guard<std::mutex> lock(g_state.mu);
+        std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
         g_state.timed_out = true;
     }
     if (d) { std::memcpy(&v, h + 24, 8); *d = v; }
@@ -639,7 +665,8 @@ int fastsgd_stream_info(const void* stream_in, void* stream, uint64_t* total_byt
 
 int fastsgd_decode_status(void* stream, int* status) {
     if (!status) return FASTSGD_E_NULL;
-    std::lock_guard<std::mutex> lock(g_state.mu);
+    std::lock_guard<std::mutex> lock(g_mu);
+    FSG_DEVICE_STATE();
     if (!g_state.ws) return FASTSGD_E_NO_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long v = 0;
@@ -707,12 +734,27 @@ int fastsgd_decompress_accumulate_host(const void* const* streams_host, const ui
     } else {
         if (cudaMemsetAsync(ddense, 0, 4ull * n, st) != cudaSuccess) return FASTSGD_E_CUDA;
     }
-    for (uint32_t i = 0; i < num_streams; ++i) {
-        if (!streams_host[i]) return FASTSGD_E_NULL;
-        if (bytes[i] > need - dense_bytes) return FASTSGD_E_NO_WORKSPACE;
-        // the staging area is reused: stream order keeps copy i+1 behind decode i
-        if (cudaMemcpyAsync(dstream, streams_host[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
-        int rc2 = fastsgd_decompress_accumulate(dstream, bytes[i], n, params, ddense, stream);
+    // The streams are copied side by side into the staging area (16-byte aligned each) as long as they fit, then decoded
+    // by one batched launch per 8; a stream that does not fit beside the others starts a new round (stream order keeps
+    // the next round's copies behind this round's launch).
+    const uint64_t room = need - dense_bytes;
+    uint32_t i = 0;
+    while (i < num_streams) {
+        std::vector<const void*> ptrs;
+        std::vector<uint64_t> sizes;
+        uint64_t used = 0;
+        while (i < num_streams) {
+            if (!streams_host[i]) return FASTSGD_E_NULL;
+            if (bytes[i] > room) return FASTSGD_E_NO_WORKSPACE;
+            const uint64_t padded = (bytes[i] + 15ull) & ~15ull;
+            if (used + padded > room) break;
+            if (cudaMemcpyAsync(dstream + used, streams_host[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTSGD_E_CUDA;
+            ptrs.push_back(dstream + used);
+            sizes.push_back(bytes[i]);
+            used += padded;
+            ++i;
+        }
+        int rc2 = fastsgd_decompress_accumulate_batch(ptrs.data(), sizes.data(), (uint32_t)ptrs.size(), n, params, ddense, stream);
         if (rc2) return rc2;
     }
     if (cudaMemcpyAsync(dense_host, ddense, 4ull * n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTSGD_E_CUDA;
