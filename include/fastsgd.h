@@ -105,12 +105,16 @@ typedef struct fastsgd_params {
  * carrying the status is written.  Nothing outside out[0, out_bytes) is
  * written.
  * Group sizes: T = 2^14 is what the fused kernel is built for (its tile is the
- * group).  Any other group_log2 in 8..20 takes a general path -- the sum kernel,
- * then the list encoder of fastsgd_compress_kv run over the dense gradient, two
- * launches per gradient and three reads of it -- with the same stream as the
- * definition gives (the paper's Algorithm 2 has no groups: it is the case
- * T >= n).  Below 2^8: FASTSGD_E_NOT_IMPLEMENTED.  The decoder takes the same
- * range as long as the stream has at most 2^17 groups.
+ * group).  Any other group_log2 in 8..20 takes a general path: the sum kernel,
+ * a kernel that selects the kept entries (i, v_i), |v_i| >= B_tau, into a list
+ * in the workspace, and the list encoder of fastsgd_compress_kv on that list
+ * (three reads of the gradient, about 1.5 times the fused kernel's time; a list
+ * beyond 4.5 M pairs does not fit and the list encoder then walks the dense
+ * gradient itself, a warp per group, which is slow for large groups).  The
+ * stream is the one the definition gives for that group size (the paper's
+ * Algorithm 2 has no groups: it is the case T >= n).  Below 2^8:
+ * FASTSGD_E_NOT_IMPLEMENTED.  The decoder takes the same range as long as the
+ * stream has at most 2^17 groups.
  * The kernel is launched cooperatively (all its thread blocks resident at
  * once, two per SM) and its blocks wait for one another with bounded waits; if
  * one of them runs out (it should not on a GPU the kernel has to itself) every

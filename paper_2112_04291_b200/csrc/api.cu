@@ -340,7 +340,8 @@ namespace {
 // The list encoder (kv.cuh).  dense = false: `count` key-value pairs.  dense = true: the gradient `values` of n
 // entries itself, read as the list (i, v_i), with its sum already in the workspace.  Caller holds g_state.mu.
 int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, uint64_t count, uint64_t n,
-                        const fastsgd_params* params, const PowTable& pw, void* out, uint64_t out_bytes, cudaStream_t st) {
+                        const fastsgd_params* params, const PowTable& pw, void* out, uint64_t out_bytes, cudaStream_t st,
+                        const unsigned long long* count_dev = nullptr, uint32_t run_if = 0u, bool given_sum = false) {
     FSG_DEVICE_STATE();
     if (g_state.kv_blocks_per_sm < 1) return FASTSGD_E_CUDA;
     const uint64_t G = groups_of(n, params->group_log2);
@@ -354,9 +355,10 @@ int launch_list_encoder(bool dense, const uint32_t* keys, const float* values, u
     ka.blk_agg = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(g_state.ws) + kKvAggOffset);
     ka.base = params->base; ka.G = (uint32_t)G; ka.chunks = (uint32_t)chunks_of(n);
     ka.tau = params->tau; ka.l = params->flag_bits; ka.group_log2 = params->group_log2;
-    ka.wait_limit = g_tun.wait_limit; ka.given_sum = dense ? 1u : 0u;
+    ka.wait_limit = g_tun.wait_limit; ka.given_sum = (dense || given_sum) ? 1u : 0u;
+    ka.count_dev = count_dev; ka.run_if = run_if;
     // a warp per 32 list entries (dense: per group) until the GPU is full; all blocks are resident: they meet at grid barriers
-    const uint64_t units = dense ? G : count;
+    const uint64_t units = dense ? G : (count_dev ? n : count);      // (a list made on the device: its length is not known here)
     const uint64_t per_warp = dense ? 1ull : 32ull;
     uint64_t grid = (units + per_warp * kKvWarps - 1) / (per_warp * kKvWarps);
     const uint64_t cap = (uint64_t)g_state.sm_count * (uint64_t)(g_state.kv_blocks_per_sm > 2 ? 2 : g_state.kv_blocks_per_sm);
@@ -408,11 +410,37 @@ int compress_launches(const float* const* grads, uint64_t n, const fastsgd_param
         // Any other group size: the sum kernel, then the list encoder over the dense gradient (the fused kernel's
         // tile is the group of 2^14).  Two launches per gradient, the gradient read three times.
         if (params->group_log2 < 8u) return FASTSGD_E_NOT_IMPLEMENTED;
+        // sum kernel; the kept entries selected into a list in the workspace (the fused kernel's scratch for dense tiles,
+        // 4.5 M pairs); the list encoder on that list -- or, should the list not fit, over the dense gradient itself
+        // (a warp per group: slow for large groups).  Which of the two runs is decided on the device.
+        unsigned char* wsb = static_cast<unsigned char*>(g_state.ws);
+        double* S = reinterpret_cast<double*>(wsb + kJobSumOffset);
+        unsigned long long* count_dev = reinterpret_cast<unsigned long long*>(wsb + kKvAggOffset + kKvAggBytes - 8);
+        unsigned char* list = wsb + ws_dense_offset(n, params->group_log2);
+        const uint64_t capacity = ((uint64_t)kMaxCtas * kDenseScratchBytes) / 8ull;
         for (uint32_t i = 0; i < num_grads; ++i) {
-            double* S = reinterpret_cast<double*>(static_cast<unsigned char*>(g_state.ws) + kJobSumOffset);
             rc = launch_sum(grads[i], n, 0u, params->tau, pw, view(g_state.ws, n, params->group_log2), S, st);
             if (rc) return rc;
-            rc = launch_list_encoder(true, nullptr, grads[i], n, n, params, pw, outs[i], out_bytes, st);
+            SelArgs sa;
+            std::memset(&sa, 0, sizeof(sa));
+            sa.grad = grads[i]; sa.n = n; sa.ctl = reinterpret_cast<Control*>(wsb);
+            sa.blk_agg = reinterpret_cast<unsigned long long*>(wsb + kKvAggOffset);
+            sa.keys = reinterpret_cast<uint32_t*>(list); sa.vals = reinterpret_cast<float*>(list + 4ull * capacity);
+            sa.count_out = count_dev; sa.capacity = capacity; sa.tau = params->tau; sa.wait_limit = g_tun.wait_limit;
+            uint64_t sgrid = (uint64_t)g_state.sm_count * 2ull;
+            const uint64_t steps = (n + 127ull) >> 7;
+            if (sgrid > (steps + kKvWarps - 1) / kKvWarps) sgrid = (steps + kKvWarps - 1) / kKvWarps;
+            if (sgrid > 511) sgrid = 511;                      // (one thread per block adds up the totals; the last slot holds the count)
+            PowTable pwc = pw;
+            void* kargs[] = {&sa, &pwc};
+            if (cudaLaunchCooperativeKernel((const void*)k_select_pairs, dim3((unsigned)sgrid), dim3(kKvThreads), kargs, 0, st) != cudaSuccess) {
+                cudaGetLastError();
+                return FASTSGD_E_CUDA;
+            }
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            rc = launch_list_encoder(false, sa.keys, sa.vals, 0, n, params, pw, outs[i], out_bytes, st, count_dev, 1u, true);
+            if (rc) return rc;
+            rc = launch_list_encoder(true, nullptr, grads[i], n, n, params, pw, outs[i], out_bytes, st, count_dev, 2u, true);
             if (rc) return rc;
         }
         return FASTSGD_OK;

@@ -58,7 +58,12 @@ struct KvArgs {
     uint32_t            slice;       // list entries per warp, a multiple of 32
     uint32_t            wait_limit;
     uint32_t            given_sum;   // 1: S is already in the workspace (the list holds kept candidates of a dense gradient); pass 1 is skipped
+    // the list was made on the device by k_select_pairs: its length is read from there (kListOverflow: it did not fit)
+    const unsigned long long* count_dev;
+    uint32_t            run_if;      // 0: always; 1: only if the list fits; 2: only if it does not (the dense walk takes over)
+    uint32_t            pad;
 };
+constexpr unsigned long long kListOverflow = ~0ull;
 
 struct KvWarp {
     float    unit[kKvUnit];          // leaves of the unit being formed; all zero between units
@@ -133,12 +138,38 @@ __device__ __forceinline__ uint32_t kv_flag_of_bl(uint32_t bl, uint32_t l, uint3
 // of them are kept, and each kept entry's delta key (Eq. 4; the first of a group counts from g * T).  `prev` is the
 // last kept key before the batch and is advanced.
 struct KvBatch { uint32_t key; float val; uint32_t vm, km, delta; bool kept; };
+
+// The walk's loads run ahead of their use: the entries of the next kAhead batches are on their way while a batch is
+// worked on (a warp walks a group alone, 32 entries per step, and every step would otherwise wait for its own load).
+constexpr int kAhead = 4;
 template <bool DENSE>
-__device__ __forceinline__ KvBatch kv_batch(const KvArgs& a, uint64_t base, uint32_t g, float thr_e, uint32_t& prev, int lane) {
+struct KvFeed {
+    uint32_t k[kAhead];
+    float    v[kAhead];
+    uint64_t next;
+    __device__ __forceinline__ void load(const KvArgs& a, int slot, uint64_t e) {
+        k[slot] = 0u; v[slot] = 0.f;
+        if (e < a.count) { k[slot] = DENSE ? (uint32_t)e : __ldg(a.keys + e); v[slot] = __ldg(a.vals + e); }
+    }
+    __device__ __forceinline__ void start(const KvArgs& a, uint64_t base, int lane) {
+#pragma unroll
+        for (int i = 0; i < kAhead; ++i) load(a, i, base + 32u * (uint32_t)i + (uint64_t)lane);
+        next = base + 32u * (uint32_t)kAhead;
+    }
+    __device__ __forceinline__ void pop(const KvArgs& a, int lane, uint32_t& key, float& val) {
+        key = k[0]; val = v[0];
+#pragma unroll
+        for (int i = 0; i + 1 < kAhead; ++i) { k[i] = k[i + 1]; v[i] = v[i + 1]; }
+        load(a, kAhead - 1, next + (uint64_t)lane);
+        next += 32u;
+    }
+};
+
+template <bool DENSE>
+__device__ __forceinline__ KvBatch kv_batch(const KvArgs& a, KvFeed<DENSE>& feed, uint64_t base, uint32_t g, float thr_e, uint32_t& prev, int lane) {
     KvBatch b;
     const uint64_t e = base + (uint64_t)lane;
-    b.key = 0u; b.val = 0.f;
-    if (e < a.count) { b.key = DENSE ? (uint32_t)e : __ldg(a.keys + e); b.val = __ldg(a.vals + e); }
+    feed.pop(a, lane, b.key, b.val);
     const bool valid = e < a.count && (b.key >> a.group_log2) == g;
     b.vm = __ballot_sync(kFullMask, valid);
     b.kept = valid && fabsf(b.val) >= thr_e;              // (thr_e is at least the smallest denormal: zeros are never kept; +inf when nothing may be kept)
@@ -158,8 +189,10 @@ __device__ __forceinline__ unsigned long long kv_group_sizes(KvWarp& ws, const K
     if (lane < 8) ws.hist[32 + lane] = 0u;
     __syncwarp();
     uint32_t prev = g << a.group_log2, count = 0u, maxd = 0u;
+    KvFeed<DENSE> feed;
+    feed.start(a, head, lane);
     for (uint64_t base = head;; base += 32u) {
-        const KvBatch b = kv_batch<DENSE>(a, base, g, thr_e, prev, lane);
+        const KvBatch b = kv_batch<DENSE>(a, feed, base, g, thr_e, prev, lane);
         if (b.kept) {
             atomicAdd(&ws.hist[b.delta ? 32 - __clz((int)b.delta) : 0], 1u);
             maxd = max(maxd, b.delta);
@@ -195,8 +228,10 @@ __device__ __forceinline__ void kv_group_pack(KvWarp& ws, const KvArgs& a, const
     const uint32_t inv_m = c_inv_m[M], round_up = (1u << a.l) - 1u;
     const uint32_t flag_pos0 = 8u * count;
     uint32_t prev = g << a.group_log2, rank = 0u, dpos = flag_pos0 + a.l * count;
+    KvFeed<DENSE> feed;
+    feed.start(a, head, lane);
     for (uint64_t base = head;; base += 32u) {
-        const KvBatch b = kv_batch<DENSE>(a, base, g, thr_e, prev, lane);
+        const KvBatch b = kv_batch<DENSE>(a, feed, base, g, thr_e, prev, lane);
         uint32_t f = 0u, w = 0u;
         if (b.kept) {
             f = min(flag_of(b.delta, a.l, inv_m), round_up);
@@ -309,7 +344,17 @@ __device__ __forceinline__ void kv_for_each_head(const KvArgs& a, uint64_t lo, u
 // in the workspace (group sizes other than the fused encoder's): every index is a list entry, a warp owns a run of groups.
 template <bool DENSE>
 __global__ void __launch_bounds__(kKvThreads, 2)
-k_compress_kv(const KvArgs a, const __grid_constant__ PowTable pw) {
+k_compress_kv(const KvArgs a_in, const __grid_constant__ PowTable pw) {
+    KvArgs a = a_in;
+    if (a.count_dev != nullptr) {
+        const unsigned long long cnt = __ldcg(a.count_dev);
+        if ((a.run_if == 1u && cnt == kListOverflow) || (a.run_if == 2u && cnt != kListOverflow)) return;      // (the same answer in every block)
+        if (!DENSE) {
+            a.count = cnt;
+            const uint64_t warps = (uint64_t)gridDim.x * kKvWarps;
+            a.slice = (uint32_t)max((((cnt + warps - 1) / warps) + 31ull) & ~31ull, 32ull);
+        }
+    }
     extern __shared__ __align__(128) unsigned char kv_smem_raw[];
     KvSmem& s = *reinterpret_cast<KvSmem*>(kv_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -462,6 +507,113 @@ k_compress_kv(const KvArgs a, const __grid_constant__ PowTable pw) {
         const unsigned int old = atom_add_acq_rel_u32(&a.ctl->exit_count, 1u);
         if (old == gridDim.x - 1u) {
             if (ld_acquire_u32(&a.ctl->error) != 0u) kv_write_header(a, kStTimeout, 0ull, 0ull, 0.0);
+            a.ctl->exit_count = 0u;
+            st_release_u32(&a.ctl->bar_gen, gen_next);
+        }
+    }
+}
+
+
+// Dense gradient -> the list of its kept entries (i, v_i), |v_i| >= B_tau, in index order, for the list encoder:
+// the general path of fastsgd_compress for group sizes other than the fused kernel's.  One cooperative launch: every
+// warp counts the kept entries of its contiguous share of the gradient, the blocks' totals meet at a grid barrier,
+// every warp then writes its entries behind those of the warps before it.  S is in the workspace (k_abs_sum).  If
+// the list does not fit `capacity` pairs, *count_out = kListOverflow and nothing is written.
+struct SelArgs {
+    const float*        grad;
+    uint64_t            n;
+    Control*            ctl;
+    unsigned long long* blk_agg;     // [gridDim.x]
+    uint32_t*           keys;        // [capacity]
+    float*              vals;        // [capacity]
+    unsigned long long* count_out;
+    uint64_t            capacity;
+    uint32_t            tau;
+    uint32_t            wait_limit;
+};
+
+__global__ void __launch_bounds__(kKvThreads, 2)
+k_select_pairs(const SelArgs a, const __grid_constant__ PowTable pw) {
+    __shared__ uint32_t s_w[kKvWarps];
+    __shared__ unsigned long long s_scan[kKvWarps], s_scanb[kKvWarps];
+    __shared__ uint32_t s_flag, s_abort;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned int gen_next = 0u;
+    if (tid == 0) { s_flag = ld_acquire_u32(&a.ctl->bar_gen) + 1u; s_abort = 0u; }
+    __syncthreads();
+    gen_next = s_flag;
+    const double S = __ldcg(reinterpret_cast<const double*>(reinterpret_cast<const unsigned char*>(a.ctl) + kJobSumOffset));
+    const float thr_e = (isfinite(S) && S != 0.0) ? fmaxf(__double2float_ru(__ddiv_rn(S, pw.P[a.tau])), __int_as_float(1)) : __int_as_float(0x7f800000);
+    // this warp's share: whole steps of 128 entries (a float4 per lane)
+    const uint64_t steps = (a.n + 127ull) >> 7;
+    const uint64_t warps = (uint64_t)gridDim.x * kKvWarps, gw = (uint64_t)blockIdx.x * kKvWarps + (uint64_t)warp;
+    const uint64_t per = (steps + warps - 1) / warps;
+    const uint64_t s0 = min(steps, gw * per), s1 = min(steps, s0 + per);
+    auto mask_of = [&](uint64_t step) -> uint32_t {
+        const float4 q = load4_guarded(a.grad, (step << 7) + 4ull * (uint64_t)lane, a.n);
+        return (fabsf(q.x) >= thr_e ? 1u : 0u) | (fabsf(q.y) >= thr_e ? 2u : 0u) | (fabsf(q.z) >= thr_e ? 4u : 0u) | (fabsf(q.w) >= thr_e ? 8u : 0u);
+    };
+    uint32_t mine = 0u;
+    for (uint64_t st = s0; st < s1; ++st) mine += (uint32_t)__popc(mask_of(st));
+    mine = __reduce_add_sync(kFullMask, mine);
+    if (lane == 0) s_w[warp] = mine;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long tot = 0ull;
+        for (int w = 0; w < kKvWarps; ++w) tot += s_w[w];
+        st_relaxed_u64(a.blk_agg + blockIdx.x, tot);
+        // grid barrier (the launch's only one): the last block to arrive opens it
+        if (atom_add_acq_rel_u32(&a.ctl->bar_count[0], 1u) == gridDim.x - 1u) {
+            a.ctl->bar_count[0] = 0u;
+            st_release_u32(&a.ctl->bar_flag[0], gen_next);
+        }
+        uint32_t spin = 0;
+        while (ld_acquire_u32(&a.ctl->bar_flag[0]) != gen_next) {
+            if (++spin > a.wait_limit) { s_abort = 1u; break; }
+            if (spin > 64u) __nanosleep(32);
+        }
+    }
+    __syncthreads();
+    if (!s_abort) {
+        unsigned long long all = (uint32_t)tid < gridDim.x ? ld_relaxed_u64(a.blk_agg + tid) : 0ull;
+        unsigned long long before = (uint32_t)tid < blockIdx.x ? all : 0ull;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            all += __shfl_xor_sync(kFullMask, all, o);
+            before += __shfl_xor_sync(kFullMask, before, o);
+        }
+        if (lane == 0) { s_scan[warp] = all; s_scanb[warp] = before; }
+        __syncthreads();
+        unsigned long long total = 0ull, base = 0ull;
+#pragma unroll
+        for (int w = 0; w < kKvWarps; ++w) { total += s_scan[w]; base += s_scanb[w]; }
+        for (int w = 0; w < warp; ++w) base += s_w[w];
+        const bool fits = total <= a.capacity;
+        if (blockIdx.x == 0 && tid == 0) *a.count_out = fits ? total : kListOverflow;
+        if (fits) {
+            unsigned long long pos = base;
+            for (uint64_t st = s0; st < s1; ++st) {
+                const uint64_t e0 = (st << 7) + 4ull * (uint64_t)lane;
+                const float4 q = load4_guarded(a.grad, e0, a.n);
+                const uint32_t m = (fabsf(q.x) >= thr_e ? 1u : 0u) | (fabsf(q.y) >= thr_e ? 2u : 0u) | (fabsf(q.z) >= thr_e ? 4u : 0u) | (fabsf(q.w) >= thr_e ? 8u : 0u);
+                const uint32_t c = (uint32_t)__popc(m);
+                const uint32_t incl = warp_incl_scan(c, lane);
+                unsigned long long p = pos + (incl - c);
+                if (m & 1u) { a.keys[p] = (uint32_t)e0;      a.vals[p] = q.x; ++p; }
+                if (m & 2u) { a.keys[p] = (uint32_t)e0 + 1u; a.vals[p] = q.y; ++p; }
+                if (m & 4u) { a.keys[p] = (uint32_t)e0 + 2u; a.vals[p] = q.z; ++p; }
+                if (m & 8u) { a.keys[p] = (uint32_t)e0 + 3u; a.vals[p] = q.w; ++p; }
+                pos += __shfl_sync(kFullMask, incl, 31);
+            }
+        }
+    } else if (blockIdx.x == 0 && tid == 0) {
+        *a.count_out = kListOverflow;                     // (a wait ran out: the dense walk takes over; the next launch's waits report it)
+    }
+    // the last block to leave bumps the generation
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int old = atom_add_acq_rel_u32(&a.ctl->exit_count, 1u);
+        if (old == gridDim.x - 1u) {
             a.ctl->exit_count = 0u;
             st_release_u32(&a.ctl->bar_gen, gen_next);
         }

@@ -816,6 +816,20 @@ def test_other_group_sizes_dense_input_and_decoder(glog, keep_div):
         assert np.allclose(gdense, odense, rtol=RTOL, atol=ATOL) and np.array_equal(gdense, odense)
 
 
+def test_other_group_sizes_when_the_kept_list_does_not_fit():
+    # general path: more kept entries than the workspace's list holds (4.5 M pairs): the dense walk takes over, same stream
+    import gpu_util as G
+    n = 6_300_001
+    v = workloads.normal(n, seed=8)
+    b = workloads.base_for_keep(v, int(0.8 * n))
+    pg, po = binding.params(b, 128, 2, 12), oracle.params(b, 128, 2, 12)
+    orc, ostream = oracle.compress(v, po)
+    assert orc == 0 and int(np.frombuffer(ostream[24:32].tobytes(), np.uint64)[0]) > 4_700_000
+    rc, status, gstream, intact = G.gpu_compress(v, pg, fill=0x31)
+    assert rc == 0 and intact and status == 0
+    assert gstream.size == ostream.size and np.array_equal(gstream, ostream)
+
+
 def test_key_value_input_status_words_and_hostile_keys():
     import torch
     import gpu_util as G
