@@ -821,8 +821,8 @@ def main():
                        "sector_bytes": float(sum(stream_bytes)) + 64.0 * float(sum(kept)),
                        "sector_gbs": (float(sum(stream_bytes)) + 64.0 * float(sum(kept))) / (ms_dec * 1e-3) / 1e9},
         "dense_zero_fill_ms": ms_zero,
-        "sparse_adam_update": {"ms": ms_adam, "touched_bytes": float(sum(stream_bytes)) * 2.0 + 40.0 * float(sum(kept)),
-                               "note": "decode + Adam step on decoded coordinates only; two launches per 8 streams; "
+        "sparse_adam_update": {"ms": ms_adam, "touched_bytes": float(sum(stream_bytes)) + 40.0 * float(sum(kept)),
+                               "note": "decode + Adam step on decoded coordinates only; one launch (up to 8 streams); "
                                        "256 MiB written before every call; not part of value / ms_per_step"},
         "compress_kv": kv_info,
         "stream": {"bytes_per_worker": float(sum(stream_bytes)) / W, "kept_per_worker": float(sum(kept)) / W,

@@ -215,7 +215,8 @@ typedef struct fastsgd_adam {
  *   hyper        host pointer
  *   grad_scratch device, n floats, ALL ZERO on entry and all zero again when
  *                the call has run: the aggregated gradient g lives here between
- *                the two passes (the caller clears it once, when it allocates it)
+ *                aggregation and update (the caller clears it once, when it
+ *                allocates it)
  *   theta, m, v  device, n floats each, updated in place where g != 0:
  *                  m = beta1 * m + (1 - beta1) * g
  *                  v = beta2 * v + (1 - beta2) * g * g
@@ -223,8 +224,10 @@ typedef struct fastsgd_adam {
  *                every operation one IEEE fp32 operation (round to nearest, no
  *                fused multiply-add), in the order written
  * g is the sum of the decoded streams in the given order, exactly as
- * fastsgd_decompress_accumulate_batch forms it.  Two launches per 8 streams:
- * aggregation, then the update.  Errors and damaged streams as for
+ * fastsgd_decompress_accumulate_batch forms it.  Up to 8 streams: one launch
+ * (the warp or block that decodes a group aggregates it and then updates its
+ * coordinates); more: two launches per 8 streams, aggregation of all of them,
+ * then the update.  Errors and damaged streams as for
  * fastsgd_decompress_accumulate_batch (theta, m, v and grad_scratch are then
  * unspecified, never accessed out of bounds).
  */

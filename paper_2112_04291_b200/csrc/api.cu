@@ -171,14 +171,20 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_decode_accumulate<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
         return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
     {   // every instantiation must be resident with the grid the launch uses (the queue of large groups relies on it)
-        int b2x[4] = {0, 0, 0, 0};
+        int b2x[6] = {0, 0, 0, 0, 0, 0};
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[0], k_decode_accumulate<false>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[1], k_decode_accumulate<true>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[2], k_decode_accumulate<false, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[3], k_decode_accumulate<true, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[4], k_decode_accumulate<false, 2>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[5], k_decode_accumulate<true, 2>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         b2 = b2x[0];
-        for (int i = 1; i < 4; ++i) if (b2x[i] < b2) b2 = b2x[i];
+        for (int i = 1; i < 6; ++i) if (b2x[i] < b2) b2 = b2x[i];
     }
     g_state.sm_count = sms;
     g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
@@ -531,10 +537,12 @@ int fastsgd_compress(const float* grad, uint64_t n, const fastsgd_params* params
 
 namespace {
 // The decoder's launches over a list of streams, 8 per launch.  adam == nullptr: aggregation into
-// dense_out; else the model-update pass (dense_out holds the aggregated gradient).
+// dense_out; else the model-update pass (dense_out holds the aggregated gradient), or, `fused` (one
+// launch's worth of streams, dense_out all zero), aggregation and update in the same launch.
 int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32_t num_streams, uint64_t n,
                     const fastsgd_params* params, float* dense_out, const fastsgd_adam* adam,
-                    float* theta, float* m, float* v, void* stream) {
+                    float* theta, float* m, float* v, void* stream, bool fused = false) {
+    if (fused && (!adam || num_streams > (uint32_t)kDecMaxStreams)) return FASTSGD_E_BAD_PARAM;
     if (!streams_in || !bytes || !dense_out || !params) return FASTSGD_E_NULL;
     if (!aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
     PowTable pw;
@@ -589,7 +597,10 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
         }
         {
             LaunchTimer lt(2, st);
-            if (adam) {
+            if (fused) {
+                if (da.W == 1u) k_decode_accumulate<true, 2><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+                else k_decode_accumulate<false, 2><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            } else if (adam) {
                 if (da.W == 1u) k_decode_accumulate<true, 1><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
                 else k_decode_accumulate<false, 1><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
             } else {
@@ -616,7 +627,10 @@ int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64
                                      float* theta, float* m, float* v, void* stream) {
     if (!hyper || !grad_scratch || !theta || !m || !v) return FASTSGD_E_NULL;
     if (!aligned(theta, 4) || !aligned(m, 4) || !aligned(v, 4)) return FASTSGD_E_ALIGN;
-    // pass 1: the aggregated gradient; pass 2: the same streams again, every key's coordinate updated once
+    // up to 8 streams: one launch, each group aggregated and its coordinates updated by the warp or block that decodes it
+    if (num_streams <= (uint32_t)kDecMaxStreams)
+        return decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, hyper, theta, m, v, stream, true);
+    // more: pass 1, the aggregated gradient; pass 2, the same streams again, every key's coordinate updated once
     int rc = decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, nullptr, nullptr, nullptr, nullptr, stream);
     if (rc) return rc;
     return decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, hyper, theta, m, v, stream);

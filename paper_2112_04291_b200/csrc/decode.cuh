@@ -538,15 +538,48 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
         if (BLOCK && tile != nullptr) {
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo[w]] : 0.f;
-            apply_run<MODE, KMAX>(a, kk, dd, vv, res);
+            apply_run<(MODE == 2 ? 0 : MODE), KMAX>(a, kk, dd, vv, res);
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = res[k];
         } else {
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
-            apply_run<MODE, KMAX>(a, kk, dd, vv, res);
+            apply_run<(MODE == 2 ? 0 : MODE), KMAX>(a, kk, dd, vv, res);
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
+        }
+    }
+
+    // MODE 2 (the caller has given every stream of the group in this one call; dense_out in global memory):
+    // the model update from the same keys, still in registers.  Every key's aggregated g is taken out of
+    // dense_out by an atomic exchange with 0: of the streams that hold a key the one that gets there first
+    // receives g and updates the coordinate, the others receive 0 (whichever it is, the result is the same);
+    // no stream waits for another, and all the exchanges are in flight together.
+    if constexpr (MODE == 2) {
+        static_assert(!BLOCK, "the block path updates from its slice in shared memory");
+        if (first) return;                                     // (uniform) nothing was applied
+        __syncwarp();
+        constexpr int KA = NS * KMAX;
+        uint32_t ka[KA]; float ga[KA];
+#pragma unroll
+        for (int w = 0; w < NS; ++w) {
+            uint32_t key = key0[w];
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) {
+                const bool on = live[w] && jb[w] + k < je[w];
+                key += dv[w][k];
+                ka[w * KMAX + k] = on ? key : 0xFFFFFFFFu;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < KA; ++i) ga[i] = ka[i] != 0xFFFFFFFFu ? atomicExch(a.dense + ka[i], 0.0f) : 0.0f;
+        constexpr int KB = KA < 8 ? KA : 8;                    // moments and parameters of eight keys loaded at a time
+#pragma unroll
+        for (int i0 = 0; i0 < KA; i0 += KB) {
+            uint32_t kb[KB]; float gb[KB], vb[KB], rb[KB];
+#pragma unroll
+            for (int i = 0; i < KB; ++i) { kb[i] = ka[i0 + i]; gb[i] = ga[i0 + i]; vb[i] = 0.0f; }
+            apply_run<1, KB>(a, kb, gb, vb, rb);
         }
     }
 }
@@ -567,6 +600,64 @@ __device__ __forceinline__ void stage_blob(uint32_t* dst, const uint32_t* src, u
         }
     }
 }
+
+// The warp path's decode of one small group whose blobs are staged (lane w holds stream w's directory
+// fields): up to four streams at a time, parsed side by side and applied in stream order.  DM: what
+// decode_multi does with the values (0, 1, or 2 = both when W <= 4 puts every stream in the one call).
+// Used by the kernel's mode 2 only: modes 0 and 1 keep the same loop in the kernel's body, where the
+// compiler's code for it measured 15 % faster on four sparse streams than through this function.
+template <int DM>
+__device__ __forceinline__ void warp_fours(const DecArgs& a, DecShared& s, const uint32_t* stage, uint32_t count, uint32_t M,
+                                           uint32_t base, uint32_t nwords, uint32_t W, uint32_t g, int lane, int warp) {
+    for (uint32_t w0 = 0; w0 < W; w0 += 4u) {
+        const uint32_t ns = W - w0 < 4u ? W - w0 : 4u;
+        const uint32_t* bl[4]; uint32_t nwv[4], cv[4], mv[4]; const float* vl[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t src = (uint32_t)i < ns ? w0 + i : w0;
+            const uint32_t c = __shfl_sync(kFullMask, count, src), b = __shfl_sync(kFullMask, base, src);
+            nwv[i] = __shfl_sync(kFullMask, nwords, src); mv[i] = __shfl_sync(kFullMask, M, src);
+            cv[i] = (uint32_t)i < ns ? c : 0u;
+            bl[i] = stage + b; vl[i] = s.val[src];
+        }
+        if (ns == 1u) {
+            const uint32_t* b1[1] = {bl[0]}; const uint32_t n1[1] = {nwv[0]}, c1[1] = {cv[0]}, m1[1] = {mv[0]}; const float* v1[1] = {vl[0]};
+            decode_multi<DM, false, 1, 4>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+        } else if (ns == 2u) {
+            const uint32_t* b2[2] = {bl[0], bl[1]}; const uint32_t n2[2] = {nwv[0], nwv[1]}, c2[2] = {cv[0], cv[1]}, m2[2] = {mv[0], mv[1]};
+            const float* v2[2] = {vl[0], vl[1]};
+            decode_multi<DM, false, 2, 4>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+        } else {
+            decode_multi<DM, false, 4, 4>(a, s, bl, nwv, cv, mv, vl, g, nullptr, lane, 32, lane, warp);
+        }
+        __syncwarp();          // these streams' stores before the next streams' loads of the same keys
+    }
+}
+
+// A decode_multi call of the kernel below.  MODE 2 (aggregation and model update in one launch): `fused`
+// when this call holds every stream of the group (both sweeps inside the call), else the caller's pass
+// (0: aggregation over all the group's calls, then 1: the update over all of them again).
+#define FSG_DECODE_MULTI(fused, B_, NS_, K_, TG_, ...)                                        \
+    do {                                                                                      \
+        if constexpr (MODE == 2) {                                                            \
+            if (fused) decode_multi<2, B_, NS_, K_, TG_>(__VA_ARGS__);                        \
+            else if (pass == 0) decode_multi<0, B_, NS_, K_, TG_>(__VA_ARGS__);               \
+            else decode_multi<1, B_, NS_, K_, TG_>(__VA_ARGS__);                              \
+        } else {                                                                              \
+            decode_multi<MODE, B_, NS_, K_, TG_>(__VA_ARGS__);                                \
+        }                                                                                     \
+    } while (0)
+
+// (the same without the fused form: the block path, whose mode 2 keeps the slice of g in shared memory)
+#define FSG_DECODE_MULTI_PASS(B_, NS_, K_, TG_, ...)                                          \
+    do {                                                                                      \
+        if constexpr (MODE == 2) {                                                            \
+            if (pass == 0) decode_multi<0, B_, NS_, K_, TG_>(__VA_ARGS__);                    \
+            else decode_multi<1, B_, NS_, K_, TG_>(__VA_ARGS__);                              \
+        } else {                                                                              \
+            decode_multi<MODE, B_, NS_, K_, TG_>(__VA_ARGS__);                                \
+        }                                                                                     \
+    } while (0)
 
 // ONE_STREAM: the launch holds a single stream (its own instantiation, so that the code of the
 // many-stream paths and of the two-groups-per-warp path do not weigh on each other)
@@ -673,6 +764,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 }
             }
             __syncwarp();
+            // (one stream: a call always holds the whole group, so that mode 2 is decode_multi's own)
             if (c2[0] <= kDecWarpSide && c2[1] <= kDecWarpSide)
                 decode_multi<MODE, false, 2, 4, true>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp, g + stride);
             else
@@ -715,6 +807,9 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         __syncwarp();
         if (__any_sync(kFullMask, count > kDecWarpSide)) {
             // longer runs per lane: two streams at a time
+            const bool fused = MODE == 2 && W <= 2u;
+            const int npass = (MODE == 2 && !fused) ? 2 : 1;
+            for (int pass = 0; pass < npass; ++pass)
             for (uint32_t w0 = 0; w0 < W; w0 += 2u) {
                 const uint32_t w1 = w0 + 1u < W ? w0 + 1u : w0;
                 const uint32_t* b2[2]; uint32_t n2[2], c2[2], m2[2]; const float* v2[2];
@@ -724,14 +819,21 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 m2[0] = __shfl_sync(kFullMask, M, w0); m2[1] = __shfl_sync(kFullMask, M, w1);
                 v2[0] = s.val[w0]; v2[1] = s.val[w1];
                 if (w0 + 1u < W) {
-                    decode_multi<MODE, false, 2, 8>(a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
+                    FSG_DECODE_MULTI(fused, false, 2, 8, false, a, s, b2, n2, c2, m2, v2, g, nullptr, lane, 32, lane, warp);
                 } else {
                     const uint32_t* b1[1] = {b2[0]}; const uint32_t n1[1] = {n2[0]}, c1[1] = {c2[0]}, m1[1] = {m2[0]}; const float* v1[1] = {v2[0]};
-                    decode_multi<MODE, false, 1, 8>(a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
+                    FSG_DECODE_MULTI(fused, false, 1, 8, false, a, s, b1, n1, c1, m1, v1, g, nullptr, lane, 32, lane, warp);
                 }
                 __syncwarp();      // these streams' stores before the next streams' loads of the same keys
             }
-        } else
+        } else {
+            if constexpr (MODE == 2) {
+                if (W <= 4u) warp_fours<2>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+                else {      // the update only after every stream's values are in
+                    warp_fours<0>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+                    warp_fours<1>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+                }
+            } else {
         // up to four streams at a time, parsed side by side and applied in stream order
         for (uint32_t w0 = 0; w0 < W; w0 += 4u) {
             const uint32_t ns = W - w0 < 4u ? W - w0 : 4u;
@@ -755,6 +857,8 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 decode_multi<MODE, false, 4, 4>(a, s, bl, nwv, cv, mv, vl, g, nullptr, lane, 32, lane, warp);
             }
             __syncwarp();          // these streams' stores before the next streams' loads of the same keys
+        }
+            }
         }
     }
     __syncthreads();
@@ -806,11 +910,16 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         // The group's slice of dense_out is brought into shared memory by one bulk copy, updated there by
         // every stream in turn, and written back by one bulk copy (needs 16-byte alignment and size).
         const bool use_tile = a.group_log2 <= 14u && ((reinterpret_cast<uintptr_t>(a.dense) & 15u) == 0u) && ((span & 3u) == 0u);
-        if (use_tile && tid == 0) {
+        // (MODE 2: dense_out is all zero by contract and is left so: the slice starts as zeros in shared memory and never leaves it)
+        const bool load_tile = use_tile && MODE != 2;
+        if (load_tile && tid == 0) {
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the last write-back has read the tile
             mbar_expect_tx(&s.tile_bar, span * 4u);
             bulk_load(s.u.tile, a.dense + lo, span * 4u, &s.tile_bar);
         }
+        if (MODE == 2 && use_tile)
+            for (uint32_t i = tid; i < (span >> 2); i += kDecThreads)
+                reinterpret_cast<float4*>(s.u.tile)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (!local && tid < (int)W) {
             uint32_t count = 0, M = 0, off = 0, nwords = 0;
             if (s.ok[tid])
@@ -822,10 +931,11 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         // parsed again -- the coordinates to update are the non-zeros of the slice.  Thread t looks at entries
         // t, t + 256, ..., eight at a time, so that the loads of their moments and parameters are in flight together
         // (neighbouring threads, neighbouring addresses).
-        const bool scan_tile = MODE == 1 && use_tile;
+        const bool scan_tile = MODE != 0 && use_tile;
+        const bool parse = !(MODE == 1 && use_tile);
         // staging offsets; a blob that does not fit is parsed from global memory
         uint32_t used = 0;
-        if (!scan_tile)
+        if (parse)
         for (uint32_t w = 0; w < W; ++w) {
             const uint32_t nw = s.g_count[w] ? s.g_nwords[w] : 0u;
             const bool fits = used + nw <= kBlockStageWords;
@@ -837,7 +947,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             }
         }
         __syncthreads();
-        if (use_tile) {
+        if (load_tile) {
             if (tid == 0) s.big[1] = mbar_wait(&s.tile_bar, tile_parity, a.try_limit) ? 1u : 0u;     // bounded wait, one thread
             __syncthreads();
             tile_parity ^= 1u;
@@ -847,23 +957,10 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 continue;
             }
         }
-        if (scan_tile) {
-            for (uint32_t i0 = 0; i0 < span; i0 += 8u * (uint32_t)kDecThreads) {
-                uint32_t kk[8]; float cur[8], vv[8], res[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t idx = i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid;
-                    cur[u] = idx < span ? s.u.tile[idx] : 0.0f;
-                    kk[u] = cur[u] != 0.0f ? lo + idx : 0xFFFFFFFFu;
-                    vv[u] = 0.0f;
-                }
-                apply_run<MODE, 8>(a, kk, cur, vv, res);
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (kk[u] != 0xFFFFFFFFu) s.u.tile[i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid] = res[u];
-            }
-            __syncthreads();
-        } else
+        // MODE 2 without the slice in shared memory: every stream aggregated into dense_out, then every stream again for the update
+        const int npass = (MODE == 2 && !use_tile) ? 2 : 1;
+        if (parse)
+        for (int pass = 0; pass < npass; ++pass)
         for (uint32_t w = 0; w < W; ++w) {
             const uint32_t c = s.g_count[w];
             const uint32_t* blob = s.g_valid[w] ? s.bstage + s.g_base[w]
@@ -876,21 +973,45 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 const uint32_t* b2[2] = {blob, blob2}; const uint32_t n2[2] = {s.g_nwords[w], s.g_nwords[w2]};
                 const uint32_t c2[2] = {c, s.g_count[w2]}, m2[2] = {s.g_M[w], s.g_M[w2]};
                 const float* v2[2] = {s.val[w], s.val[w2]};
-                decode_multi<MODE, true, 2, 4>(a, s, b2, n2, c2, m2, v2, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+                FSG_DECODE_MULTI_PASS(true, 2, 4, false, a, s, b2, n2, c2, m2, v2, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
                 ++w;
             } else if (c == 0u) {
                 continue;
             } else if (c <= 4u * (uint32_t)kDecThreads) {
                 const uint32_t* b1[1] = {blob}; const uint32_t n1[1] = {s.g_nwords[w]}, c1[1] = {c}, m1[1] = {s.g_M[w]};
                 const float* v1[1] = {s.val[w]};
-                decode_multi<MODE, true, 1, 4>(a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
+                FSG_DECODE_MULTI_PASS(true, 1, 4, false, a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
             } else {
-                decode_long<MODE>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
-                                  tid, kDecThreads, lane, warp);
+                if constexpr (MODE == 2) {
+                    if (pass == 0) decode_long<0>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                                                  tid, kDecThreads, lane, warp);
+                    else decode_long<1>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                                        tid, kDecThreads, lane, warp);
+                } else {
+                    decode_long<MODE>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
+                                      tid, kDecThreads, lane, warp);
+                }
             }
             __syncthreads();       // these streams' updates before the next stream's
         }
-        if (use_tile && tid == 0) {
+        if (scan_tile) {
+            for (uint32_t i0 = 0; i0 < span; i0 += 8u * (uint32_t)kDecThreads) {
+                uint32_t kk[8]; float cur[8], vv[8], res[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t idx = i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid;
+                    cur[u] = idx < span ? s.u.tile[idx] : 0.0f;
+                    kk[u] = cur[u] != 0.0f ? lo + idx : 0xFFFFFFFFu;
+                    vv[u] = 0.0f;
+                }
+                apply_run<1, 8>(a, kk, cur, vv, res);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (kk[u] != 0xFFFFFFFFu) s.u.tile[i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid] = res[u];
+            }
+            __syncthreads();
+        }
+        if (load_tile && tid == 0) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // the updates above, before the copy reads them
             asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                          ::"l"(__cvta_generic_to_global(a.dense + lo)), "r"(smem_u32(s.u.tile)), "r"(span * 4u) : "memory");

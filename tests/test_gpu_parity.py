@@ -563,7 +563,7 @@ def test_tiles_below_the_threshold_are_never_read_again(tiles, workers):
                 assert 0 < d < n // 10
 
 
-@pytest.mark.parametrize("workers", [1, 3, 8, 10])
+@pytest.mark.parametrize("workers", [1, 2, 3, 5, 8, 10])
 def test_sparse_adam_update_equals_the_oracles(workers):
     # the workers' streams decoded and one Adam step applied where the aggregated gradient is non-zero:
     # theta, m, v bit-equal to the oracle's, untouched coordinates untouched, the scratch vector back to zero;
@@ -612,6 +612,48 @@ def test_sparse_adam_update_equals_the_oracles(workers):
         for s in streams:
             assert oracle.decompress_accumulate(s, n, po, dense) == 0
         assert np.array_equal(m0[dense == 0], om[dense == 0])
+
+
+@pytest.mark.parametrize("group_log2, workers, shift", [(14, 2, 1), (14, 4, 3), (16, 1, 0), (16, 4, 0), (12, 3, 0), (10, 2, 2)])
+def test_sparse_adam_update_other_group_sizes_and_unaligned_scratch(group_log2, workers, shift):
+    # the update in one launch on the paths that the usual layout does not reach: groups wider than the slice a block
+    # keeps in shared memory, a scratch vector that is not 16-byte aligned (both: aggregation in global memory, then
+    # every stream again for the update), narrow groups; a key shared by all workers; theta, m, v bit-equal to the oracle's
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(900 + 10 * group_log2 + workers)
+    n = 9 * 65536 + 4 * 777
+    grads = [workloads.student_t_layers(n, seed=70 + w, blocks=5, lo=1e-4, hi=1e-1) for w in range(workers)]
+    for g in grads[1:]:
+        g[::97] = grads[0][::97]
+    base = workloads.base_for_keep(grads[0], n // 12)
+    pg, po = binding.params(base, 128, 2, group_log2), oracle.params(base, 128, 2, group_log2)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    bufs = [G.Guarded(cap) for _ in range(workers)]
+    streams, sizes = [], []
+    for w in range(workers):
+        assert binding.compress(G.to_dev(grads[w]), pg, bufs[w].view) == 0
+        total, d, status = binding.stream_info(bufs[w].view)
+        assert status == 0 and d > 0
+        streams.append(bufs[w].view[:total].cpu().numpy()); sizes.append(total)
+    theta0 = rng.standard_normal(n).astype(np.float32)
+    m0 = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    v0 = (rng.standard_normal(n) ** 2 * 1e-6).astype(np.float32)
+    lr, b1, b2, eps = 3e-3, 0.8, 0.99, 1e-7
+    ot, om, ov = theta0.copy(), m0.copy(), v0.copy()
+    assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+    assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+    theta, m, v = (torch.from_numpy(x).to(G.dev()) for x in (theta0, m0, v0))
+    gs = G.Guarded(4 * (n + 4))
+    scratch = gs.view.view(torch.float32)[shift:shift + n]
+    for rep in range(2):
+        rc = binding.sparse_adam_update_batch([b.view for b in bufs], sizes, n, pg, binding.Adam(lr, b1, b2, eps),
+                                              scratch, theta, m, v)
+        assert rc == 0 and binding.decode_status() == 0 and gs.intact()
+        assert not bool(gs.view.any().item())
+    assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
+    assert 0 < int((ot != theta0).sum()) < n // 2
 
 
 def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
