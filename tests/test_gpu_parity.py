@@ -656,6 +656,52 @@ def test_sparse_adam_update_other_group_sizes_and_unaligned_scratch(group_log2, 
     assert 0 < int((ot != theta0).sum()) < n // 2
 
 
+@pytest.mark.parametrize("workers", [1, 3])
+def test_model_update_on_damaged_streams_reports_the_decoders_status_and_stays_in_bounds(workers):
+    # the one-launch update validates a group exactly as the aggregation does: on randomly damaged streams it reports
+    # the status the oracle's decoder reports for the same streams and writes nowhere outside theta, m, v and the scratch
+    import torch
+    import gpu_util as G
+    n = 6 * 16384 + 321
+    rng = np.random.default_rng(4100 + workers)
+    grads = [workloads.student_t_layers(n, seed=11 * w + 3, blocks=5, lo=1e-3, hi=1e-1) for w in range(workers)]
+    b = workloads.base_for_keep(grads[0], n // 30)
+    pg, po = _params(b)
+    binding.ensure_workspace(n, pg)
+    sound = [oracle.compress(v, po)[1] for v in grads]
+    fixed = 64 + 8 * 7
+    gt, gm, gv, gs = (G.Guarded(4 * n) for _ in range(4))
+    theta, m, v, scratch = (x.view.view(torch.float32) for x in (gt, gm, gv, gs))
+    h = binding.Adam(1e-3, 0.9, 0.999, 1e-8)
+    seen = set()
+    for case in range(36):
+        streams = [s.copy() for s in sound]
+        victim = case % workers
+        s = streams[victim]
+        region = case % 3
+        for _ in range(int(rng.integers(1, 4))):
+            pos = int(rng.integers(0, 64)) if region == 0 else (int(rng.integers(64, fixed)) if region == 1 else int(rng.integers(fixed, s.size)))
+            s[pos] ^= np.uint8(rng.integers(1, 256))
+        # the oracle's decoder, stream by stream: the first failing stream's status (streams are independent)
+        expect = 0
+        for t in streams:
+            st = oracle.decompress_accumulate(t, n, po, np.zeros(n, np.float32))
+            if st != 0 and expect == 0:
+                expect = st
+        bufs = [G.Guarded(t.size + (-t.size) % 16) for t in streams]
+        for bf, t in zip(bufs, streams):
+            bf.view[:t.size].copy_(torch.from_numpy(t))
+        for x in (theta, m, v, scratch):
+            x.zero_()
+        rc = binding.sparse_adam_update_batch([bf.view for bf in bufs], [t.size for t in streams], n, pg, h, scratch, theta, m, v)
+        assert rc == 0, case
+        st = binding.decode_status()
+        assert all(x.intact() for x in (gt, gm, gv, gs)) and all(bf.intact() for bf in bufs), case
+        assert st == expect, (case, st, expect)
+        seen.add(st)
+    assert len(seen) >= 3
+
+
 def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
     import torch
     import gpu_util as G
