@@ -990,7 +990,7 @@ __device__ __forceinline__ void sum_rest(CmpSmem& s, const CmpArgs& a, uint32_t 
 // is always listed, since whoever encodes it writes the header.  Returns the length of the list
 // (valid in thread 0).
 // The first kListAhead x 512 tiles' maxima, asked for before the partials are reduced (the two waits overlap).
-constexpr int kListAhead = 4;
+constexpr int kListAhead = 8;
 __device__ __forceinline__ void tile_maxima_ahead(const CmpArgs& a, float (&tm)[kListAhead], int tid) {
 #pragma unroll
     for (int j = 0; j < kListAhead; ++j) {
