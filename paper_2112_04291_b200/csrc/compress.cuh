@@ -1179,7 +1179,7 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         s.wait_limit = b.wait_limit; s.try_limit = b.try_limit;
         s.held[0] = 0xFFFFFFFFu; s.held[1] = 0xFFFFFFFFu;
         uint32_t team = 0u;
-        if (b.teams == 2u) {                  // (the host launches exactly two blocks per SM then)
+        if (SEVERAL && b.teams == 2u) {       // (the host launches exactly two blocks per SM then)
             unsigned int smid;
             asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
             team = atomicAdd(b.sm_slots + (smid & 255u), 1u) & 1u;
@@ -1187,14 +1187,15 @@ k_compress(const CmpBatch b, const __grid_constant__ PowTable pw) {
         s.team = team;
     }
     __syncthreads();
-    const uint32_t team = s.team, step = b.teams;
-    const uint32_t grid = gridDim.x / b.teams;              // blocks of a team
+    // (one gradient: no teams, nothing of the schedule below is compiled in)
+    const uint32_t team = SEVERAL ? s.team : 0u, step = SEVERAL ? b.teams : 1u;
+    const uint32_t grid = SEVERAL ? gridDim.x / b.teams : gridDim.x;              // blocks of a team
     // The team's own gradients: team, team + step, ...  With two teams, to keep their control steps
     // apart and their ends together: the blocks of team 1 first take up to two tiles each of
     // gradient 0's sum pass (so team 0 runs ahead), and the team that does not own the last
     // gradient H joins H's encode pass when it is done with its own.
-    const uint32_t nown = b.jobs > team ? (b.jobs - team + step - 1u) / step : 0u;
-    const uint32_t H = b.jobs - 1u;
+    const uint32_t nown = !SEVERAL ? 1u : (b.jobs > team ? (b.jobs - team + step - 1u) / step : 0u);
+    const uint32_t H = SEVERAL ? b.jobs - 1u : 0u;
     const bool helper = step == 2u && (H & 1u) != team;
     const uint32_t niter = nown + (helper ? 1u : 0u);
     uint32_t parity = 0;                      // bit st: parity the next wait on stage st expects

@@ -668,7 +668,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
     extern __shared__ __align__(128) unsigned char dec_smem_raw[];
     DecShared& s = *reinterpret_cast<DecShared*>(dec_smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t W = a.W;
+    const uint32_t W = ONE_STREAM ? 1u : a.W;         // (one stream: a constant, so that none of the many-stream code is compiled in)
 #ifdef FASTSGD_TRACE
     // per-block %globaltimer stamps: start, tables ready, own groups done, end; groups taken from the queue
     unsigned long long T0 = 0, T1 = 0, T2 = 0; unsigned int taken = 0;
