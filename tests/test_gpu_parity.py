@@ -702,6 +702,41 @@ def test_model_update_on_damaged_streams_reports_the_decoders_status_and_stays_i
     assert len(seen) >= 3
 
 
+def test_three_hundred_launches_in_a_row_give_the_same_bytes():
+    # every launch leaves the workspace as it found it: three gradients compressed in one launch, their streams decoded
+    # and the model updated, 300 times back to back with nothing but the outputs cleared in between -- the streams, the
+    # aggregated gradient and theta / m / v never differ from the first round's (which equal the oracle's)
+    import torch
+    import gpu_util as G
+    n = 1_500_007
+    host = [workloads.student_t_layers(n, seed=31 + w, blocks=6) for w in range(3)]
+    b = workloads.base_for_keep(host[0], n // 120)
+    pg, po = _params(b)
+    binding.ensure_workspace(n, pg)
+    grads = [G.to_dev(v) for v in host]
+    cap = binding.compress_bound(n, pg)
+    outs = [torch.zeros(cap, dtype=torch.uint8, device=G.dev()) for _ in range(3)]
+    dense, theta, m, v, scratch = (torch.zeros(n, dtype=torch.float32, device=G.dev()) for _ in range(5))
+    h = binding.Adam(1e-3, 0.9, 0.999, 1e-8)
+    ref = None
+    for it in range(300):
+        for t in outs + [dense, theta, m, v]:
+            t.zero_()
+        assert binding.compress_batch(grads, pg, outs) == 0
+        assert binding.decompress_accumulate_batch(outs, [cap] * 3, n, pg, dense) == 0
+        assert binding.sparse_adam_update_batch(outs, [cap] * 3, n, pg, h, scratch, theta, m, v) == 0
+        if ref is None:
+            assert binding.decode_status() == 0
+            for w in range(3):
+                orc, ostream = oracle.compress(host[w], po)
+                total, d, status = binding.stream_info(outs[w])
+                assert status == orc == 0 and np.array_equal(outs[w][:total].cpu().numpy(), ostream)
+            ref = [t.clone() for t in outs + [dense, theta, m, v]]
+        elif it % 10 == 9 or it < 5:
+            assert all(torch.equal(a, r) for a, r in zip(outs + [dense, theta, m, v], ref)), it
+            assert binding.decode_status() == 0 and not bool(scratch.any().item())
+
+
 def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
     import torch
     import gpu_util as G
