@@ -752,6 +752,17 @@ def main():
 
     adam_all()
     ms_adam = timed_flushed(adam_all, sub) / sub
+    # the same step on the state kept as (theta, m, v, g) per coordinate
+    adam_state = torch.zeros(4 * n, dtype=torch.float32, device=dev)
+
+    def adam_packed():
+        rc = binding.sparse_adam_update_packed_batch(outs, [cap] * W, n, pg, hyper, adam_state)
+        if rc:
+            raise binding.FastSGDError(rc, "fastsgd_sparse_adam_update_packed_batch")
+
+    adam_packed()
+    ms_adam_packed = timed_flushed(adam_packed, sub) / sub
+    del adam_state
     assert binding.decode_status() == 0
     del theta, adam_m, adam_v, adam_g
 
@@ -868,7 +879,8 @@ def main():
                        "sector_bytes": float(sum(stream_bytes)) + 64.0 * float(sum(kept)),
                        "sector_gbs": (float(sum(stream_bytes)) + 64.0 * float(sum(kept))) / (ms_dec * 1e-3) / 1e9},
         "dense_zero_fill_ms": ms_zero,
-        "sparse_adam_update": {"ms": ms_adam, "touched_bytes": float(sum(stream_bytes)) + 40.0 * float(sum(kept)),
+        "sparse_adam_update": {"ms": ms_adam, "packed_state_ms": ms_adam_packed,
+                               "touched_bytes": float(sum(stream_bytes)) + 40.0 * float(sum(kept)),
                                "note": "decode + Adam step on decoded coordinates only; one launch (up to 8 streams); "
                                        "256 MiB written before every call; not part of value / ms_per_step"},
         "compress_kv": kv_info,

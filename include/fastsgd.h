@@ -237,6 +237,24 @@ int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64
                                      float* theta, float* m, float* v, void* stream);
 
 /*
+ * The same update with the model's state kept as one array of four floats per
+ * coordinate, (theta, m, v, g): a coordinate's step then reads and writes one
+ * 16-byte entry instead of one 32-byte sector in each of three arrays (the
+ * update of scattered coordinates is bound by memory transactions, Sec. 4.1's
+ * "model updating" part).  g is the scratch of the call above, interleaved.
+ *   state        device, 16-byte aligned, 4 n floats: state[4 i + 0] = theta_i,
+ *                [4 i + 1] = m_i, [4 i + 2] = v_i, [4 i + 3] = g_i; every g_i
+ *                ZERO on entry and zero again when the call has run
+ *   other arguments, the arithmetic, the order of the streams, errors and
+ *                damaged streams: as for fastsgd_sparse_adam_update_batch
+ * One launch.  At most 8 streams and groups of at most 2^14 indices
+ * (group_log2 <= 14): otherwise FASTSGD_E_NOT_IMPLEMENTED.
+ */
+int fastsgd_sparse_adam_update_packed_batch(const void* const* streams_in, const uint64_t* bytes,
+                                            uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                            const fastsgd_adam* hyper, float* state, void* stream);
+
+/*
  * Algorithm 2 exactly as printed (Sec. 3.3): one delta chain over all kept keys
  * starting from preKey = 0, one M = max(1, bitlen(maxDelta)), and the binary
  * sequence BK = flag || delta for each key in turn, most significant bit first

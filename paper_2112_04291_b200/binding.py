@@ -28,7 +28,7 @@ EXPORTS = [
     "fastsgd_decode_status", "fastsgd_abs_sum", "fastsgd_host_scratch_bytes",
     "fastsgd_compress_host", "fastsgd_decompress_accumulate_host", "fastsgd_launch_count",
     "fastsgd_strerror", "fastsgd_version", "fastsgd_kernel_timing_enable", "fastsgd_kernel_timing_read", "fastsgd_abs_sum_noalloc",
-    "fastsgd_sparse_adam_update_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
+    "fastsgd_sparse_adam_update_batch", "fastsgd_sparse_adam_update_packed_batch", "fastsgd_key_encode_paper", "fastsgd_key_encode_paper_bound",
     "fastsgd_compress_kv",
     "fastsgd_debug_set_wait_limits", "fastsgd_debug_layout", "fastsgd_debug_trace_compiled", "fastsgd_debug_set_grid",
 ]
@@ -83,6 +83,8 @@ def lib():
         L.fastsgd_key_encode_paper.argtypes = [vp, u64, C.c_uint32, vp, u64, vp]
         L.fastsgd_sparse_adam_update_batch.restype = C.c_int
         L.fastsgd_sparse_adam_update_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, C.POINTER(Adam), vp, vp, vp, vp, vp]
+        L.fastsgd_sparse_adam_update_packed_batch.restype = C.c_int
+        L.fastsgd_sparse_adam_update_packed_batch.argtypes = [C.POINTER(vp), u64p, C.c_uint32, u64, PP, C.POINTER(Adam), vp, vp]
         L.fastsgd_compress_bound.restype = u64
         L.fastsgd_compress_bound.argtypes = [u64, PP]
         L.fastsgd_workspace_bytes.restype = u64
@@ -222,6 +224,17 @@ def sparse_adam_update_batch(streams_in, nbytes, n: int, p: Params, hyper: Adam,
     sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
     return lib().fastsgd_sparse_adam_update_batch(ptrs, sizes, k, int(n), C.byref(p), C.byref(hyper), grad_scratch.data_ptr(),
                                                   theta.data_ptr(), m.data_ptr(), v.data_ptr(), _stream_handle(stream))
+
+
+def sparse_adam_update_packed_batch(streams_in, nbytes, n: int, p: Params, hyper: Adam, state: torch.Tensor, stream=None) -> int:
+    """fastsgd_sparse_adam_update_packed_batch: the same step on the state kept as (theta, m, v, g) per coordinate."""
+    assert state.is_cuda and state.dtype == torch.float32 and state.is_contiguous() and state.numel() == 4 * n
+    k = len(streams_in)
+    assert all(s.is_cuda and s.dtype == torch.uint8 for s in streams_in) and len(nbytes) == k
+    ptrs = (C.c_void_p * k)(*[int(s.data_ptr()) for s in streams_in])
+    sizes = (C.c_uint64 * k)(*[int(b) for b in nbytes])
+    return lib().fastsgd_sparse_adam_update_packed_batch(ptrs, sizes, k, int(n), C.byref(p), C.byref(hyper), state.data_ptr(),
+                                                         _stream_handle(stream))
 
 
 def compress_kv(keys: torch.Tensor, values: torch.Tensor, n: int, p: Params, out: torch.Tensor, stream=None) -> int:

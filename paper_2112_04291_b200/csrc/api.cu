@@ -175,16 +175,22 @@ int ensure_device_setup() {
         return FASTSGD_E_CUDA;
     if (cudaFuncSetAttribute(k_decode_accumulate<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
         return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<false, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_accumulate<true, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecShared)) != cudaSuccess)
+        return FASTSGD_E_CUDA;
     {   // every instantiation must be resident with the grid the launch uses (the queue of large groups relies on it)
-        int b2x[6] = {0, 0, 0, 0, 0, 0};
+        int b2x[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[0], k_decode_accumulate<false>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[1], k_decode_accumulate<true>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[2], k_decode_accumulate<false, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[3], k_decode_accumulate<true, 1>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[4], k_decode_accumulate<false, 2>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[5], k_decode_accumulate<true, 2>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[6], k_decode_accumulate<false, 3>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2x[7], k_decode_accumulate<true, 3>, kDecThreads, sizeof(DecShared)) != cudaSuccess) return FASTSGD_E_CUDA;
         b2 = b2x[0];
-        for (int i = 1; i < 6; ++i) if (b2x[i] < b2) b2 = b2x[i];
+        for (int i = 1; i < 8; ++i) if (b2x[i] < b2) b2 = b2x[i];
     }
     g_state.sm_count = sms;
     g_state.sum_blocks_per_sm = b1 > 0 ? b1 : 1;
@@ -541,8 +547,9 @@ namespace {
 // launch's worth of streams, dense_out all zero), aggregation and update in the same launch.
 int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32_t num_streams, uint64_t n,
                     const fastsgd_params* params, float* dense_out, const fastsgd_adam* adam,
-                    float* theta, float* m, float* v, void* stream, bool fused = false) {
+                    float* theta, float* m, float* v, void* stream, bool fused = false, bool packed = false) {
     if (fused && (!adam || num_streams > (uint32_t)kDecMaxStreams)) return FASTSGD_E_BAD_PARAM;
+    if (packed && !fused) return FASTSGD_E_BAD_PARAM;
     if (!streams_in || !bytes || !dense_out || !params) return FASTSGD_E_NULL;
     if (!aligned(dense_out, 4)) return FASTSGD_E_ALIGN;
     PowTable pw;
@@ -597,7 +604,10 @@ int decode_launches(const void* const* streams_in, const uint64_t* bytes, uint32
         }
         {
             LaunchTimer lt(2, st);
-            if (fused) {
+            if (packed) {
+                if (da.W == 1u) k_decode_accumulate<true, 3><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+                else k_decode_accumulate<false, 3><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
+            } else if (fused) {
                 if (da.W == 1u) k_decode_accumulate<true, 2><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
                 else k_decode_accumulate<false, 2><<<(unsigned)grid, kDecThreads, sizeof(DecShared), st>>>(da, pw);
             } else if (adam) {
@@ -634,6 +644,17 @@ int fastsgd_sparse_adam_update_batch(const void* const* streams_in, const uint64
     int rc = decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, nullptr, nullptr, nullptr, nullptr, stream);
     if (rc) return rc;
     return decode_launches(streams_in, bytes, num_streams, n, params, grad_scratch, hyper, theta, m, v, stream);
+}
+
+int fastsgd_sparse_adam_update_packed_batch(const void* const* streams_in, const uint64_t* bytes,
+                                            uint32_t num_streams, uint64_t n, const fastsgd_params* params,
+                                            const fastsgd_adam* hyper, float* state, void* stream) {
+    if (!hyper || !state || !params) return FASTSGD_E_NULL;
+    if (!aligned(state, 16)) return FASTSGD_E_ALIGN;
+    // (the update of a group lives in the 64 KiB slice of shared memory of the block that decodes it: groups of up to 2^14
+    //  indices, one launch's worth of streams)
+    if (params->group_log2 > 14u || num_streams > (uint32_t)kDecMaxStreams) return FASTSGD_E_NOT_IMPLEMENTED;
+    return decode_launches(streams_in, bytes, num_streams, n, params, state, hyper, nullptr, nullptr, nullptr, stream, true, true);
 }
 
 uint64_t fastsgd_key_encode_paper_bound(uint64_t d, uint32_t flag_bits) {

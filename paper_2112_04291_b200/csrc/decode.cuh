@@ -58,6 +58,15 @@ struct DecArgs {
     float               lr, beta1, beta2, eps;
 };
 
+// Modes of the decoder (template parameter MODE): 0 aggregation; 1 model update as a pass of its own; 2 both in one
+// launch; 3 both in one launch on the packed state (theta, m, v, g per coordinate, g where dense_out[i] would be);
+// 4 and 5: what 0 and 1 are to 2, for 3 (a group whose streams do not fit one decode_multi call).
+__host__ __device__ constexpr bool mode_packed(int mode) { return mode >= 3; }
+__host__ __device__ constexpr bool mode_fused(int mode) { return mode == 2 || mode == 3; }
+__host__ __device__ constexpr int mode_apply(int mode) { return (mode == 1 || mode == 5) ? 1 : 0; }       // what apply_run does in the first sweep
+// index of coordinate k's entry of dense_out (g) as a float
+template <int MODE> __device__ __forceinline__ uint32_t dense_at(uint32_t k) { return mode_packed(MODE) ? 4u * k + 3u : k; }
+
 // What a thread's run of K decoded (key, value) pairs does to the entries `cur` of dense_out at those keys
 // (distinct; 0xFFFFFFFF: no key); the results are stored there by the caller.
 // MODE 0: aggregation, cur + value.  MODE 1: model update: `cur` is the aggregated gradient g at that
@@ -65,12 +74,34 @@ struct DecArgs {
 // Adam step (the experimental set-up's equations, no bias correction; one IEEE fp32 operation at a
 // time) and g returns to zero, so that a key that several streams hold is updated once.  All loads of
 // the moments and the parameters are issued before the first of them is needed.
-template <int MODE, int K>
+// PACKED: the model's state is one array of (theta, m, v, g) per coordinate (dense_out points at it): one 16-byte
+// load and one 16-byte store per updated coordinate instead of three sectors read and written.
+template <int MODE, int K, bool PACKED = false>
 __device__ __forceinline__ void apply_run(const DecArgs& a, const uint32_t (&kk)[K], const float (&cur)[K],
                                           const float (&value)[K], float (&res)[K]) {
     if (MODE == 0) {
 #pragma unroll
         for (int k = 0; k < K; ++k) res[k] = __fadd_rn(cur[k], value[k]);
+        return;
+    }
+    if constexpr (PACKED) {
+        float4* state = reinterpret_cast<float4*>(a.dense);
+        float4 st[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const bool on = kk[k] != 0xFFFFFFFFu && cur[k] != 0.0f;
+            st[k] = on ? state[kk[k]] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            if (kk[k] != 0xFFFFFFFFu && cur[k] != 0.0f) {
+                const float mk = __fadd_rn(__fmul_rn(a.beta1, st[k].y), __fmul_rn(__fsub_rn(1.0f, a.beta1), cur[k]));
+                const float vk = __fadd_rn(__fmul_rn(a.beta2, st[k].z), __fmul_rn(__fsub_rn(1.0f, a.beta2), __fmul_rn(cur[k], cur[k])));
+                const float step = __fdiv_rn(a.lr, __fsqrt_rn(__fadd_rn(vk, a.eps)));
+                state[kk[k]] = make_float4(__fsub_rn(st[k].x, __fmul_rn(step, mk)), mk, vk, 0.0f);
+            }
+            res[k] = 0.0f;
+        }
         return;
     }
     float pm[K], pv[K], pt[K];
@@ -538,15 +569,15 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
         if (BLOCK && tile != nullptr) {
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? tile[kk[k] - lo[w]] : 0.f;
-            apply_run<(MODE == 2 ? 0 : MODE), KMAX>(a, kk, dd, vv, res);
+            apply_run<mode_apply(MODE), KMAX, mode_packed(MODE)>(a, kk, dd, vv, res);
 #pragma unroll
             for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) tile[kk[k] - lo[w]] = res[k];
         } else {
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[kk[k]] : 0.f;
-            apply_run<(MODE == 2 ? 0 : MODE), KMAX>(a, kk, dd, vv, res);
+            for (int k = 0; k < KMAX; ++k) dd[k] = kk[k] != 0xFFFFFFFFu ? a.dense[dense_at<MODE>(kk[k])] : 0.f;
+            apply_run<mode_apply(MODE), KMAX, mode_packed(MODE)>(a, kk, dd, vv, res);
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[kk[k]] = res[k];
+            for (int k = 0; k < KMAX; ++k) if (kk[k] != 0xFFFFFFFFu) a.dense[dense_at<MODE>(kk[k])] = res[k];
         }
     }
 
@@ -555,7 +586,7 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
     // dense_out by an atomic exchange with 0: of the streams that hold a key the one that gets there first
     // receives g and updates the coordinate, the others receive 0 (whichever it is, the result is the same);
     // no stream waits for another, and all the exchanges are in flight together.
-    if constexpr (MODE == 2) {
+    if constexpr (mode_fused(MODE)) {
         static_assert(!BLOCK, "the block path updates from its slice in shared memory");
         if (first) return;                                     // (uniform) nothing was applied
         __syncwarp();
@@ -572,14 +603,14 @@ __device__ __forceinline__ void decode_multi(const DecArgs& a, DecShared& s, con
             }
         }
 #pragma unroll
-        for (int i = 0; i < KA; ++i) ga[i] = ka[i] != 0xFFFFFFFFu ? atomicExch(a.dense + ka[i], 0.0f) : 0.0f;
+        for (int i = 0; i < KA; ++i) ga[i] = ka[i] != 0xFFFFFFFFu ? atomicExch(a.dense + dense_at<MODE>(ka[i]), 0.0f) : 0.0f;
         constexpr int KB = KA < 8 ? KA : 8;                    // moments and parameters of eight keys loaded at a time
 #pragma unroll
         for (int i0 = 0; i0 < KA; i0 += KB) {
             uint32_t kb[KB]; float gb[KB], vb[KB], rb[KB];
 #pragma unroll
             for (int i = 0; i < KB; ++i) { kb[i] = ka[i0 + i]; gb[i] = ga[i0 + i]; vb[i] = 0.0f; }
-            apply_run<1, KB>(a, kb, gb, vb, rb);
+            apply_run<1, KB, mode_packed(MODE)>(a, kb, gb, vb, rb);
         }
     }
 }
@@ -639,10 +670,10 @@ __device__ __forceinline__ void warp_fours(const DecArgs& a, DecShared& s, const
 // (0: aggregation over all the group's calls, then 1: the update over all of them again).
 #define FSG_DECODE_MULTI(fused, B_, NS_, K_, TG_, ...)                                        \
     do {                                                                                      \
-        if constexpr (MODE == 2) {                                                            \
-            if (fused) decode_multi<2, B_, NS_, K_, TG_>(__VA_ARGS__);                        \
-            else if (pass == 0) decode_multi<0, B_, NS_, K_, TG_>(__VA_ARGS__);               \
-            else decode_multi<1, B_, NS_, K_, TG_>(__VA_ARGS__);                              \
+        if constexpr (mode_fused(MODE)) {                                                     \
+            if (fused) decode_multi<MODE, B_, NS_, K_, TG_>(__VA_ARGS__);                     \
+            else if (pass == 0) decode_multi<(MODE == 3 ? 4 : 0), B_, NS_, K_, TG_>(__VA_ARGS__);  \
+            else decode_multi<(MODE == 3 ? 5 : 1), B_, NS_, K_, TG_>(__VA_ARGS__);            \
         } else {                                                                              \
             decode_multi<MODE, B_, NS_, K_, TG_>(__VA_ARGS__);                                \
         }                                                                                     \
@@ -651,9 +682,9 @@ __device__ __forceinline__ void warp_fours(const DecArgs& a, DecShared& s, const
 // (the same without the fused form: the block path, whose mode 2 keeps the slice of g in shared memory)
 #define FSG_DECODE_MULTI_PASS(B_, NS_, K_, TG_, ...)                                          \
     do {                                                                                      \
-        if constexpr (MODE == 2) {                                                            \
-            if (pass == 0) decode_multi<0, B_, NS_, K_, TG_>(__VA_ARGS__);                    \
-            else decode_multi<1, B_, NS_, K_, TG_>(__VA_ARGS__);                              \
+        if constexpr (mode_fused(MODE)) {                                                     \
+            if (pass == 0) decode_multi<(MODE == 3 ? 4 : 0), B_, NS_, K_, TG_>(__VA_ARGS__);  \
+            else decode_multi<(MODE == 3 ? 5 : 1), B_, NS_, K_, TG_>(__VA_ARGS__);            \
         } else {                                                                              \
             decode_multi<MODE, B_, NS_, K_, TG_>(__VA_ARGS__);                                \
         }                                                                                     \
@@ -661,7 +692,7 @@ __device__ __forceinline__ void warp_fours(const DecArgs& a, DecShared& s, const
 
 // ONE_STREAM: the launch holds a single stream (its own instantiation, so that the code of the
 // many-stream paths and of the two-groups-per-warp path do not weigh on each other)
-// MODE: what a decoded value does to dense_out (apply_value): 0 aggregation, 1 model update.
+// MODE: what a decoded value does to dense_out: 0 aggregation, 1 model update, 2 both, 3 both on the packed state (see mode_packed).
 template <bool ONE_STREAM, int MODE = 0>
 __global__ void __launch_bounds__(kDecThreads, 2)
 k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
@@ -807,8 +838,8 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         __syncwarp();
         if (__any_sync(kFullMask, count > kDecWarpSide)) {
             // longer runs per lane: two streams at a time
-            const bool fused = MODE == 2 && W <= 2u;
-            const int npass = (MODE == 2 && !fused) ? 2 : 1;
+            const bool fused = mode_fused(MODE) && W <= 2u;
+            const int npass = (mode_fused(MODE) && !fused) ? 2 : 1;
             for (int pass = 0; pass < npass; ++pass)
             for (uint32_t w0 = 0; w0 < W; w0 += 2u) {
                 const uint32_t w1 = w0 + 1u < W ? w0 + 1u : w0;
@@ -827,11 +858,11 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 __syncwarp();      // these streams' stores before the next streams' loads of the same keys
             }
         } else {
-            if constexpr (MODE == 2) {
-                if (W <= 4u) warp_fours<2>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+            if constexpr (mode_fused(MODE)) {
+                if (W <= 4u) warp_fours<MODE>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
                 else {      // the update only after every stream's values are in
-                    warp_fours<0>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
-                    warp_fours<1>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+                    warp_fours<(MODE == 3 ? 4 : 0)>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
+                    warp_fours<(MODE == 3 ? 5 : 1)>(a, s, stage, count, M, base, nwords, W, g, lane, warp);
                 }
             } else {
         // up to four streams at a time, parsed side by side and applied in stream order
@@ -909,16 +940,19 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
         const uint32_t lo = (uint32_t)lo64, span = (uint32_t)((hi64 < a.n ? hi64 : a.n) - lo64);
         // The group's slice of dense_out is brought into shared memory by one bulk copy, updated there by
         // every stream in turn, and written back by one bulk copy (needs 16-byte alignment and size).
-        const bool use_tile = a.group_log2 <= 14u && ((reinterpret_cast<uintptr_t>(a.dense) & 15u) == 0u) && ((span & 3u) == 0u);
-        // (MODE 2: dense_out is all zero by contract and is left so: the slice starts as zeros in shared memory and never leaves it)
-        const bool load_tile = use_tile && MODE != 2;
+        // (packed state: the slice of g is only ever formed in shared memory, so the copies' alignment rules do not matter;
+        //  the host admits no wider groups there)
+        const bool use_tile = a.group_log2 <= 14u &&
+                              (MODE == 3 || (((reinterpret_cast<uintptr_t>(a.dense) & 15u) == 0u) && ((span & 3u) == 0u)));
+        // (modes 2 and 3: g is all zero by contract and is left so: the slice starts as zeros in shared memory and never leaves it)
+        const bool load_tile = use_tile && !mode_fused(MODE);
         if (load_tile && tid == 0) {
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the last write-back has read the tile
             mbar_expect_tx(&s.tile_bar, span * 4u);
             bulk_load(s.u.tile, a.dense + lo, span * 4u, &s.tile_bar);
         }
-        if (MODE == 2 && use_tile)
-            for (uint32_t i = tid; i < (span >> 2); i += kDecThreads)
+        if (mode_fused(MODE) && use_tile)
+            for (uint32_t i = tid; i < ((span + 3u) >> 2); i += kDecThreads)
                 reinterpret_cast<float4*>(s.u.tile)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (!local && tid < (int)W) {
             uint32_t count = 0, M = 0, off = 0, nwords = 0;
@@ -958,7 +992,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
             }
         }
         // MODE 2 without the slice in shared memory: every stream aggregated into dense_out, then every stream again for the update
-        const int npass = (MODE == 2 && !use_tile) ? 2 : 1;
+        const int npass = (mode_fused(MODE) && !use_tile) ? 2 : 1;
         if (parse)
         for (int pass = 0; pass < npass; ++pass)
         for (uint32_t w = 0; w < W; ++w) {
@@ -982,7 +1016,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                 const float* v1[1] = {s.val[w]};
                 FSG_DECODE_MULTI_PASS(true, 1, 4, false, a, s, b1, n1, c1, m1, v1, g, use_tile ? s.u.tile : nullptr, tid, kDecThreads, lane, warp);
             } else {
-                if constexpr (MODE == 2) {
+                if constexpr (mode_fused(MODE)) {
                     if (pass == 0) decode_long<0>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
                                                   tid, kDecThreads, lane, warp);
                     else decode_long<1>(a, s, blob, s.g_nwords[w], g, c, s.g_M[w], s.val[w], use_tile ? s.u.tile : nullptr,
@@ -1004,7 +1038,7 @@ k_decode_accumulate(const DecArgs a, const __grid_constant__ PowTable pw) {
                     kk[u] = cur[u] != 0.0f ? lo + idx : 0xFFFFFFFFu;
                     vv[u] = 0.0f;
                 }
-                apply_run<1, 8>(a, kk, cur, vv, res);
+                apply_run<1, 8, mode_packed(MODE)>(a, kk, cur, vv, res);
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
                     if (kk[u] != 0xFFFFFFFFu) s.u.tile[i0 + (uint32_t)u * (uint32_t)kDecThreads + (uint32_t)tid] = res[u];

@@ -673,6 +673,7 @@ def test_model_update_on_damaged_streams_reports_the_decoders_status_and_stays_i
     gt, gm, gv, gs = (G.Guarded(4 * n) for _ in range(4))
     theta, m, v, scratch = (x.view.view(torch.float32) for x in (gt, gm, gv, gs))
     h = binding.Adam(1e-3, 0.9, 0.999, 1e-8)
+    gstate = G.Guarded(16 * n)
     seen = set()
     for case in range(36):
         streams = [s.copy() for s in sound]
@@ -699,6 +700,11 @@ def test_model_update_on_damaged_streams_reports_the_decoders_status_and_stays_i
         assert all(x.intact() for x in (gt, gm, gv, gs)) and all(bf.intact() for bf in bufs), case
         assert st == expect, (case, st, expect)
         seen.add(st)
+        # the same streams through the call on the packed state
+        gstate.view.zero_()
+        rc = binding.sparse_adam_update_packed_batch([bf.view for bf in bufs], [t.size for t in streams], n, pg, h,
+                                                     gstate.view.view(torch.float32))
+        assert rc == 0 and binding.decode_status() == expect and gstate.intact() and all(bf.intact() for bf in bufs), case
     assert len(seen) >= 3
 
 
@@ -735,6 +741,54 @@ def test_three_hundred_launches_in_a_row_give_the_same_bytes():
         elif it % 10 == 9 or it < 5:
             assert all(torch.equal(a, r) for a, r in zip(outs + [dense, theta, m, v], ref)), it
             assert binding.decode_status() == 0 and not bool(scratch.any().item())
+
+
+@pytest.mark.parametrize("workers, n", [(1, 41 * 16384 - 1234), (2, 9 * 16384 + 3), (4, 41 * 16384 - 1234), (8, 20 * 16384 + 1)])
+def test_model_update_on_the_packed_state_equals_the_oracles(workers, n):
+    # the same step with theta, m, v and the scratch g interleaved four floats to a coordinate: theta, m, v bit-equal to
+    # the oracle's on its three arrays, every g back to zero, two steps in a row, groups of every density, a last group
+    # whose length is no multiple of four, keys shared by all workers, two workers that cancel
+    import torch
+    import gpu_util as G
+    rng = np.random.default_rng(5200 + workers)
+    grads = [workloads.student_t_layers(n, seed=90 + w, blocks=7, lo=1e-4, hi=1e-1) for w in range(workers)]
+    for g in grads[1:]:
+        g[::101] = grads[0][::101]
+    if workers >= 4:
+        grads[3] = -grads[1]
+    base = workloads.base_for_keep(grads[0], n // 25)
+    pg, po = _params(base)
+    binding.ensure_workspace(n, pg)
+    cap = binding.compress_bound(n, pg)
+    bufs = [G.Guarded(cap) for _ in range(workers)]
+    assert binding.compress_batch([G.to_dev(v) for v in grads], pg, [b.view for b in bufs]) == 0
+    streams, sizes = [], []
+    for b in bufs:
+        total, d, status = binding.stream_info(b.view)
+        assert status == 0
+        streams.append(b.view[:total].cpu().numpy()); sizes.append(total)
+    theta0 = rng.standard_normal(n).astype(np.float32)
+    m0 = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    v0 = (rng.standard_normal(n) ** 2 * 1e-6).astype(np.float32)
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    ot, om, ov = theta0.copy(), m0.copy(), v0.copy()
+    gstate = G.Guarded(16 * n)
+    state = gstate.view.view(torch.float32)
+    host = np.zeros((n, 4), np.float32)
+    host[:, 0], host[:, 1], host[:, 2] = theta0, m0, v0
+    state.copy_(torch.from_numpy(host.reshape(-1)))
+    for rep in range(2):
+        assert oracle.sparse_adam_update(streams, n, po, lr, b1, b2, eps, ot, om, ov) == 0
+        rc = binding.sparse_adam_update_packed_batch([b.view for b in bufs], sizes, n, pg, binding.Adam(lr, b1, b2, eps), state)
+        assert rc == 0 and binding.decode_status() == 0 and gstate.intact()
+        got = state.cpu().numpy().reshape(n, 4)
+        assert not got[:, 3].any()
+        assert np.array_equal(got[:, 0], ot) and np.array_equal(got[:, 1], om) and np.array_equal(got[:, 2], ov)
+    assert 0 < int((ot != theta0).sum()) < n // 2
+    # what the call does not take
+    p16 = binding.params(base, 128, 2, 16)
+    binding.ensure_workspace(n, p16)
+    assert binding.sparse_adam_update_packed_batch([b.view for b in bufs], sizes, n, p16, binding.Adam(lr, b1, b2, eps), state) == binding.E_NOT_IMPLEMENTED
 
 
 def test_sparse_adam_update_single_stream_with_dense_tiles_and_bad_arguments():
