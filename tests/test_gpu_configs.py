@@ -216,6 +216,14 @@ def test_config2_sparse_adam_update_as_benchmarked():
     assert binding.decode_status() == 0 and not bool(scratch.any().item())
     assert np.array_equal(theta.cpu().numpy(), ot) and np.array_equal(m.cpu().numpy(), om) and np.array_equal(v.cpu().numpy(), ov)
     assert 0 < int((ot != theta0).sum()) <= 4 * n // 100
+    # the same step on the packed state (theta, m, v, g per coordinate), as bench.py's packed_state_ms times it
+    host = np.zeros((n, 4), np.float32)
+    host[:, 0] = theta0
+    state = torch.from_numpy(host.reshape(-1)).cuda()
+    assert binding.sparse_adam_update_packed_batch(outs, [cap] * W, n, pg, binding.Adam(lr, b1, b2, eps), state) == 0
+    got = state.cpu().numpy().reshape(n, 4)
+    assert binding.decode_status() == 0 and not got[:, 3].any()
+    assert np.array_equal(got[:, 0], ot) and np.array_equal(got[:, 1], om) and np.array_equal(got[:, 2], ov)
 
 
 def test_config3_key_value_input_as_benchmarked():
